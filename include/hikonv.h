@@ -1,0 +1,196 @@
+/*
+ * hikonv.h - C interface of the packed low-bit convolution library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes 1-D and 2-D convolutions of 1..8-bit quantised codes by packing
+ * N activations and K weights into two 32-bit words with S-bit slots, so that ONE
+ * 32x32->64 multiply yields N+K-1 partial convolution sums (Theorem 1), which are
+ * overlap-added across blocks (Theorem 2), accumulated over input channels and kernel
+ * rows while still packed (Theorem 3, the DNN guard-bit rule), then split into int32
+ * (Algorithm 2 / Eq. 29) and optionally requantised.
+ *
+ * Conventions for every entry point
+ *   - Codes are stored one per byte (int8_t).  A signed p-bit code is its int8 value; an
+ *     unsigned p-bit code is the byte read as uint8 (so unsigned 8-bit codes use all 256
+ *     byte values).  Codes are ASSUMED to lie in their p-bit range; a code outside it
+ *     silently breaks the guard bits.
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  All memory is owned
+ *     by the caller; the library allocates nothing and keeps no pointer after a call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device
+ *     entry points enqueue their kernels on it and return without synchronising.
+ *   - Every function returns a hikonv_status (as int); nothing aborts, nothing traps on
+ *     the device.  Arguments are validated on the host before any launch.
+ *   - There is no CPU fallback: without a CUDA device the device entry points return
+ *     HIKONV_ERR_CUDA.
+ */
+#ifndef HIKONV_H
+#define HIKONV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HIKONV_OK = 0,
+    HIKONV_ERR_INVALID_ARG = 1, /* null pointer, p/q outside 1..8, K < 1, sizes < 0, bad enum        */
+    HIKONV_ERR_UNSUPPORTED = 2, /* stride != 1, an algorithm that is not built, pad >= K               */
+    HIKONV_ERR_NO_FIT = 3,      /* no (N >= 1, S) satisfies the operand, slot and accumulator bounds   */
+    HIKONV_ERR_WORKSPACE = 4,   /* workspace pointer null/misaligned or workspace_bytes too small      */
+    HIKONV_ERR_CUDA = 5         /* a CUDA runtime call failed (see cudaGetLastError)                   */
+} hikonv_status;
+
+typedef enum {
+    HIKONV_ALGO_PACKED32 = 0,      /* packed operands, 32x32->64 multiply (mad.wide)                    */
+    HIKONV_ALGO_PACKED64EMU = 1,   /* 64x64 multiplier emulated from 32-bit pieces: not built           */
+    HIKONV_ALGO_UNPACKED_IMAD = 2  /* comparator: one product per 32-bit multiply-add, int32 accumulate */
+} hikonv_algo;
+
+typedef enum {
+    HIKONV_GB_SINGLE = 0, /* Eq. 11: Gb = ceil(log2 min(K, N))          */
+    HIKONV_GB_1D = 1,     /* 1-D extension: Gb = ceil(log2 K)            */
+    HIKONV_GB_DNN = 2     /* DNN extension: Gb = ceil(log2(M min(K, N))) */
+} hikonv_gb_mode;
+
+/* Result of the paper's throughput search (Algorithm 1). */
+typedef struct {
+    int N;   /* activations per packed word            */
+    int K;   /* weights per packed word                */
+    int S;   /* slot width in bits (Eq. 6)             */
+    int Gb;  /* guard bits of the chosen pair          */
+    int ops; /* N K + (N-1)(K-1), Eq. 24               */
+} hikonv_plan_t;
+
+/* The layout the CUDA kernels actually run with (exact value-range analysis, see below). */
+typedef struct {
+    int N;           /* activations per 32-bit word A                                        */
+    int S;           /* slot width                                                            */
+    int Kc;          /* weights per 32-bit word B (taps per chunk)                            */
+    int J;           /* number of weight chunks, ceil(K / Kc); J > 1 implies Kc == N          */
+    int segments;    /* N + Kc - 1 slots of the 64-bit product                                */
+    int top_bits;    /* width of the highest slot, 64 - S (segments - 1), capped at S         */
+    int M;           /* products that may be summed in the 64-bit accumulator before a split  */
+    int signed_prod; /* 1 when either operand is signed (signed multiply, biased split)       */
+    int S_paper;     /* Eq. 6 with the mode's guard bits, for reference                       */
+} hikonv_layout_t;
+
+/* Optional overrides for experiments and tests; zero in a field means "choose automatically".
+ * Pass NULL for fully automatic behaviour. */
+typedef struct {
+    int N;          /* force activations per word                                   */
+    int S;          /* force slot width                                             */
+    int M;          /* force the number of accumulated products between two splits  */
+    int tile;       /* kernel-specific tile selector (0 = automatic)                */
+} hikonv_tuning_t;
+
+/*
+ * hikonv_plan - the paper's configuration search (Section IV-D, Algorithm 1; host only).
+ * Maximises Eq. 24 over (N, K) subject to Eq. 7-8 with S from Eq. 6 and the guard bits of
+ * `mode` (hikonv_gb_mode; M is the number of accumulated feature maps, used by the DNN rule).
+ * K_fixed > 0 fixes the kernel length and searches N only.  LA, LB are the multiplier's
+ * operand widths (1..64).  The search ranges are inclusive (the printed strict bounds cannot
+ * reproduce the paper's own counts).  Returns HIKONV_ERR_NO_FIT when not even N = K = 1 fits.
+ */
+int hikonv_plan(int p, int q, int LA, int LB, int mode, int M, int K_fixed, hikonv_plan_t *out);
+
+/*
+ * hikonv_layout - the packed layout used by the CUDA kernels for a 32x32->64 multiplier (host only).
+ * Starts from the paper's slot width (Eq. 6 with Gb = ceil(log2 K) for dims == 1, Theorem 2) and
+ * verifies it against the exact value ranges of the codes: both packed operands must fit a 32-bit
+ * register (31 bits for an unsigned operand of a signed multiply), every slot must hold the
+ * extreme sum it can receive, and the top slot must fit what is left of 64 bits.  S is widened
+ * when the printed rule is too small (signed 1-bit codes).  For dims == 2 (Theorem 3, Eq. 23)
+ * S is chosen as large as N allows so that M, the number of (channel, kernel-row) products
+ * accumulated before a split, is as large as possible, and N is chosen by a cost model.
+ * K taps that do not fit one word are cut into J chunks of N taps (Theorem 2 applied to the
+ * kernel).  `total_terms` is Ci*K for dims == 2 (ignored for dims == 1); `tune` may be NULL.
+ */
+int hikonv_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int total_terms,
+                  const hikonv_tuning_t *tune, hikonv_layout_t *out);
+
+/*
+ * hikonv_pack - Eq. 5: words[x] = sum_{n<N} in[x N + n] * 2^(S n), modulo 2^word_bits.
+ * d_in: n codes (device, int8 storage, `bits` wide, signed or not).  The tail of the last word is
+ * zero-filled.  d_words: ceil(n / N) words of word_bits (32 or 64) bits, device, naturally aligned.
+ * For signed codes the word is the two's-complement sum, which equals the slot-by-slot
+ * decrementer form of Eq. 28.  Requires bits + (N-1) S <= word_bits.
+ */
+int hikonv_pack(const int8_t *d_in, size_t n, int bits, int is_signed, int S, int N, int word_bits,
+                void *d_words, void *stream);
+
+/*
+ * hikonv_conv1d - full 1-D convolution F_{len,K}(f, g) (Eq. 2-4 via Theorems 1 and 2).
+ * d_f: len codes of p bits; d_g: K codes of q bits; d_y: len + K - 1 int32 outputs (device, 4-byte
+ * aligned), y[m] = sum_k f[m-k] g[k] with f zero outside [0, len).
+ * algo: HIKONV_ALGO_PACKED32 or HIKONV_ALGO_UNPACKED_IMAD.  tune may be NULL.
+ * len >= 1, 1 <= K <= 64.
+ */
+int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p, int q,
+                  int f_signed, int g_signed, int32_t *d_y, int algo, const hikonv_tuning_t *tune,
+                  void *stream);
+
+/* Device scratch needed by hikonv_conv1d_host: room for f, g and y on the device. */
+size_t hikonv_conv1d_host_workspace_bytes(size_t len, int K);
+
+/*
+ * hikonv_conv1d_host - the same convolution with HOST buffers: copies h_f and h_g to the device
+ * workspace, runs hikonv_conv1d, copies len + K - 1 int32 results back to h_y, all on `stream`
+ * (asynchronous when the host buffers are pinned; the caller synchronises the stream).
+ * d_workspace: device memory of at least hikonv_conv1d_host_workspace_bytes(len, K) bytes,
+ * 256-byte aligned.
+ */
+int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, int p, int q,
+                       int f_signed, int g_signed, int32_t *h_y, void *d_workspace,
+                       size_t workspace_bytes, int algo, const hikonv_tuning_t *tune, void *stream);
+
+/*
+ * hikonv_conv2d - one convolution layer (Eq. 16 through Theorem 3 and Eq. 23), stride 1, zero padding.
+ * d_x: [B][Ci][H][W] codes of p bits; d_w: [Co][Ci][K][K] codes of q bits;
+ * output [B][Co][Ho][Wo], Ho = H + 2 pad - K + 1, Wo = W + 2 pad - K + 1:
+ *   requant == 0: d_out is int32, the exact sums;
+ *   requant != 0: d_out is int8, clamp(sum >> shift, lo, hi) with an arithmetic (floor) shift,
+ *                 0 <= shift <= 31, -128 <= lo <= hi <= 255 (values above 127 are stored as the
+ *                 byte of the unsigned code).
+ * The packed path first writes the reversed, packed kernel rows (g = W[co][ci][kh][K-1:0], Theorem 3)
+ * to d_workspace (hikonv_conv2d_workspace_bytes bytes, 256-byte aligned), then runs the layer; both
+ * on `stream`.  The unpacked comparator uses the workspace for int32 copies of the weights.
+ * stride must be 1 and 0 <= pad < K.
+ */
+int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,
+                  int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out,
+                  int requant, int shift, int lo, int hi, void *d_workspace, size_t workspace_bytes,
+                  int algo, const hikonv_tuning_t *tune, void *stream);
+
+size_t hikonv_conv2d_workspace_bytes(int Ci, int Co, int K);
+
+/* Device scratch needed by hikonv_conv2d_host: x, w, out and the kernel workspace. */
+size_t hikonv_conv2d_host_workspace_bytes(int B, int Ci, int H, int W, int Co, int K, int pad, int requant);
+
+/* hikonv_conv2d with HOST buffers (copies in, runs, copies out, all on `stream`). */
+int hikonv_conv2d_host(const int8_t *h_x, int B, int Ci, int H, int W, const int8_t *h_w, int Co, int K,
+                       int stride, int pad, int p, int q, int x_signed, int w_signed, void *h_out,
+                       int requant, int shift, int lo, int hi, void *d_workspace, size_t workspace_bytes,
+                       int algo, const hikonv_tuning_t *tune, void *stream);
+
+/*
+ * hikonv_maxpool2x2_i8 - 2x2 max-pool, stride 2, on [B][C][H][W] byte codes -> [B][C][H/2][W/2].
+ * Not part of the paper's method (its pooling is not accelerated); glue for the full-network
+ * workload.  is_signed selects int8 or uint8 comparison.
+ */
+int hikonv_maxpool2x2_i8(const int8_t *d_in, int B, int C, int H, int W, int is_signed, int8_t *d_out,
+                         void *stream);
+
+/* Number of wide multiplies (packed) or 32-bit multiply-adds (unpacked) the last-planned launch of
+ * the given problem executes, for roofline accounting.  Host only. */
+double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int f_signed, int g_signed, int algo,
+                                const hikonv_tuning_t *tune);
+double hikonv_conv2d_multiplies(int B, int Ci, int H, int W, int Co, int K, int pad, int p, int q,
+                                int x_signed, int w_signed, int algo, const hikonv_tuning_t *tune);
+
+const char *hikonv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIKONV_H */

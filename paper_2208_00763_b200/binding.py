@@ -1,0 +1,217 @@
+"""ctypes binding of ``libhikonv.so``: same names as the C interface, argument marshalling only.
+
+PyTorch is used for device memory and streams; every arithmetic step runs in the CUDA
+library.  Loading fails loudly when the library has not been built: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhikonv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA = range(6)
+ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD = 0, 1, 2
+GB_SINGLE, GB_1D, GB_DNN = 0, 1, 2
+
+
+class HikonvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, status_string(status), status))
+
+
+class PlanT(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "K", "S", "Gb", "ops")]
+
+
+class LayoutT(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "S", "Kc", "J", "segments", "top_bits", "M", "signed_prod", "S_paper")]
+
+
+class TuningT(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "S", "M", "tile")]
+
+
+_lib = None
+
+_vp, _sz, _i, _d = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_double
+
+_SIGNATURES = {
+    "hikonv_plan": (_i, [_i] * 7 + [ctypes.POINTER(PlanT)]),
+    "hikonv_layout": (_i, [_i] * 7 + [ctypes.POINTER(TuningT), ctypes.POINTER(LayoutT)]),
+    "hikonv_pack": (_i, [_vp, _sz, _i, _i, _i, _i, _i, _vp, _vp]),
+    "hikonv_conv1d": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _i, ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv1d_host_workspace_bytes": (_sz, [_sz, _i]),
+    "hikonv_conv1d_host": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _i, ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv2d": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz, _i,
+                           ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv2d_workspace_bytes": (_sz, [_i, _i, _i]),
+    "hikonv_conv2d_host_workspace_bytes": (_sz, [_i] * 8),
+    "hikonv_conv2d_host": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz,
+                                _i, ctypes.POINTER(TuningT), _vp]),
+    "hikonv_maxpool2x2_i8": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
+    "hikonv_conv1d_multiplies": (_d, [_sz, _i, _i, _i, _i, _i, _i, ctypes.POINTER(TuningT)]),
+    "hikonv_conv2d_multiplies": (_d, [_i] * 12 + [ctypes.POINTER(TuningT)]),
+    "hikonv_status_string": (ctypes.c_char_p, [_i]),
+}
+
+
+def exported_names():
+    return sorted(_SIGNATURES)
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "CUDA library %s is missing: run `python -m paper_2208_00763_b200.build` "
+                "(or __graft_entry__.build()) first; there is no CPU fallback" % LIB_PATH)
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = handle
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().hikonv_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise HikonvError(status, where)
+
+
+def _tune(tune: Optional[dict]):
+    if not tune:
+        return None
+    t = TuningT(int(tune.get("N", 0)), int(tune.get("S", 0)), int(tune.get("M", 0)), int(tune.get("tile", 0)))
+    return ctypes.byref(t)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_i8(t: torch.Tensor, name: str) -> int:
+    if not t.is_cuda or t.dtype not in (torch.int8, torch.uint8) or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA int8/uint8 tensor" % name)
+    return t.data_ptr()
+
+
+# ------------------------------------------------------------------ host-only planning
+
+def plan(p, q, LA=32, LB=32, mode=GB_SINGLE, M=1, K_fixed=0) -> dict:
+    out = PlanT()
+    _check(lib().hikonv_plan(p, q, LA, LB, mode, M, K_fixed, ctypes.byref(out)), "hikonv_plan")
+    return {n: getattr(out, n) for n, _ in PlanT._fields_}
+
+
+def layout(p, q, f_signed, g_signed, K, dims, total_terms=0, tune=None) -> dict:
+    out = LayoutT()
+    _check(lib().hikonv_layout(p, q, int(f_signed), int(g_signed), K, dims, total_terms, _tune(tune), ctypes.byref(out)),
+           "hikonv_layout")
+    return {n: getattr(out, n) for n, _ in LayoutT._fields_}
+
+
+# ------------------------------------------------------------------ device entry points
+
+def pack(d_in: torch.Tensor, bits: int, is_signed: bool, S: int, N: int, word_bits: int = 32, stream=None) -> torch.Tensor:
+    n = d_in.numel()
+    n_words = (n + N - 1) // N
+    out = torch.empty(n_words, dtype=torch.int32 if word_bits == 32 else torch.int64, device=d_in.device)
+    _check(lib().hikonv_pack(_dev_i8(d_in, "d_in"), n, bits, int(is_signed), S, N, word_bits, out.data_ptr(), _stream(stream)),
+           "hikonv_pack")
+    return out
+
+
+def conv1d(d_f: torch.Tensor, d_g: torch.Tensor, p: int, q: int, f_signed: bool, g_signed: bool,
+           algo: int = ALGO_PACKED32, tune=None, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    n, K = d_f.numel(), d_g.numel()
+    if out is None:
+        out = torch.empty(n + K - 1, dtype=torch.int32, device=d_f.device)
+    _check(lib().hikonv_conv1d(_dev_i8(d_f, "d_f"), n, _dev_i8(d_g, "d_g"), K, p, q, int(f_signed), int(g_signed),
+                               out.data_ptr(), algo, _tune(tune), _stream(stream)), "hikonv_conv1d")
+    return out
+
+
+def conv1d_host_workspace_bytes(n: int, K: int) -> int:
+    return int(lib().hikonv_conv1d_host_workspace_bytes(n, K))
+
+
+def conv1d_host(h_f: torch.Tensor, h_g: torch.Tensor, p, q, f_signed, g_signed, h_y: torch.Tensor,
+                d_workspace: torch.Tensor, algo: int = ALGO_PACKED32, tune=None, stream=None) -> None:
+    """Host buffers in, host buffer out (pinned tensors make the copies asynchronous)."""
+    n, K = h_f.numel(), h_g.numel()
+    _check(lib().hikonv_conv1d_host(h_f.data_ptr(), n, h_g.data_ptr(), K, p, q, int(f_signed), int(g_signed),
+                                    h_y.data_ptr(), d_workspace.data_ptr(), d_workspace.numel() * d_workspace.element_size(),
+                                    algo, _tune(tune), _stream(stream)), "hikonv_conv1d_host")
+
+
+def conv2d_workspace_bytes(Ci: int, Co: int, K: int) -> int:
+    return int(lib().hikonv_conv2d_workspace_bytes(Ci, Co, K))
+
+
+def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_signed: bool, w_signed: bool,
+           requant: Optional[tuple] = None, algo: int = ALGO_PACKED32, tune=None, workspace: Optional[torch.Tensor] = None,
+           out: Optional[torch.Tensor] = None, stride: int = 1, stream=None) -> torch.Tensor:
+    """requant = (shift, lo, hi) selects int8 output, None the exact int32 sums."""
+    B, Ci, H, W = d_x.shape
+    Co, Ci2, K, K2 = d_w.shape
+    if Ci != Ci2 or K != K2:
+        raise ValueError("weight shape does not match the input")
+    Ho, Wo = H + 2 * pad - K + 1, W + 2 * pad - K + 1
+    if workspace is None:
+        workspace = torch.empty(conv2d_workspace_bytes(Ci, Co, K), dtype=torch.uint8, device=d_x.device)
+    if out is None:
+        out = torch.empty((B, Co, max(Ho, 0), max(Wo, 0)), dtype=torch.int8 if requant else torch.int32, device=d_x.device)
+    shift, lo, hi = requant if requant else (0, 0, 0)
+    _check(lib().hikonv_conv2d(_dev_i8(d_x, "d_x"), B, Ci, H, W, _dev_i8(d_w, "d_w"), Co, K, stride, pad, p, q,
+                               int(x_signed), int(w_signed), out.data_ptr(), 1 if requant else 0, shift, lo, hi,
+                               workspace.data_ptr(), workspace.numel() * workspace.element_size(), algo, _tune(tune),
+                               _stream(stream)), "hikonv_conv2d")
+    return out
+
+
+def conv2d_host_workspace_bytes(B, Ci, H, W, Co, K, pad, requant) -> int:
+    return int(lib().hikonv_conv2d_host_workspace_bytes(B, Ci, H, W, Co, K, pad, 1 if requant else 0))
+
+
+def conv2d_host(h_x: torch.Tensor, h_w: torch.Tensor, pad, p, q, x_signed, w_signed, h_out: torch.Tensor,
+                d_workspace: torch.Tensor, requant: Optional[tuple] = None, algo: int = ALGO_PACKED32, tune=None,
+                stride: int = 1, stream=None) -> None:
+    B, Ci, H, W = h_x.shape
+    Co, _, K, _ = h_w.shape
+    shift, lo, hi = requant if requant else (0, 0, 0)
+    _check(lib().hikonv_conv2d_host(h_x.data_ptr(), B, Ci, H, W, h_w.data_ptr(), Co, K, stride, pad, p, q, int(x_signed),
+                                    int(w_signed), h_out.data_ptr(), 1 if requant else 0, shift, lo, hi,
+                                    d_workspace.data_ptr(), d_workspace.numel() * d_workspace.element_size(), algo,
+                                    _tune(tune), _stream(stream)), "hikonv_conv2d_host")
+
+
+def maxpool2x2_i8(d_in: torch.Tensor, is_signed: bool, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    B, C, H, W = d_in.shape
+    if out is None:
+        out = torch.empty((B, C, H // 2, W // 2), dtype=d_in.dtype, device=d_in.device)
+    _check(lib().hikonv_maxpool2x2_i8(_dev_i8(d_in, "d_in"), B, C, H, W, int(is_signed), out.data_ptr(), _stream(stream)),
+           "hikonv_maxpool2x2_i8")
+    return out
+
+
+def conv1d_multiplies(n, K, p, q, f_signed, g_signed, algo=ALGO_PACKED32, tune=None) -> float:
+    return float(lib().hikonv_conv1d_multiplies(n, K, p, q, int(f_signed), int(g_signed), algo, _tune(tune)))
+
+
+def conv2d_multiplies(B, Ci, H, W, Co, K, pad, p, q, x_signed, w_signed, algo=ALGO_PACKED32, tune=None) -> float:
+    return float(lib().hikonv_conv2d_multiplies(B, Ci, H, W, Co, K, pad, p, q, int(x_signed), int(w_signed), algo, _tune(tune)))

@@ -1,0 +1,355 @@
+// hikonv_conv1d: full 1-D convolution, packed (Theorems 1 and 2) and unpacked comparator.
+//
+// Packed kernel, per warp: a run of "chunks" of 32 consecutive blocks, one block of N outputs
+// per lane.  For block x a lane
+//   packs   A_x = sum_n f[xN+n] 2^(S n)                                  (Eq. 5)
+//   forms   Q_x = bias + sum_j A_{x-j} * B_j                              (Eq. 9; J > 1 when the
+//           kernel is cut into chunks of N taps, A_{x-j} comes from lane - j by shuffle)
+//   adds    the carry of block x-1:  D_x = Q_x + (Q_{x-1} >> S N)         (Theorem 2, the
+//           "previous product shifted right" step of Section V-A; lane - 1 by shuffle)
+//   splits  y[xN+m] = ((D_x >> S m) & mask) - carry_bias[m],  m < N       (Algorithm 2's shift
+//           and mask; the per-slot bias replaces the sign-borrow increment of Eq. 29)
+// Outputs are staged per warp in shared memory and written with coalesced 16-byte stores.
+#include "hikonv_cuda.cuh"
+
+namespace hikonv {
+
+constexpr int kThreads1D = 256;
+constexpr int kWarps1D = kThreads1D / 32;
+
+struct Conv1dParams {
+    const int8_t *f;
+    const int8_t *g;
+    int32_t *y;
+    long long len;
+    long long n_out;
+    long long n_chunks;      // chunks of 32 blocks covering n_out outputs
+    int K, S, J, Kc;
+    int hi_shift;            // S * N
+    int g_signed;
+    int chunks_per_warp;
+    int y_aligned16;
+    uint32_t mask;
+    uint64_t bias;
+    int seg_shift[kMaxN1D];  // S * m
+    int32_t carry_bias[kMaxN1D];
+};
+
+__host__ __device__ constexpr int stage_chunks(int N) { return N >= 16 ? 1 : (16 / N > 0 ? 16 / N : 1); }
+
+template <int N, bool F_SIGNED>
+__device__ __forceinline__ void load_block_codes(const Conv1dParams &p, long long chunk, int lane, int32_t (&v)[N]) {
+    const long long base = (chunk * 32 + lane) * (long long)N;
+    if (chunk >= 0 && (chunk * 32 + 32) * (long long)N <= p.len) {       // whole chunk inside the signal
+        const int8_t *src = p.f + base;
+#pragma unroll
+        for (int n = 0; n < N; ++n) v[n] = load_code<F_SIGNED>(src + n);
+    } else {
+#pragma unroll
+        for (int n = 0; n < N; ++n) {
+            const long long idx = base + n;
+            v[n] = (idx >= 0 && idx < p.len) ? load_code<F_SIGNED>(p.f + idx) : 0;   // Eq. 2: zero outside
+        }
+    }
+}
+
+template <int N, bool SIGNED_PROD, bool F_SIGNED>
+__global__ void __launch_bounds__(kThreads1D) conv1d_packed_kernel(const Conv1dParams p) {
+    constexpr int G = stage_chunks(N);
+    __shared__ uint32_t s_B[kMaxJ];
+    __shared__ __align__(16) int32_t s_out[kWarps1D][G * 32 * N];
+
+    if (threadIdx.x < p.J) {            // pack the kernel chunk B_j (Eq. 5 on g)
+        const int j = threadIdx.x;
+        uint32_t b = 0;
+        for (int k = 0; k < p.Kc; ++k) {
+            const int idx = j * p.Kc + k;
+            if (idx < p.K) {
+                const int8_t raw = __ldg(p.g + idx);
+                const int32_t v = p.g_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+                b += (uint32_t)v << (p.S * k);
+            }
+        }
+        s_B[j] = b;
+    }
+    __syncthreads();
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long c0 = ((long long)blockIdx.x * kWarps1D + warp) * p.chunks_per_warp;
+    if (c0 >= p.n_chunks) return;
+    const long long c1 = (c0 + p.chunks_per_warp < p.n_chunks) ? c0 + p.chunks_per_warp : p.n_chunks;
+
+    uint32_t slot_pow[N];               // 2^(S n): packing by multiply-add
+#pragma unroll
+    for (int n = 0; n < N; ++n) slot_pow[n] = 1u << (p.S * n);
+    const uint32_t B0 = s_B[0];
+    int32_t *stage = s_out[warp];
+
+    uint32_t prevA = 0, prevHi = 0;
+    int32_t vnext[N];
+    load_block_codes<N, F_SIGNED>(p, c0 - 1, lane, vnext);
+    long long group_c0 = c0;
+    for (long long c = c0 - 1; c < c1; ++c) {
+        int32_t v[N];
+#pragma unroll
+        for (int n = 0; n < N; ++n) v[n] = vnext[n];
+        if (c + 1 < c1) load_block_codes<N, F_SIGNED>(p, c + 1, lane, vnext);
+
+        uint32_t A = (uint32_t)v[0];
+#pragma unroll
+        for (int n = 1; n < N; ++n) A += (uint32_t)v[n] * slot_pow[n];
+
+        uint64_t Q = p.bias;
+        mad_wide<SIGNED_PROD>(Q, A, B0);
+        for (int j = 1; j < p.J; ++j) {
+            const uint32_t src = (lane >= 32 - j) ? prevA : A;          // block x-j sits in lane-j of this or the previous chunk
+            const uint32_t Aj = __shfl_sync(0xFFFFFFFFu, src, (lane - j) & 31);
+            mad_wide<SIGNED_PROD>(Q, Aj, s_B[j]);
+        }
+        const uint32_t hi = shr64_lo(Q, p.hi_shift);                     // slots N.. of this block's product
+        uint32_t carry = __shfl_up_sync(0xFFFFFFFFu, hi, 1);
+        if (lane == 0) carry = prevHi;
+        prevHi = __shfl_sync(0xFFFFFFFFu, hi, 31);
+        prevA = A;
+        if (c < c0) continue;           // the chunk before the run only seeds the carries
+
+        const uint64_t D = Q + (uint64_t)carry;
+        int32_t out[N];
+#pragma unroll
+        for (int m = 0; m < N; ++m) out[m] = (int32_t)(shr64_lo(D, p.seg_shift[m]) & p.mask) - p.carry_bias[m];
+
+        const int slot = (int)(c - group_c0);
+        int32_t *dst = stage + (slot * 32 + lane) * N;
+        if (N % 4 == 0) {
+#pragma unroll
+            for (int m = 0; m < N; m += 4) *reinterpret_cast<int4 *>(dst + m) = make_int4(out[m], out[m + 1], out[m + 2], out[m + 3]);
+        } else if (N % 2 == 0) {
+#pragma unroll
+            for (int m = 0; m < N; m += 2) *reinterpret_cast<int2 *>(dst + m) = make_int2(out[m], out[m + 1]);
+        } else {
+#pragma unroll
+            for (int m = 0; m < N; ++m) dst[m] = out[m];
+        }
+
+        if (slot == G - 1 || c == c1 - 1) {     // write the staged group out, coalesced
+            __syncwarp();
+            const long long first = group_c0 * 32 * (long long)N;
+            const int count = (slot + 1) * 32 * N;
+            if (p.y_aligned16 && first + count <= p.n_out) {
+                const int4 *s4 = reinterpret_cast<const int4 *>(stage);
+                int4 *d4 = reinterpret_cast<int4 *>(p.y + first);
+                for (int i = lane; i < count / 4; i += 32) d4[i] = s4[i];
+            } else {
+                for (int i = lane; i < count; i += 32)
+                    if (first + i < p.n_out) p.y[first + i] = stage[i];
+            }
+            __syncwarp();
+            group_c0 = c + 1;
+        }
+    }
+}
+
+// Comparator: one product per 32-bit multiply-add.  Each thread computes four consecutive outputs
+// with a sliding window over f.
+struct Conv1dUnpackedParams {
+    const int8_t *f;
+    const int8_t *g;
+    int32_t *y;
+    long long len;
+    long long n_out;
+    int K;
+    int g_signed;
+    int y_aligned16;
+};
+
+// One kernel tap for four neighbouring outputs: y[t0+o] += f[t0+o-k] g[k], then slide the window
+// one element towards lower indices for the next tap.
+template <bool F_SIGNED>
+__device__ __forceinline__ void unpacked_tap(const Conv1dUnpackedParams &p, long long t0, int k, int K, bool interior,
+                                             int32_t gk, int32_t (&w)[4], int32_t (&acc)[4]) {
+#pragma unroll
+    for (int o = 0; o < 4; ++o) acc[o] += w[o] * gk;
+    if (k + 1 < K) {
+        const long long idx = t0 - (k + 1);
+        w[3] = w[2];
+        w[2] = w[1];
+        w[1] = w[0];
+        w[0] = (interior || (idx >= 0 && idx < p.len)) ? load_code<F_SIGNED>(p.f + idx) : 0;
+    }
+}
+
+template <int KT, bool F_SIGNED>
+__global__ void __launch_bounds__(kThreads1D) conv1d_unpacked_kernel(const Conv1dUnpackedParams p) {
+    __shared__ int32_t s_g[kMaxK];
+    const int K = KT > 0 ? KT : p.K;
+    if (threadIdx.x < K) {
+        const int8_t raw = __ldg(p.g + threadIdx.x);
+        s_g[threadIdx.x] = p.g_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+    }
+    __syncthreads();
+    const long long t0 = ((long long)blockIdx.x * kThreads1D + threadIdx.x) * 4;
+    if (t0 >= p.n_out) return;
+    const bool interior = (t0 - (K - 1) >= 0) && (t0 + 3 < p.len);
+    int32_t w[4];
+#pragma unroll
+    for (int o = 0; o < 4; ++o) {
+        const long long idx = t0 + o;
+        w[o] = (interior || idx < p.len) ? load_code<F_SIGNED>(p.f + idx) : 0;
+    }
+    int32_t acc[4] = {0, 0, 0, 0};
+    if (KT > 0) {
+#pragma unroll
+        for (int k = 0; k < KT; ++k) unpacked_tap<F_SIGNED>(p, t0, k, KT, interior, s_g[k], w, acc);
+    } else {
+        for (int k = 0; k < K; ++k) unpacked_tap<F_SIGNED>(p, t0, k, K, interior, s_g[k], w, acc);
+    }
+    if (p.y_aligned16 && t0 + 3 < p.n_out) {
+        *reinterpret_cast<int4 *>(p.y + t0) = make_int4(acc[0], acc[1], acc[2], acc[3]);
+    } else {
+#pragma unroll
+        for (int o = 0; o < 4; ++o)
+            if (t0 + o < p.n_out) p.y[t0 + o] = acc[o];
+    }
+}
+
+template <int N>
+static int launch_packed_n(const Conv1dParams &p, bool signed_prod, bool f_signed, unsigned grid, cudaStream_t st) {
+    if (!signed_prod)
+        conv1d_packed_kernel<N, false, false><<<grid, kThreads1D, 0, st>>>(p);
+    else if (f_signed)
+        conv1d_packed_kernel<N, true, true><<<grid, kThreads1D, 0, st>>>(p);
+    else
+        conv1d_packed_kernel<N, true, false><<<grid, kThreads1D, 0, st>>>(p);
+    return launch_status();
+}
+
+static int launch_packed(int N, const Conv1dParams &p, bool sp, bool fs, unsigned grid, cudaStream_t st) {
+    switch (N) {
+        case 1: return launch_packed_n<1>(p, sp, fs, grid, st);
+        case 2: return launch_packed_n<2>(p, sp, fs, grid, st);
+        case 3: return launch_packed_n<3>(p, sp, fs, grid, st);
+        case 4: return launch_packed_n<4>(p, sp, fs, grid, st);
+        case 5: return launch_packed_n<5>(p, sp, fs, grid, st);
+        case 6: return launch_packed_n<6>(p, sp, fs, grid, st);
+        case 7: return launch_packed_n<7>(p, sp, fs, grid, st);
+        case 8: return launch_packed_n<8>(p, sp, fs, grid, st);
+        case 9: return launch_packed_n<9>(p, sp, fs, grid, st);
+        case 10: return launch_packed_n<10>(p, sp, fs, grid, st);
+        case 11: return launch_packed_n<11>(p, sp, fs, grid, st);
+        case 12: return launch_packed_n<12>(p, sp, fs, grid, st);
+        default: return HIKONV_ERR_UNSUPPORTED;
+    }
+}
+
+template <bool F_SIGNED>
+static int launch_unpacked(const Conv1dUnpackedParams &p, unsigned grid, cudaStream_t st) {
+    switch (p.K) {
+        case 3: conv1d_unpacked_kernel<3, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
+        case 5: conv1d_unpacked_kernel<5, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
+        case 7: conv1d_unpacked_kernel<7, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
+        default: conv1d_unpacked_kernel<0, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
+    }
+    return launch_status();
+}
+
+static int check_conv1d_args(const void *f, size_t len, const void *g, int K, int p, int q, const void *y, int algo) {
+    if (!f || !g || !y || len < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
+    if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
+    if (len > (size_t)1 << 40) return HIKONV_ERR_UNSUPPORTED;
+    if (algo == HIKONV_ALGO_PACKED64EMU) return HIKONV_ERR_UNSUPPORTED;
+    if (algo != HIKONV_ALGO_PACKED32 && algo != HIKONV_ALGO_UNPACKED_IMAD) return HIKONV_ERR_INVALID_ARG;
+    if (((uintptr_t)y) % 4 != 0) return HIKONV_ERR_INVALID_ARG;
+    return HIKONV_OK;
+}
+
+}  // namespace hikonv
+
+using namespace hikonv;
+
+extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p, int q, int f_signed,
+                             int g_signed, int32_t *d_y, int algo, const hikonv_tuning_t *tune, void *stream) {
+    int rc = check_conv1d_args(d_f, len, d_g, K, p, q, d_y, algo);
+    if (rc != HIKONV_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const long long n_out = (long long)len + K - 1;
+    const int y_aligned16 = ((uintptr_t)d_y % 16 == 0) ? 1 : 0;
+
+    if (algo == HIKONV_ALGO_UNPACKED_IMAD) {
+        Conv1dUnpackedParams up;
+        up.f = d_f; up.g = d_g; up.y = d_y; up.len = (long long)len; up.n_out = n_out; up.K = K;
+        up.g_signed = g_signed ? 1 : 0; up.y_aligned16 = y_aligned16;
+        const long long threads = (n_out + 3) / 4;
+        const long long grid = (threads + kThreads1D - 1) / kThreads1D;
+        if (grid > 0x7FFFFFFFLL) return HIKONV_ERR_UNSUPPORTED;
+        return f_signed ? launch_unpacked<true>(up, (unsigned)grid, st) : launch_unpacked<false>(up, (unsigned)grid, st);
+    }
+
+    hikonv_layout_t L;
+    rc = make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L);
+    if (rc != HIKONV_OK) return rc;
+    if (L.N > kMaxN1D) return HIKONV_ERR_UNSUPPORTED;
+    const SplitConsts sc = make_split_consts(L, p, q, f_signed, g_signed, K, 1);
+
+    Conv1dParams kp;
+    kp.f = d_f; kp.g = d_g; kp.y = d_y; kp.len = (long long)len; kp.n_out = n_out;
+    const long long n_blocks = (n_out + L.N - 1) / L.N;
+    kp.n_chunks = (n_blocks + 31) / 32;
+    kp.K = K; kp.S = L.S; kp.J = L.J; kp.Kc = L.Kc; kp.hi_shift = L.S * L.N;
+    kp.g_signed = g_signed ? 1 : 0;
+    kp.y_aligned16 = y_aligned16;
+    kp.mask = sc.slot_mask;
+    kp.bias = sc.bias;
+    for (int m = 0; m < kMaxN1D; ++m) {
+        kp.seg_shift[m] = m < L.N ? L.S * m : 0;
+        kp.carry_bias[m] = m < L.N ? sc.carry_bias[m] : 0;
+    }
+    // long runs amortise the one seeding chunk per warp; short problems spread over the SMs first
+    long long cpw = tune && tune->tile > 0 ? tune->tile : 16;
+    int sms = 148;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    const long long want_warps = (long long)sms * kWarps1D * 4;
+    if (kp.n_chunks / cpw < want_warps) cpw = kp.n_chunks / want_warps;
+    if (cpw < 1) cpw = 1;
+    kp.chunks_per_warp = (int)cpw;
+    const long long warps = (kp.n_chunks + cpw - 1) / cpw;
+    const long long grid = (warps + kWarps1D - 1) / kWarps1D;
+    if (grid > 0x7FFFFFFFLL) return HIKONV_ERR_UNSUPPORTED;
+    return launch_packed(L.N, kp, L.signed_prod != 0, f_signed != 0, (unsigned)grid, st);
+}
+
+extern "C" size_t hikonv_conv1d_host_workspace_bytes(size_t len, int K) {
+    if (K < 1) return 0;
+    return align_up(len, 256) + align_up((size_t)K, 256) + align_up((len + (size_t)K - 1) * sizeof(int32_t), 256);
+}
+
+extern "C" int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, int p, int q, int f_signed,
+                                  int g_signed, int32_t *h_y, void *d_workspace, size_t workspace_bytes, int algo,
+                                  const hikonv_tuning_t *tune, void *stream) {
+    if (!h_f || !h_g || !h_y || len < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
+    if (!d_workspace || ((uintptr_t)d_workspace % 256) != 0 || workspace_bytes < hikonv_conv1d_host_workspace_bytes(len, K))
+        return HIKONV_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    int8_t *d_f = (int8_t *)d_workspace;
+    int8_t *d_g = d_f + align_up(len, 256);
+    int32_t *d_y = (int32_t *)(d_g + align_up((size_t)K, 256));
+    HIKONV_CUDA_TRY(cudaMemcpyAsync(d_f, h_f, len, cudaMemcpyHostToDevice, st));
+    HIKONV_CUDA_TRY(cudaMemcpyAsync(d_g, h_g, (size_t)K, cudaMemcpyHostToDevice, st));
+    const int rc = hikonv_conv1d(d_f, len, d_g, K, p, q, f_signed, g_signed, d_y, algo, tune, st);
+    if (rc != HIKONV_OK) return rc;
+    HIKONV_CUDA_TRY(cudaMemcpyAsync(h_y, d_y, (len + (size_t)K - 1) * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    return HIKONV_OK;
+}
+
+extern "C" double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int f_signed, int g_signed, int algo,
+                                           const hikonv_tuning_t *tune) {
+    if (len < 1 || K < 1) return 0.0;
+    const double n_out = (double)len + K - 1;
+    if (algo == HIKONV_ALGO_UNPACKED_IMAD) return n_out * K;
+    hikonv_layout_t L;
+    if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L) != HIKONV_OK) return 0.0;
+    const double blocks = (double)(((long long)n_out + L.N - 1) / L.N);
+    return blocks * L.J;
+}

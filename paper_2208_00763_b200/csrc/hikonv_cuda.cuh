@@ -1,0 +1,45 @@
+// Small device/host helpers shared by the CUDA translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "hikonv_internal.h"
+
+namespace hikonv {
+
+// Evaluates a CUDA runtime call; on failure returns HIKONV_ERR_CUDA from the enclosing function.
+#define HIKONV_CUDA_TRY(expr)                                 \
+    do {                                                      \
+        cudaError_t _e = (expr);                              \
+        if (_e != cudaSuccess) return HIKONV_ERR_CUDA;        \
+    } while (0)
+
+// After a kernel launch: report a launch failure without clearing an earlier sticky error.
+inline int launch_status() { return cudaPeekAtLastError() == cudaSuccess ? HIKONV_OK : HIKONV_ERR_CUDA; }
+
+// One 32x32->64 multiply-accumulate, acc += a * b (the packed multiply of Eq. 9).
+template <bool SIGNED>
+__device__ __forceinline__ void mad_wide(uint64_t &acc, uint32_t a, uint32_t b) {
+    if (SIGNED)
+        asm("mad.wide.s32 %0, %1, %2, %0;" : "+l"(acc) : "r"(a), "r"(b));
+    else
+        asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(acc) : "r"(a), "r"(b));
+}
+
+// Low 32 bits of (v >> sh) for 0 <= sh < 64.
+__device__ __forceinline__ uint32_t shr64_lo(uint64_t v, int sh) { return (uint32_t)(v >> sh); }
+
+// A code byte as a 32-bit value (sign- or zero-extended).
+template <bool SIGNED>
+__device__ __forceinline__ int32_t code_value(int8_t b) {
+    return SIGNED ? (int32_t)b : (int32_t)(uint8_t)b;
+}
+
+template <bool SIGNED>
+__device__ __forceinline__ int32_t load_code(const int8_t *p) {
+    return code_value<SIGNED>(__ldg(p));
+}
+
+}  // namespace hikonv

@@ -1,0 +1,43 @@
+// Internal declarations shared by the translation units of the library (not installed).
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+
+#include "hikonv.h"
+
+namespace hikonv {
+
+constexpr int kMaxN1D = 12;     // largest N the 1-D kernels are instantiated for
+constexpr int kMaxN2D = 4;      // largest N the 2-D kernels are instantiated for
+constexpr int kMaxSegments = 24;
+constexpr int kMaxK = 64;       // longest kernel accepted
+constexpr int kMaxJ = 16;       // most weight chunks per kernel row
+
+// Constants of the biased split.  Every slot m of the 64-bit accumulator starts at
+// seg_bias[m] = -(smallest sum the slot can receive), so every stored field is non-negative and
+// slots never borrow from each other; the bias is subtracted after extraction.
+struct SplitConsts {
+    uint64_t bias;                      // sum_m seg_bias[m] 2^(S m): initial accumulator value
+    int32_t seg_bias[kMaxSegments];     // per product slot
+    int32_t carry_bias[kMaxSegments];   // slot m of (product + carry of the previous block), m < N
+    uint32_t slot_mask;                 // 2^S - 1
+};
+
+// Cost-model constants for the 2-D planner, in scheduler cycles per warp instruction.
+struct CostModel {
+    double mul_cycles = 2.0;        // one 32x32->64 multiply-accumulate
+    double split_cycles_per_seg = 5.0;
+};
+
+int validate_codes(int p, int q);
+// Exact-range layout search; `packed_overlap` selects the 1-D rule (block carries are added
+// before the split, so a slot holds all K terms).
+int make_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int total_terms,
+                int row_outputs, const hikonv_tuning_t *tune, hikonv_layout_t *out);
+SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int f_signed, int g_signed, int K, int M);
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace hikonv

@@ -1,0 +1,274 @@
+// Host-side planning: the paper's throughput search (Algorithm 1) and the exact-range layout
+// the CUDA kernels run with.
+#include <algorithm>
+#include <cstring>
+
+#include "hikonv_internal.h"
+
+namespace hikonv {
+
+typedef __int128 i128;
+
+static int ceil_log2(long long v) {
+    int b = 0;
+    while ((1LL << b) < v) ++b;
+    return b;
+}
+
+// Eq. 11, the 1-D rule and the DNN rule.
+static int guard_bits(int mode, int N, int K, int M) {
+    switch (mode) {
+        case HIKONV_GB_SINGLE: return ceil_log2(std::min(K, N));
+        case HIKONV_GB_1D: return ceil_log2(K);
+        case HIKONV_GB_DNN: return ceil_log2((long long)M * std::min(K, N));
+        default: return -1;
+    }
+}
+
+// Eq. 6.
+static int slice_bits(int p, int q, int Gb) {
+    if (p == 1) return q + Gb;
+    if (q == 1) return p + Gb;
+    return p + q + Gb;
+}
+
+int validate_codes(int p, int q) {
+    if (p < 1 || p > 8 || q < 1 || q > 8) return HIKONV_ERR_INVALID_ARG;
+    return HIKONV_OK;
+}
+
+struct Range {
+    long long lo, hi;
+};
+
+static Range code_range(int bits, int is_signed) {
+    if (is_signed) return {-(1LL << (bits - 1)), (1LL << (bits - 1)) - 1};
+    return {0, (1LL << bits) - 1};
+}
+
+// Largest and smallest value of sum_{n<count} v 2^(S n) over codes v in r.
+static void packed_range(Range r, int count, int S, i128 *lo, i128 *hi) {
+    i128 geo = 0;
+    for (int n = 0; n < count; ++n) geo += (i128)1 << (S * n);
+    *lo = (i128)r.lo * geo;
+    *hi = (i128)r.hi * geo;
+}
+
+static bool operand_fits(Range r, int count, int S, bool signed_mul) {
+    if ((long long)S * (count - 1) > 60) return false;
+    i128 lo, hi;
+    packed_range(r, count, S, &lo, &hi);
+    if (signed_mul) return lo >= -((i128)1 << 31) && hi <= ((i128)1 << 31) - 1;
+    return lo >= 0 && hi <= ((i128)1 << 32) - 1;
+}
+
+// Number of (n, k) pairs with n + k == m, 0 <= n < N, 0 <= k < kc.
+static int pair_count(int m, int N, int kc) {
+    int lo = std::max(0, m - kc + 1), hi = std::min(m, N - 1);
+    return hi >= lo ? hi - lo + 1 : 0;
+}
+
+// Does a value range fit a w-bit slot once it is biased by -lo (so that the stored field is >= 0)?
+static bool slot_fits(i128 lo, i128 hi, int w) {
+    if (w < 1) return lo == 0 && hi == 0;
+    if (w > 62) w = 62;
+    return hi - lo <= ((i128)1 << w) - 1;
+}
+
+// Checks one candidate (N, S) and fills Kc, J, segments, top_bits and the largest M (capped).
+// `packed_overlap`: the carry of block x-1 is added to block x's product before the split.
+static bool check_candidate(int p, int q, int fs, int gs, int K, int N, int S, bool packed_overlap,
+                            long long M_cap, hikonv_layout_t *L) {
+    if (S < 1 || S > 31 || N < 1) return false;
+    const bool sp = fs || gs;
+    const Range fr = code_range(p, fs), gr = code_range(q, gs);
+    if (!operand_fits(fr, N, S, sp)) return false;
+    // weights: one word if the whole kernel fits and its carry reaches only the next block,
+    // else chunks of N taps (Theorem 2 applied to the kernel)
+    int Kc, J;
+    if (K <= N + 1 && operand_fits(gr, K, S, sp)) {
+        Kc = K;
+        J = 1;
+    } else {
+        Kc = N;
+        J = ceil_div(K, N);
+        if (!operand_fits(gr, Kc, S, sp)) return false;
+    }
+    if (J > kMaxJ) return false;
+    const int NS = N + Kc - 1;
+    if (NS > kMaxSegments) return false;
+    if ((long long)S * (NS - 1) >= 64) return false;
+    const int top_bits = std::min(S, 64 - S * (NS - 1));
+    const long long prods[4] = {fr.lo * gr.lo, fr.lo * gr.hi, fr.hi * gr.lo, fr.hi * gr.hi};
+    const long long pmin = *std::min_element(prods, prods + 4), pmax = *std::max_element(prods, prods + 4);
+    // term counts per slot
+    int T[kMaxSegments] = {0};
+    for (int j = 0; j < J; ++j) {
+        const int kc = std::min(Kc, K - j * Kc);
+        for (int m = 0; m < NS; ++m) T[m] += pair_count(m, N, kc);
+    }
+    auto fits_with = [&](long long M) {
+        for (int m = 0; m < NS; ++m) {
+            const int w = (m == NS - 1) ? top_bits : S;
+            if (!slot_fits((i128)M * T[m] * pmin, (i128)M * T[m] * pmax, w)) return false;
+        }
+        if (packed_overlap) {
+            for (int m = 0; m < N; ++m) {
+                const int t = T[m] + (m + N < NS ? T[m + N] : 0);
+                if (!slot_fits((i128)M * t * pmin, (i128)M * t * pmax, S)) return false;
+            }
+        }
+        return true;
+    };
+    if (!fits_with(1)) return false;
+    long long lo = 1, hi = std::max(1LL, M_cap);   // largest M in [1, M_cap] that fits (monotone)
+    while (lo < hi) {
+        const long long mid = (lo + hi + 1) / 2;
+        if (fits_with(mid)) lo = mid; else hi = mid - 1;
+    }
+    L->N = N;
+    L->S = S;
+    L->Kc = Kc;
+    L->J = J;
+    L->segments = NS;
+    L->top_bits = top_bits;
+    L->M = (int)lo;
+    L->signed_prod = sp ? 1 : 0;
+    return true;
+}
+
+int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, int row_outputs,
+                const hikonv_tuning_t *tune, hikonv_layout_t *out) {
+    if (validate_codes(p, q) != HIKONV_OK || K < 1 || K > kMaxK || !out || (dims != 1 && dims != 2))
+        return HIKONV_ERR_INVALID_ARG;
+    fs = fs ? 1 : 0;
+    gs = gs ? 1 : 0;
+    const int forceN = tune ? tune->N : 0, forceS = tune ? tune->S : 0, forceM = tune ? tune->M : 0;
+    if (forceN < 0 || forceS < 0 || forceM < 0) return HIKONV_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    hikonv_layout_t best;
+    bool found = false;
+    if (dims == 1) {
+        // Theorem 2: Gb = ceil(log2 K); widen S until the exact ranges fit
+        const int S_paper = slice_bits(p, q, guard_bits(HIKONV_GB_1D, 1, K, 1));
+        const int maxN = forceN ? forceN : kMaxN1D;
+        for (int S = forceS ? forceS : S_paper; S <= (forceS ? forceS : 31) && !found; ++S) {
+            double best_rate = 0.0;
+            for (int N = forceN ? forceN : 1; N <= maxN; ++N) {
+                hikonv_layout_t c;
+                if (!check_candidate(p, q, fs, gs, K, N, S, true, 1, &c)) continue;
+                const double rate = (double)c.N / c.J;   // outputs per multiply
+                if (rate > best_rate + 1e-9) {
+                    best_rate = rate;
+                    best = c;
+                    found = true;
+                }
+            }
+        }
+        if (found) best.S_paper = S_paper;
+    } else {
+        if (total_terms < 1) return HIKONV_ERR_INVALID_ARG;
+        const CostModel cm;
+        double best_cost = 0.0;
+        const int maxN = forceN ? forceN : kMaxN2D;
+        const int wo = row_outputs > 0 ? row_outputs : 64;
+        for (int N = forceN ? forceN : 1; N <= maxN; ++N) {
+            // a wider slot allows more accumulations between two splits, but may push the kernel
+            // row into several chunks: score every feasible (N, S)
+            for (int S = forceS ? forceS : 31; S >= (forceS ? forceS : 1); --S) {
+                hikonv_layout_t c;
+                if (!check_candidate(p, q, fs, gs, K, N, S, false, total_terms, &c)) continue;
+                const double blocks = (double)(ceil_div(wo, N) + c.J);   // words per output row, halo included
+                const double per_mul = cm.mul_cycles + cm.split_cycles_per_seg * c.segments / (double)c.M;
+                const double cost = blocks * c.J * per_mul / (double)wo; // cycles per output pixel and (ci, kh)
+                if (!found || cost <= best_cost + 1e-12) {      // ties: the narrower slot
+                    best_cost = cost;
+                    best = c;
+                    found = true;
+                }
+            }
+        }
+        if (found) {
+            // reference value of the printed rule for the chosen N (DNN guard bits with the chosen M)
+            best.S_paper = slice_bits(p, q, guard_bits(HIKONV_GB_DNN, best.N, std::min(K, best.Kc), best.M));
+        }
+    }
+    if (!found) return HIKONV_ERR_NO_FIT;
+    if (forceM) {
+        if (forceM > best.M) return HIKONV_ERR_NO_FIT;
+        best.M = forceM;
+    }
+    *out = best;
+    return HIKONV_OK;
+}
+
+// Term counts per product slot for a layout: T[m] = number of code products that land in slot m
+// of one accumulated product (all J chunks).
+static void term_counts(const hikonv_layout_t &L, int K, int *T) {
+    for (int m = 0; m < L.segments; ++m) T[m] = 0;
+    for (int j = 0; j < L.J; ++j) {
+        const int kc = std::min(L.Kc, K - j * L.Kc);
+        for (int m = 0; m < L.segments; ++m) T[m] += pair_count(m, L.N, kc);
+    }
+}
+
+SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int fs, int gs, int K, int M) {
+    SplitConsts c;
+    std::memset(&c, 0, sizeof(c));
+    c.slot_mask = (L.S >= 32) ? 0xFFFFFFFFu : ((1u << L.S) - 1u);
+    const Range fr = code_range(p, fs ? 1 : 0), gr = code_range(q, gs ? 1 : 0);
+    const long long prods[4] = {fr.lo * gr.lo, fr.lo * gr.hi, fr.hi * gr.lo, fr.hi * gr.hi};
+    const long long pmin = *std::min_element(prods, prods + 4);
+    int T[kMaxSegments];
+    term_counts(L, K, T);
+    for (int m = 0; m < L.segments; ++m) {
+        const long long b = -(long long)M * T[m] * pmin;      // >= 0: lifts the most negative sum to 0
+        c.seg_bias[m] = (int32_t)b;
+        c.bias += (uint64_t)b << (L.S * m);
+    }
+    for (int m = 0; m < L.N; ++m)
+        c.carry_bias[m] = c.seg_bias[m] + (m + L.N < L.segments ? c.seg_bias[m + L.N] : 0);
+    return c;
+}
+
+}  // namespace hikonv
+
+using namespace hikonv;
+
+extern "C" int hikonv_plan(int p, int q, int LA, int LB, int mode, int M, int K_fixed, hikonv_plan_t *out) {
+    if (!out || p < 1 || q < 1 || p > 32 || q > 32 || LA < 1 || LB < 1 || LA > 64 || LB > 64) return HIKONV_ERR_INVALID_ARG;
+    if (mode != HIKONV_GB_SINGLE && mode != HIKONV_GB_1D && mode != HIKONV_GB_DNN) return HIKONV_ERR_INVALID_ARG;
+    if (M < 1 || K_fixed < 0) return HIKONV_ERR_INVALID_ARG;
+    hikonv_plan_t best = {0, 0, 0, 0, 0};
+    const int k_lo = K_fixed ? K_fixed : 1, k_hi = K_fixed ? K_fixed : LB;
+    for (int k = k_lo; k <= k_hi; ++k) {
+        for (int n = 1; n <= LA; ++n) {
+            const int Gb = guard_bits(mode, n, k, M);
+            const int S = slice_bits(p, q, Gb);
+            if (p + (long long)(n - 1) * S > LA) break;          // Eq. 7 (monotone in n up to the Gb steps)
+            if (q + (long long)(k - 1) * S > LB) continue;       // Eq. 8
+            const int ops = n * k + (n - 1) * (k - 1);           // Eq. 24
+            if (ops > best.ops) best = {n, k, S, Gb, ops};
+        }
+    }
+    if (best.ops == 0) return HIKONV_ERR_NO_FIT;
+    *out = best;
+    return HIKONV_OK;
+}
+
+extern "C" int hikonv_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int total_terms,
+                             const hikonv_tuning_t *tune, hikonv_layout_t *out) {
+    return make_layout(p, q, f_signed, g_signed, K, dims, total_terms, 0, tune, out);
+}
+
+extern "C" const char *hikonv_status_string(int status) {
+    switch (status) {
+        case HIKONV_OK: return "ok";
+        case HIKONV_ERR_INVALID_ARG: return "invalid argument";
+        case HIKONV_ERR_UNSUPPORTED: return "unsupported configuration";
+        case HIKONV_ERR_NO_FIT: return "no packed layout fits the multiplier";
+        case HIKONV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case HIKONV_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}

@@ -1,0 +1,177 @@
+"""CPU checks of the C interface: the library builds, loads and exports every declared entry
+point; the host-only planning calls agree with the brute-force oracle and with the paper's
+printed numbers; argument validation returns status codes without touching a GPU."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import direct, packed_model as pm, plan as oplan
+from paper_2208_00763_b200 import binding as hk
+from paper_2208_00763_b200 import build as lib_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built_library():
+    lib_build.build()
+    return hk.lib()
+
+
+def _declared_names():
+    text = open(os.path.join(ROOT, "include", "hikonv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hikonv_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound():
+    names = _declared_names()
+    assert "hikonv_pack" in names and "hikonv_conv1d" in names and "hikonv_conv2d" in names
+    raw = ctypes.CDLL(hk.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), "library does not export %s" % n
+    assert sorted(hk.exported_names()) == names
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(hk, "_lib", None)
+    monkeypatch.setattr(hk, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        hk.lib()
+
+
+@pytest.mark.parametrize("mode", [hk.GB_SINGLE, hk.GB_1D, hk.GB_DNN])
+def test_plan_matches_bruteforce_oracle(mode):
+    for LA, LB in ((32, 32), (27, 18)):
+        for p in range(1, 9):
+            for q in range(1, 9):
+                for M in ((1,) if mode != hk.GB_DNN else (1, 4, 21)):
+                    got = hk.plan(p, q, LA, LB, mode, M)
+                    assert got == oplan.search(p, q, LA, LB, mode, M)
+                    for K in (1, 3, 5):
+                        ref = oplan.search(p, q, LA, LB, mode, M, K_fixed=K)
+                        if ref["ops"] == 0:
+                            with pytest.raises(hk.HikonvError):
+                                hk.plan(p, q, LA, LB, mode, M, K)
+                        else:
+                            assert hk.plan(p, q, LA, LB, mode, M, K) == ref
+
+
+def test_plan_printed_counts():
+    assert hk.plan(4, 4)["ops"] == 13 and hk.plan(8, 8)["ops"] == 5
+    assert hk.plan(1, 1, 27, 18)["ops"] == 60 and hk.plan(4, 4, 27, 18)["ops"] == 8 and hk.plan(8, 8, 27, 18)["ops"] == 2
+    assert hk.plan(1, 1)["ops"] == 113 and hk.plan(1, 1, 33, 32)["ops"] == 128
+    four = hk.plan(4, 4, 32, 32, hk.GB_1D, 1, 3)
+    assert (four["N"], four["K"], four["Gb"], four["S"]) == (3, 3, 2, 10)
+
+
+def test_plan_rejects_bad_arguments():
+    out = hk.PlanT()
+    lib = hk.lib()
+    assert lib.hikonv_plan(0, 4, 32, 32, 0, 1, 0, ctypes.byref(out)) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_plan(4, 4, 32, 32, 7, 1, 0, ctypes.byref(out)) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_plan(4, 4, 32, 32, 0, 1, 0, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_plan(8, 8, 4, 4, 0, 1, 0, ctypes.byref(out)) == hk.ERR_NO_FIT
+    assert hk.status_string(hk.ERR_NO_FIT) and hk.status_string(99) == "unknown status"
+
+
+def _extreme_vectors(p, q, fs, gs, n, K):
+    flo, fhi = (-(1 << (p - 1)), (1 << (p - 1)) - 1) if fs else (0, (1 << p) - 1)
+    glo, ghi = (-(1 << (q - 1)), (1 << (q - 1)) - 1) if gs else (0, (1 << q) - 1)
+    out = []
+    for fv in (flo, fhi):
+        for gv in (glo, ghi):
+            out.append(([fv] * n, [gv] * K))
+    out.append(([flo if i % 2 else fhi for i in range(n)], [ghi if i % 2 else glo for i in range(K)]))
+    return out
+
+
+def _model_conv1d(f, g, L, bias_per_slot):
+    """The kernel's arithmetic in big integers: chunked kernel, carries added before the split,
+    slots lifted by a bias instead of Eq. 29's borrow increment; 32-bit operands, 64-bit product."""
+    N, S, Kc, J = L["N"], L["S"], L["Kc"], L["J"]
+    n_out = len(f) + len(g) - 1
+    nb = (n_out + N - 1) // N
+    fpad = list(f) + [0] * ((nb + 1) * N)
+    A = [pm.pack(fpad[x * N:(x + 1) * N], S) for x in range(nb)]
+    Bw = [pm.pack(g[j * Kc:(j + 1) * Kc], S) for j in range(J)]
+    lim = 1 << 31
+    for a in A:
+        assert (-lim <= a < lim) if L["signed_prod"] else (0 <= a < 2 * lim)
+    for b in Bw:
+        assert (-lim <= b < lim) if L["signed_prod"] else (0 <= b < 2 * lim)
+    bias = sum(b << (S * m) for m, b in enumerate(bias_per_slot))
+    y, prev_hi = [], bias >> (S * N)
+    for x in range(nb):
+        Q = bias + sum(A[x - j] * Bw[j] for j in range(J) if x - j >= 0)
+        assert 0 <= Q < (1 << 64)
+        D = Q + prev_hi
+        for m in range(N):
+            carry_bias = bias_per_slot[m] + (bias_per_slot[m + N] if m + N < len(bias_per_slot) else 0)
+            y.append(((D >> (S * m)) & ((1 << S) - 1)) - carry_bias)
+        prev_hi = Q >> (S * N)
+    return y[:n_out]
+
+
+@pytest.mark.parametrize("signed", [False, True])
+def test_layout_1d_is_exact_on_extreme_codes(signed):
+    # every (p, K) of the bitwidth sweep: the layout the kernels use reproduces the plain
+    # convolution on the inputs that stress the slots hardest
+    for p in range(1, 9):
+        for K in (1, 2, 3, 5, 7, 9):
+            L = hk.layout(p, p, signed, signed, K, 1)
+            assert L["J"] == -(-K // L["Kc"]) and L["segments"] == L["N"] + L["Kc"] - 1
+            assert L["S"] >= L["S_paper"] and L["S"] * (L["segments"] - 1) < 64
+            lo_f = -(1 << (p - 1)) if signed else 0
+            hi_f = (1 << (p - 1)) - 1 if signed else (1 << p) - 1
+            pmin = min(a * b for a in (lo_f, hi_f) for b in (lo_f, hi_f))
+            T = [0] * L["segments"]
+            for j in range(L["J"]):
+                kc = min(L["Kc"], K - j * L["Kc"])
+                for n in range(L["N"]):
+                    for k in range(kc):
+                        T[n + k] += 1
+            bias = [-t * pmin for t in T]
+            for f, g in _extreme_vectors(p, p, signed, signed, 3 * L["N"] + 2, K):
+                assert _model_conv1d(f, g, L, bias) == direct.conv1d_full(f, g).tolist()
+
+
+def test_layout_2d_known_cases():
+    c3 = hk.layout(4, 4, True, True, 3, 2, 64 * 3)
+    assert c3["J"] == 1 and c3["Kc"] == 3 and c3["M"] >= 1 and c3["S"] * (c3["segments"] - 1) < 64
+    forced = hk.layout(4, 4, True, True, 3, 2, 64 * 3, {"N": 2})
+    assert forced["N"] == 2
+    with pytest.raises(hk.HikonvError):
+        hk.layout(8, 8, True, True, 3, 2, 64 * 3, {"N": 4})     # four 8-bit codes never fit 32 bits with products
+    with pytest.raises(hk.HikonvError):
+        hk.layout(4, 4, True, True, 3, 2, 64 * 3, {"N": 3, "S": 13, "M": 1000})
+
+
+def test_device_entry_points_validate_before_touching_cuda():
+    lib = hk.lib()
+    assert lib.hikonv_conv1d(None, 10, None, 3, 4, 4, 0, 0, None, 0, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_conv1d(8, 10, 8, 3, 9, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 8, 1, None, None) == hk.ERR_UNSUPPORTED     # 64x64 emulation not built
+    assert lib.hikonv_conv1d(8, 10, 8, 0, 4, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_pack(None, 10, 4, 0, 10, 3, 32, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_pack(8, 10, 4, 0, 10, 4, 32, 8, None) == hk.ERR_NO_FIT
+    assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 2, 1, 4, 4, 0, 0, 8, 0, 0, 0, 0, 256, 1 << 20, 0, None, None) == hk.ERR_UNSUPPORTED
+    assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 0, 0, 0, 0, None, 0, 0, None, None) == hk.ERR_WORKSPACE
+    assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 1, 40, 0, 15, 256, 1 << 20, 0, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_maxpool2x2_i8(None, 1, 1, 4, 4, 0, None, None) == hk.ERR_INVALID_ARG
+    assert hk.conv2d_workspace_bytes(64, 64, 3) >= 64 * 3 * 64 * 4
+    assert hk.conv1d_host_workspace_bytes(1000, 3) >= 1000 + 3 + 4 * 1002
+
+
+def test_multiply_counts():
+    # packed 4-bit K = 3: one multiply per block of N = 3 outputs; comparator: K per output
+    n = 3000
+    assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 3)
+    assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_UNPACKED_IMAD) == (n + 2) * 3
+    packed = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_PACKED32)
+    unpacked = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_UNPACKED_IMAD)
+    macs = 2 * 16 * 10 * 12 * 8 * 9
+    assert 0 < packed < macs / 2 and unpacked >= macs

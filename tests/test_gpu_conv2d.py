@@ -1,0 +1,143 @@
+"""GPU parity, 2-D layers and the compact CNN, against the int64 oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import direct
+from paper_2208_00763_b200 import binding as hk
+from paper_2208_00763_b200 import inputs
+from paper_2208_00763_b200 import network
+from gpu_util import assert_exact, dev
+
+pytestmark = pytest.mark.gpu
+
+ALGOS = [hk.ALGO_PACKED32, hk.ALGO_UNPACKED_IMAD]
+
+
+def _layer(x, w, pad, p, q, xs, ws, algo, requant=None, tune=None):
+    return hk.conv2d(dev(x), dev(w), pad, p, q, xs, ws, requant=requant, algo=algo, tune=tune)
+
+
+SHAPES = [
+    # B, Ci, H, W, Co, K, pad
+    (1, 1, 1, 1, 1, 1, 0),
+    (1, 3, 5, 7, 2, 3, 1),
+    (2, 5, 9, 11, 7, 3, 1),
+    (3, 16, 14, 14, 40, 3, 1),      # several images per tile
+    (2, 8, 6, 70, 20, 3, 1),        # wide rows: row segments
+    (1, 4, 20, 300, 16, 3, 1),
+    (2, 6, 8, 9, 5, 3, 0),          # valid convolution
+    (1, 7, 10, 12, 9, 5, 2),        # 5x5: the kernel row is cut into chunks
+    (2, 3, 9, 10, 4, 7, 3),
+    (2, 12, 5, 6, 36, 1, 0),        # 1x1
+    (1, 2, 4, 5, 3, 2, 1),          # even kernel
+    (5, 9, 3, 4, 70, 3, 1),         # more than 64 output channels, tiny images
+]
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("shape", SHAPES)
+def test_layer_shapes(shape, algo):
+    B, Ci, H, W, Co, K, pad = shape
+    for (p, q, xs, ws) in ((4, 4, True, True), (4, 4, False, True), (8, 4, False, True), (2, 2, False, False)):
+        x, w = inputs.conv2d_case(B, Ci, H, W, Co, K, p, q, xs, ws, seed=sum(shape) + p)
+        ref = direct.conv2d_nchw(x, w, pad)
+        assert_exact(_layer(x, w, pad, p, q, xs, ws, algo), ref, "%s p=%d q=%d" % (shape, p, q))
+
+
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_every_bitwidth(bits):
+    for signed in (False, True):
+        x, w = inputs.conv2d_case(2, 10, 7, 13, 12, 3, bits, bits, signed, signed, seed=bits)
+        ref = direct.conv2d_nchw(x, w, 1)
+        for algo in ALGOS:
+            assert_exact(_layer(x, w, 1, bits, bits, signed, signed, algo), ref, "bits=%d signed=%d algo=%d" % (bits, signed, algo))
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4])
+def test_forced_words_per_block(n):
+    x, w = inputs.conv2d_case(2, 40, 9, 17, 24, 3, 4, 4, True, True, seed=40 + n)
+    ref = direct.conv2d_nchw(x, w, 1)
+    assert_exact(_layer(x, w, 1, 4, 4, True, True, hk.ALGO_PACKED32, tune={"N": n}), ref, "N=%d" % n)
+    # a short split period exercises many splits per output
+    assert_exact(_layer(x, w, 1, 4, 4, True, True, hk.ALGO_PACKED32, tune={"N": n, "M": 1}), ref, "N=%d M=1" % n)
+    assert_exact(_layer(x, w, 1, 4, 4, True, True, hk.ALGO_PACKED32, tune={"N": n, "tile": 1}), ref, "N=%d one row per tile" % n)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_extreme_codes(algo):
+    for (p, q, xs, ws) in ((4, 4, True, True), (4, 4, False, True), (8, 4, False, True), (8, 8, True, True), (1, 1, True, True)):
+        for x, w in inputs.extreme_2d(2, 70, 6, 10, 8, 3, p, q, xs, ws):
+            assert_exact(_layer(x, w, 1, p, q, xs, ws, algo), direct.conv2d_nchw(x, w, 1), "extreme p=%d q=%d" % (p, q))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_requantize(algo):
+    x, w = inputs.conv2d_case(2, 32, 10, 12, 16, 3, 4, 4, True, True, seed=77)
+    acc = direct.conv2d_nchw(x, w, 1)
+    for (shift, lo, hi) in ((6, -8, 7), (0, -128, 127), (5, 0, 15), (3, 0, 255)):
+        got = _layer(x, w, 1, 4, 4, True, True, algo, requant=(shift, lo, hi))
+        torch.cuda.synchronize()
+        g = got.cpu().numpy()
+        g = g.astype(np.int64) if lo < 0 else g.view(np.uint8).astype(np.int64)
+        assert np.array_equal(g, direct.requant(acc, shift, lo, hi)), (shift, lo, hi)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_c3_layer_sampled_images(algo):
+    # full-size launch (batch 32); the oracle checks three whole images of it
+    s = inputs.C3_SHAPE
+    x, w = inputs.layer_case(s)
+    got = _layer(x, w, s["pad"], s["p"], s["q"], s["x_signed"], s["w_signed"], algo, requant=(s["shift"], s["lo"], s["hi"]))
+    torch.cuda.synchronize()
+    g = got.cpu().numpy().astype(np.int64)
+    for b in (0, 13, 31):
+        ref = direct.requant(direct.conv2d_nchw(x[b:b + 1], w, s["pad"]), s["shift"], s["lo"], s["hi"])
+        assert np.array_equal(g[b:b + 1], ref), "image %d" % b
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_c4_layer_sampled_images(algo):
+    s = inputs.C4_SHAPE
+    x, w = inputs.layer_case(s)
+    assert abs(float((x == 0).mean()) - (0.3 + 0.7 / 16)) < 0.01
+    got = _layer(x, w, s["pad"], s["p"], s["q"], s["x_signed"], s["w_signed"], algo)
+    torch.cuda.synchronize()
+    g = got.cpu().numpy().astype(np.int64)
+    for b in (0, 31, 63):
+        assert np.array_equal(g[b:b + 1], direct.conv2d_nchw(x[b:b + 1], w, s["pad"])), "image %d" % b
+
+
+def test_host_buffer_entry_point():
+    x, w = inputs.conv2d_case(2, 8, 9, 10, 12, 3, 4, 4, False, True, seed=5)
+    h_x = torch.from_numpy(inputs.to_storage(x)).pin_memory()
+    h_w = torch.from_numpy(inputs.to_storage(w)).pin_memory()
+    h_o = torch.empty((2, 12, 9, 10), dtype=torch.int32).pin_memory()
+    ws = torch.empty(hk.conv2d_host_workspace_bytes(2, 8, 9, 10, 12, 3, 1, False), dtype=torch.uint8, device="cuda")
+    hk.conv2d_host(h_x, h_w, 1, 4, 4, False, True, h_o, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(h_o.numpy().astype(np.int64), direct.conv2d_nchw(x, w, 1))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_compact_cnn_small_batch(algo):
+    x, layers, head_w = inputs.c5_network(batch=2, H=32, W=64)
+    ref_head, ref_acts = direct.cnn_forward(x, layers, head_w)
+    net = network.CompactCnn(layers, head_w, device="cuda")
+    head, acts = net.forward(dev(x), algo=algo, keep_activations=True)
+    for i, (a, r) in enumerate(zip(acts, ref_acts)):
+        assert_exact(a, r, "layer %d" % (i + 1))
+    assert_exact(head, ref_head, "head")
+
+
+def test_compact_cnn_full_size_sampled():
+    # the benchmark configuration (batch 64, 3x160x320); the oracle checks two images end to end
+    x, layers, head_w = inputs.c5_network()
+    net = network.CompactCnn(layers, head_w, device="cuda")
+    head, _ = net.forward(dev(x))
+    torch.cuda.synchronize()
+    g = head.cpu().numpy().astype(np.int64)
+    assert g.shape == (64, 36, 10, 20)
+    for b in (0, 63):
+        ref_head, _ = direct.cnn_forward(x[b:b + 1], layers, head_w)
+        assert np.array_equal(g[b:b + 1], ref_head), "image %d" % b

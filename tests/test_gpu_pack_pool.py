@@ -1,0 +1,56 @@
+"""GPU parity for the standalone packing kernel and the 2x2 max-pool."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import direct
+from paper_2208_00763_b200 import binding as hk
+from paper_2208_00763_b200 import inputs
+from gpu_util import dev
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_pack_matches_eq5():
+    rng = np.random.default_rng(1)
+    for signed in (False, True):
+        for (bits, S, N, wb) in ((4, 10, 3, 32), (4, 13, 3, 32), (1, 3, 11, 32), (8, 18, 2, 32), (4, 10, 7, 64), (8, 21, 3, 64),
+                                 (2, 6, 5, 32), (4, 4, 8, 32)):
+            for n in (1, N, 1000, 100003):
+                v = inputs.uniform_codes(rng, (n,), bits, signed)
+                words = hk.pack(dev(v), bits, signed, S, N, wb)
+                torch.cuda.synchronize()
+                got = words.cpu().numpy()
+                got = got.view(np.uint32).astype(np.uint64) if wb == 32 else got.view(np.uint64)
+                assert np.array_equal(got, direct.pack_words(v, S, N, wb)), (bits, S, N, wb, n, signed)
+
+
+def test_pack_reproduces_the_printed_multiplicands():
+    vals = {}
+    with open(os.path.join(GOLDEN, "worked_example_f32.txt")) as fh:
+        for line in fh:
+            if "=" in line and not line.startswith("#"):
+                k, v = line.split("=", 1)
+                vals[k.strip()] = v.strip()
+    f = np.array([int(t) for t in vals["f"].split()])
+    g = np.array([int(t) for t in vals["g"].split()])
+    # the figure stores the first element in the top slot: feed the mirrored sequences
+    A = hk.pack(dev(f[::-1].copy()), 4, False, 10, 3, 32)
+    B = hk.pack(dev(g[::-1].copy()), 4, False, 10, 2, 32)
+    torch.cuda.synchronize()
+    assert int(A[0]) == int(vals["multiplicand_f"]) and int(B[0]) == int(vals["multiplicand_g"])
+    assert int(A[0]) * int(B[0]) == int(vals["product"])
+
+
+def test_maxpool():
+    rng = np.random.default_rng(2)
+    for signed in (False, True):
+        for shape in ((1, 1, 2, 2), (2, 3, 6, 10), (3, 5, 7, 9), (4, 16, 40, 80)):
+            v = inputs.uniform_codes(rng, shape, 8, signed)
+            out = hk.maxpool2x2_i8(dev(v), signed)
+            torch.cuda.synchronize()
+            got = inputs.from_storage(out.cpu().numpy(), signed)
+            assert np.array_equal(got, direct.maxpool2x2(v)), (shape, signed)
