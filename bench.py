@@ -1,0 +1,452 @@
+#!/usr/bin/env python
+"""Benchmark of the packed low-bit convolution path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+
+A "step" is one pass of the whole hot path over the 1-D bitwidth sweep: 48 full convolutions of a
+2^24-element signal (p = q = 1..8, K in {3,5,7}, unsigned and signed), each launch reading its own
+16 MiB input and writing its own 64 MiB int32 output, so a step streams about 3.9 GB and nothing
+is served from L2.  The metric is effective multiply-accumulates of the plain definition per
+second.  The line also carries the roofline of the dominant kernel, the same path timed end to
+end from pinned host buffers, the oracle timed on the host cores, and (unless --no-extra) the
+2-D layer and full-network workloads with the one-product-per-multiply comparator beside them.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "effective low-bit conv MAC/s"
+UNIT = "MAC/s"
+HBM_FALLBACK_GBS = 6650.0            # earlier pool measurement, used only when MEASURED_PEAKS.json is absent
+IMAD_PER_CLK_PER_SM = 64             # 32-bit integer multiply-add lanes per SM per clock (confirmed by microbenchmark)
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of each kernel,
+# with the SHA-256 of the kernel source at capture time (a changed source voids the figure).
+NCU_TRAFFIC = {
+    # "conv1d_packed": {"sha256": "...", "bytes_per_output": ...},
+}
+
+
+def _source_hash(name: str) -> str:
+    with open(os.path.join(ROOT, "paper_2208_00763_b200", "csrc", name), "rb") as fh:
+        return hashlib.sha256(fh.read()).hexdigest()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return HBM_FALLBACK_GBS, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [t.strip() for t in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm and CPU baseline: the oracle as it stands, on the host cores
+# ----------------------------------------------------------------------------------------------
+
+def oracle_inputs(sample_len: int, seed_offset: int = 0):
+    from paper_2208_00763_b200 import inputs
+    data = []
+    for case in inputs.c2_cases(sample_len):
+        f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"],
+                                  case["seed"] + seed_offset)
+        data.append((f, g))
+    return data
+
+
+def oracle_sweep(data):
+    """One pass of the sweep through the oracle (int64 direct convolution).  Returns (MACs, seconds)."""
+    from oracle import direct
+    macs = 0.0
+    t0 = time.perf_counter()
+    for f, g in data:
+        direct.conv1d_full(f, g)
+        macs += float(f.size + g.size - 1) * g.size
+    return macs, time.perf_counter() - t0
+
+
+def cpu_baseline(sample_len: int):
+    """The oracle as it stands on the host cores: the 48 sweep cases at `sample_len`, repeated for about 10 s."""
+    from oracle import direct
+    data = oracle_inputs(sample_len)
+    oracle_sweep(data[:2])
+    macs, secs, passes = 0.0, 0.0, 0
+    while secs < 10.0 and passes < 50:
+        m, s = oracle_sweep(data)
+        macs += m
+        secs += s
+        passes += 1
+    return {"value": macs / secs, "unit": UNIT, "cores": direct.num_threads(), "kind": "oracle",
+            "sample": "%d pass(es) over the 48 sweep cases at signal length %d (benchmark length 2^24), int64 direct "
+                      "convolution, OpenMP over outputs, %.1f s of CPU time" % (passes, sample_len, secs)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import direct
+    sample_len = 1 << 22
+    data = oracle_inputs(sample_len)
+    for _ in range(args.warmup):
+        oracle_sweep(data[:4])
+    total_macs, total_secs = 0.0, 0.0
+    for _ in range(args.steps):
+        m, s = oracle_sweep(data)
+        total_macs += m
+        total_secs += s
+    value = total_macs / total_secs
+    sample = "each step: the 48 sweep cases at signal length %d (1/4 of the benchmark length)" % sample_len
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total_secs / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": "c2: 1-D bitwidth sweep, 48 full convolutions (p=q=1..8, K=3/5/7, unsigned+signed); " + sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": direct.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2208_00763_b200 import binding as hk
+    from paper_2208_00763_b200 import inputs, network
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    hk.lib()
+    hbm_peak_gbs, sm_max_mhz, peak_kind = measured_peaks()
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    imad_peak = sms * IMAD_PER_CLK_PER_SM * sm_max_mhz * 1e6        # multiply-adds per second
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms: float) -> float:
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- the sweep: every rank runs the whole sweep on its own data (weak scaling, no exchange)
+    length = args.length
+    cases = inputs.c2_cases(length)
+    host_f, host_g = [], []
+    for case in cases:
+        f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"],
+                                  case["seed"] + 100000 * rank)
+        host_f.append(torch.from_numpy(inputs.to_storage(f)))
+        host_g.append(torch.from_numpy(inputs.to_storage(g)))
+    d_f = [t.to(dev) for t in host_f]
+    d_g = [t.to(dev) for t in host_g]
+    d_y = [torch.empty(length + c["K"] - 1, dtype=torch.int32, device=dev) for c in cases]
+    macs_per_step = float(sum((length + c["K"] - 1) * c["K"] for c in cases))
+    outputs_per_step = float(sum(length + c["K"] - 1 for c in cases))
+
+    def sweep(algo):
+        for c, f, g, y in zip(cases, d_f, d_g, d_y):
+            hk.conv1d(f, g, c["p"], c["q"], c["f_signed"], c["g_signed"], algo=algo, out=y)
+
+    def timed_graph(fn, steps, warmup):
+        """Warm up eagerly, capture one step in a CUDA graph, replay it `steps` times between events."""
+        side = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(side):
+            for _ in range(max(warmup, 3)):
+                fn()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fn()
+        graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(steps):
+            graph.replay()
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    total_ms = max_over_ranks(timed_graph(lambda: sweep(hk.ALGO_PACKED32), args.steps, args.warmup))
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = total_ms / args.steps
+    value = world * macs_per_step / (ms_per_step * 1e-3)
+    launches_per_step = len(cases)
+
+    # roofline of the dominant kernel (conv1d_packed): 1 input byte + 4 output bytes per output
+    avg_launch_s = total_ms * 1e-3 / (args.steps * launches_per_step)
+    bytes_per_launch = 5.0 * outputs_per_step / launches_per_step
+    achieved_gbs = bytes_per_launch / avg_launch_s / 1e9
+    traffic = None
+    rec = NCU_TRAFFIC.get("conv1d_packed")
+    if rec and rec.get("sha256") == _source_hash("hikonv_conv1d.cu"):
+        traffic = rec["bytes_per_output"] * outputs_per_step / launches_per_step
+    roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": hbm_peak_gbs, "unit": "GB/s",
+                "frac": achieved_gbs / hbm_peak_gbs, "traffic": traffic, "peak_kind": "of " + peak_kind,
+                "kernel": "conv1d_packed_kernel", "bytes_per_output": 5}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int64", "data": "synthetic",
+        "config": {"workload": "c2: 1-D bitwidth sweep, 48 full convolutions of length 2^%d (p=q=1..8, K=3/5/7, unsigned+signed), "
+                               "int8-stored codes in, int32 out" % (length.bit_length() - 1),
+                   "l2": "inputs larger than L2: every launch of a step has its own input and output buffers (%.1f GB per step)"
+                         % ((outputs_per_step * 4 + len(cases) * length) / 1e9),
+                   "launch": "one CUDA graph replay per step"},
+        "gpu_launches": args.steps * launches_per_step,
+        "roofline": roofline,
+    }
+    if clocks is not None:
+        line["clocks"] = clocks
+
+    if rank == 0 and world == 1:
+        # ---- end to end: pinned host buffers through the host-buffer entry point, copies inside the timed region
+        ws = torch.empty(hk.conv1d_host_workspace_bytes(length, 7), dtype=torch.uint8, device=dev)
+        pin_f = [t.pin_memory() for t in host_f]
+        pin_g = [t.pin_memory() for t in host_g]
+        pin_y = torch.empty(length + 6, dtype=torch.int32).pin_memory()
+
+        def e2e_step():
+            for c, f, g in zip(cases, pin_f, pin_g):
+                hk.conv1d_host(f, g, c["p"], c["q"], c["f_signed"], c["g_signed"], pin_y[: length + c["K"] - 1], ws)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+        line["e2e"] = {"value": macs_per_step / (e2e_ms * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": int(sum(t.numel() for t in host_f) + sum(t.numel() for t in host_g)),
+                       "d2h_bytes_per_step": int(outputs_per_step * 4), "ms_per_step": e2e_ms}
+        del pin_f, pin_y, ws
+
+        # ---- the comparator on the same sweep, and per-case times
+        if not args.no_extra:
+            extra = {}
+            un_ms = timed_graph(lambda: sweep(hk.ALGO_UNPACKED_IMAD), args.steps, args.warmup) / args.steps
+            extra["c2_unpacked"] = {"value": macs_per_step / (un_ms * 1e-3), "unit": UNIT, "ms_per_step": un_ms,
+                                    "hbm_frac": 5.0 * outputs_per_step / (un_ms * 1e-3) / 1e9 / hbm_peak_gbs}
+            del d_y
+            extra["c2_by_bits"] = per_bitwidth_table(torch, hk, cases, d_f, d_g, length)
+            del d_f, d_g
+            torch.cuda.empty_cache()
+            extra.update(layer_workloads(torch, np, hk, inputs, network, dev, imad_peak))
+            line["extra"] = extra
+        line["cpu_baseline"] = cpu_baseline(1 << 22)
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def per_bitwidth_table(torch, hk, cases, d_f, d_g, length):
+    """Microseconds per launch for every sweep case, packed and comparator.  Each timed graph holds 12 launches
+    that rotate over the three inputs of the same bitwidth and signedness and over three output buffers
+    (240 MB per cycle), so no launch finds its data in L2."""
+    table = {}
+    ys = [torch.empty(length + 6, dtype=torch.int32, device=d_f[0].device) for _ in range(3)]
+    for i, c in enumerate(cases):
+        same = [j for j, o in enumerate(cases) if o["p"] == c["p"] and o["f_signed"] == c["f_signed"]]
+        row = {}
+        for name, algo in (("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD)):
+            def fn():
+                for r in range(12):
+                    hk.conv1d(d_f[same[r % len(same)]], d_g[i], c["p"], c["q"], c["f_signed"], c["g_signed"], algo=algo,
+                              out=ys[r % 3][: length + c["K"] - 1])
+            fn()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(3):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            row[name] = e0.elapsed_time(e1) * 1e3 / 36
+        table["p%d_K%d_%s" % (c["p"], c["K"], "s" if c["f_signed"] else "u")] = row
+    return table
+
+
+def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
+    """2-D layers and the compact CNN: event-timed launches with an L2 flush before each."""
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def time_fn(fn, iters=10):
+        fn()
+        fn()
+        torch.cuda.synchronize()
+        total = 0.0
+        for _ in range(iters):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            total += e0.elapsed_time(e1)
+        return total / iters
+
+    for name, shape in (("c3", inputs.C3_SHAPE), ("c4", inputs.C4_SHAPE)):
+        x, w = inputs.layer_case(shape)
+        d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
+        d_w = torch.from_numpy(inputs.to_storage(w)).to(dev)
+        ws = torch.empty(hk.conv2d_workspace_bytes(shape["Ci"], shape["Co"], shape["K"]), dtype=torch.uint8, device=dev)
+        rq = (shape["shift"], shape["lo"], shape["hi"]) if shape["requant"] else None
+        Ho = shape["H"] + 2 * shape["pad"] - shape["K"] + 1
+        Wo = shape["W"] + 2 * shape["pad"] - shape["K"] + 1
+        o = torch.empty((shape["B"], shape["Co"], Ho, Wo), dtype=torch.int8 if rq else torch.int32, device=dev)
+        macs = float(shape["B"]) * shape["Co"] * Ho * Wo * shape["Ci"] * shape["K"] ** 2
+        rec = {"macs": macs}
+        for key, algo in (("packed", hk.ALGO_PACKED32), ("unpacked", hk.ALGO_UNPACKED_IMAD)):
+            ms = time_fn(lambda: hk.conv2d(d_x, d_w, shape["pad"], shape["p"], shape["q"], shape["x_signed"], shape["w_signed"],
+                                           requant=rq, algo=algo, workspace=ws, out=o))
+            muls = hk.conv2d_multiplies(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
+                                        shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], algo)
+            rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT,
+                        "roofline": {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": imad_peak / 1e12,
+                                     "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / imad_peak, "traffic": None}}
+        rec["layout"] = hk.layout(shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], shape["K"], 2, shape["Ci"] * shape["K"])
+        rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
+        out[name] = rec
+        del d_x, d_w, o
+
+    x, layers, head_w = inputs.c5_network()
+    d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
+    net = network.CompactCnn(layers, head_w, device=dev)
+    macs = 0.0
+    H, W = x.shape[2], x.shape[3]
+    for L in layers:
+        Co, Ci, K, _ = L["w"].shape
+        macs += float(x.shape[0]) * Co * H * W * Ci * K * K
+        if L["pool"]:
+            H, W = H // 2, W // 2
+    macs += float(x.shape[0]) * head_w.shape[0] * H * W * head_w.shape[1]
+    rec = {"macs": macs}
+    for key, algo in (("packed", hk.ALGO_PACKED32), ("unpacked", hk.ALGO_UNPACKED_IMAD)):
+        ms = time_fn(lambda: net.forward(d_x, algo=algo), iters=5)
+        rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT}
+    rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
+    out["c5"] = rec
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the comparator, per-case and 2-D workloads")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--length", type=int, default=1 << 24, help="signal length of the sweep (benchmark value: 2^24)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
