@@ -38,7 +38,8 @@ typedef enum {
     HIKONV_ERR_UNSUPPORTED = 2, /* stride != 1, an algorithm that is not built, pad >= K               */
     HIKONV_ERR_NO_FIT = 3,      /* no (N >= 1, S) satisfies the operand, slot and accumulator bounds   */
     HIKONV_ERR_WORKSPACE = 4,   /* workspace pointer null/misaligned or workspace_bytes too small      */
-    HIKONV_ERR_CUDA = 5         /* a CUDA runtime call failed (see cudaGetLastError)                   */
+    HIKONV_ERR_CUDA = 5,        /* a CUDA runtime call failed (see cudaGetLastError)                   */
+    HIKONV_ERR_TOO_LARGE = 6    /* the layer needs more scratch than the built-in static buffer holds  */
 } hikonv_status;
 
 typedef enum {
@@ -163,6 +164,34 @@ int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *
                   int algo, const hikonv_tuning_t *tune, void *stream);
 
 size_t hikonv_conv2d_workspace_bytes(int Ci, int Co, int K);
+
+/*
+ * hikonv_conv2d_static_scratch - hikonv_conv2d for callers that cannot provide device scratch.
+ * (The paper has no counterpart; this is a deployment convenience of this library.)
+ *
+ * Some callers cannot allocate device memory at the point where they run a layer: code that runs
+ * inside a memory-capped serving process whose pool is owned by another component, plug-ins that are
+ * handed input and output tensors only, and real-time loops where cudaMalloc (which synchronises the
+ * device and can fail late) is forbidden after start-up.  For them the packed kernel rows go to a
+ * fixed buffer of HIKONV_STATIC_SCRATCH_BYTES that lives inside the library image on every GPU that
+ * loads it, from load until the process exits.  Arguments are those of hikonv_conv2d without the
+ * workspace pair; results are identical.
+ *
+ *   - Limit: hikonv_conv2d_workspace_bytes(Ci, Co, K) must not exceed HIKONV_STATIC_SCRATCH_BYTES,
+ *     otherwise HIKONV_ERR_TOO_LARGE is returned and nothing is launched.
+ *   - The function calls no cudaMalloc/cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the buffer's device address (once per device, with that
+ *     device current).  Make that first call during start-up, before any stream capture.
+ *   - All calls on a device share the one buffer and it keeps the previous call's contents.  Nothing
+ *     in it has to start at zero: every call rewrites all words it later reads.  Two calls whose
+ *     kernels can overlap on the GPU (different streams, no dependency between them) race on the
+ *     buffer; order them on one stream or with events.
+ */
+#define HIKONV_STATIC_SCRATCH_BYTES (4u << 20)
+int hikonv_conv2d_static_scratch(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,
+                                 int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out,
+                                 int requant, int shift, int lo, int hi, int algo, const hikonv_tuning_t *tune,
+                                 void *stream);
 
 /* Device scratch needed by hikonv_conv2d_host: x, w, out and the kernel workspace. */
 size_t hikonv_conv2d_host_workspace_bytes(int B, int Ci, int H, int W, int Co, int K, int pad, int requant);

@@ -14,7 +14,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhikonv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE = range(7)
+STATIC_SCRATCH_BYTES = 4 << 20
 ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD = 0, 1, 2
 GB_SINGLE, GB_1D, GB_DNN = 0, 1, 2
 
@@ -51,6 +52,8 @@ _SIGNATURES = {
     "hikonv_conv2d": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz, _i,
                            ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d_workspace_bytes": (_sz, [_i, _i, _i]),
+    "hikonv_conv2d_static_scratch": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i,
+                                          ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d_host_workspace_bytes": (_sz, [_i] * 8),
     "hikonv_conv2d_host": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz,
                                 _i, ctypes.POINTER(TuningT), _vp]),
@@ -181,6 +184,27 @@ def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_sig
                                int(x_signed), int(w_signed), out.data_ptr(), 1 if requant else 0, shift, lo, hi,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), algo, _tune(tune),
                                _stream(stream)), "hikonv_conv2d")
+    return out
+
+
+def conv2d_static_scratch(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_signed: bool, w_signed: bool,
+                          out: torch.Tensor, requant: Optional[tuple] = None, algo: int = ALGO_PACKED32, tune=None,
+                          stride: int = 1, stream=None) -> torch.Tensor:
+    """``conv2d`` without a workspace: the packed kernel rows go to the library's built-in device buffer.
+
+    For callers that may not allocate device memory when the layer runs (they own only the input and
+    output tensors, or allocation is forbidden after start-up).  ``out`` must be preallocated by the
+    caller.  Layers whose packed weights exceed ``STATIC_SCRATCH_BYTES`` raise ``ERR_TOO_LARGE``; calls
+    that may overlap on the GPU must be ordered by the caller, since they share the buffer.
+    """
+    B, Ci, H, W = d_x.shape
+    Co, Ci2, K, K2 = d_w.shape
+    if Ci != Ci2 or K != K2:
+        raise ValueError("weight shape does not match the input")
+    shift, lo, hi = requant if requant else (0, 0, 0)
+    _check(lib().hikonv_conv2d_static_scratch(_dev_i8(d_x, "d_x"), B, Ci, H, W, _dev_i8(d_w, "d_w"), Co, K, stride, pad, p, q,
+                                              int(x_signed), int(w_signed), out.data_ptr(), 1 if requant else 0, shift, lo, hi,
+                                              algo, _tune(tune), _stream(stream)), "hikonv_conv2d_static_scratch")
     return out
 
 

@@ -16,6 +16,7 @@
 // times TN channels, the k dimension runs over (ci, kh, j).
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 
 #include "hikonv_cuda.cuh"
 
@@ -472,6 +473,45 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
     rc = launch_status();
     if (rc != HIKONV_OK) return rc;
     return launch_conv2d(s, x_signed != 0, st);
+}
+
+// ---- scratch that needs no allocation: a fixed buffer inside the library image, one copy per GPU
+static __device__ __align__(256) unsigned char g_static_scratch[HIKONV_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void *g_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle, so the address is asked for once per device and cached.
+int static_scratch_address(void **out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HIKONV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return HIKONV_ERR_CUDA;
+        g_scratch_ptr[dev] = ptr;
+    }
+    *out = g_scratch_ptr[dev];
+    return HIKONV_OK;
+}
+}  // namespace
+
+extern "C" int hikonv_conv2d_static_scratch(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,
+                                            int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out,
+                                            int requant, int shift, int lo, int hi, int algo, const hikonv_tuning_t *tune,
+                                            void *stream) {
+    if (Ci < 1 || Co < 1 || K < 1) return HIKONV_ERR_INVALID_ARG;
+    const size_t need = hikonv_conv2d_workspace_bytes(Ci, Co, K);
+    if (need > (size_t)HIKONV_STATIC_SCRATCH_BYTES) return HIKONV_ERR_TOO_LARGE;
+    void *scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != HIKONV_OK) return rc;
+    // the packing kernel writes every word the layer kernel reads, so stale contents are harmless
+    return hikonv_conv2d(d_x, B, Ci, H, W, d_w, Co, K, stride, pad, p, q, x_signed, w_signed, d_out, requant, shift, lo, hi,
+                         scratch, (size_t)HIKONV_STATIC_SCRATCH_BYTES, algo, tune, stream);
 }
 
 extern "C" size_t hikonv_conv2d_host_workspace_bytes(int B, int Ci, int H, int W, int Co, int K, int pad, int requant) {

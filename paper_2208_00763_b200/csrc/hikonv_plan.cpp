@@ -269,6 +269,7 @@ extern "C" const char *hikonv_status_string(int status) {
         case HIKONV_ERR_NO_FIT: return "no packed layout fits the multiplier";
         case HIKONV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case HIKONV_ERR_CUDA: return "CUDA runtime error";
+        case HIKONV_ERR_TOO_LARGE: return "layer needs more scratch than the built-in static buffer holds";
         default: return "unknown status";
     }
 }
