@@ -217,8 +217,17 @@ def run_ours(args):
         return float(t.item())
 
     # ---- the sweep: every rank runs the whole sweep on its own data (weak scaling, no exchange)
+    if args.workload != "c2":
+        return run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks,
+                              imad_peak)
     length = args.length
     cases = inputs.c2_cases(length)
+    if args.cases:
+        keep = set(args.cases.split(","))
+        cases = [c for c in cases if "p%d_K%d_%s" % (c["p"], c["K"], "s" if c["f_signed"] else "u") in keep]
+        if not cases:
+            raise SystemExit("--cases matched nothing (names look like p4_K3_s)")
+        cases = cases * args.case_copies      # separate buffers per copy keep a short sweep out of L2
     host_f, host_g = [], []
     for case in cases:
         f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"],
@@ -280,8 +289,8 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int64", "data": "synthetic",
-        "config": {"workload": "c2: 1-D bitwidth sweep, 48 full convolutions of length 2^%d (p=q=1..8, K=3/5/7, unsigned+signed), "
-                               "int8-stored codes in, int32 out" % (length.bit_length() - 1),
+        "config": {"workload": "c2: 1-D bitwidth sweep, %d full convolutions of length 2^%d (p=q=1..8, K=3/5/7, unsigned+signed), "
+                               "int8-stored codes in, int32 out" % (len(cases), length.bit_length() - 1),
                    "l2": "inputs larger than L2: every launch of a step has its own input and output buffers (%.1f GB per step)"
                          % ((outputs_per_step * 4 + len(cases) * length) / 1e9),
                    "launch": "one CUDA graph replay per step"},
@@ -291,7 +300,7 @@ def run_ours(args):
     if clocks is not None:
         line["clocks"] = clocks
 
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.cases:
         # ---- end to end: pinned host buffers through the host-buffer entry point, copies inside the timed region
         ws = torch.empty(hk.conv1d_host_workspace_bytes(length, 7), dtype=torch.uint8, device=dev)
         pin_f = [t.pin_memory() for t in host_f]
@@ -330,6 +339,95 @@ def run_ours(args):
             line["extra"] = extra
         line["cpu_baseline"] = cpu_baseline(1 << 22)
 
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks, imad_peak):
+    """Main line for --workload c3/c4/c5: a step is one layer (or one network pass) on this rank's batch,
+    timed with one event pair per step and an L2 flush (256 MB memset) before each step."""
+    algo = hk.ALGO_PACKED32 if args.algo == "packed" else hk.ALGO_UNPACKED_IMAD
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    launches = 0
+    if args.workload in ("c3", "c4"):
+        shape = dict(inputs.C3_SHAPE if args.workload == "c3" else inputs.C4_SHAPE)
+        if args.batch:
+            shape["B"] = args.batch
+        shape["seed"] = shape["seed"] + 1000 * rank
+        x, w = inputs.layer_case(shape)
+        d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
+        d_w = torch.from_numpy(inputs.to_storage(w)).to(dev)
+        ws = torch.empty(hk.conv2d_workspace_bytes(shape["Ci"], shape["Co"], shape["K"]), dtype=torch.uint8, device=dev)
+        rq = (shape["shift"], shape["lo"], shape["hi"]) if shape["requant"] else None
+        Ho = shape["H"] + 2 * shape["pad"] - shape["K"] + 1
+        Wo = shape["W"] + 2 * shape["pad"] - shape["K"] + 1
+        o = torch.empty((shape["B"], shape["Co"], Ho, Wo), dtype=torch.int8 if rq else torch.int32, device=dev)
+        macs = float(shape["B"]) * shape["Co"] * Ho * Wo * shape["Ci"] * shape["K"] ** 2
+        muls = hk.conv2d_multiplies(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
+                                    shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], algo)
+
+        def step():
+            hk.conv2d(d_x, d_w, shape["pad"], shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], requant=rq,
+                      algo=algo, workspace=ws, out=o)
+        launches_per_step = 2
+        name = "%s: 2-D layer %dx%dx%dx%d -> %d channels, %dx%d, pad %d, p=%d q=%d" % (
+            args.workload, shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["K"], shape["pad"],
+            shape["p"], shape["q"])
+        h2d = d_x.numel() + d_w.numel()
+        d2h = o.numel() * o.element_size()
+    else:
+        x, layers, head_w = inputs.c5_network(seed=5 + 1000 * rank, batch=args.batch or 64)
+        d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
+        net = network.CompactCnn(layers, head_w, device=dev)
+        macs, muls = 0.0, None
+        H, W = x.shape[2], x.shape[3]
+        for L in layers:
+            Co, Ci, K, _ = L["w"].shape
+            macs += float(x.shape[0]) * Co * H * W * Ci * K * K
+            if L["pool"]:
+                H, W = H // 2, W // 2
+        macs += float(x.shape[0]) * head_w.shape[0] * H * W * head_w.shape[1]
+
+        def step():
+            net.forward(d_x, algo=algo)
+        launches_per_step = 2 * 9 + 4
+        name = "c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head" % x.shape[0]
+        h2d = d_x.numel()
+        d2h = x.shape[0] * 36 * H * W * 4
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    total = 0.0
+    for _ in range(args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step()
+        e1.record()
+        e1.synchronize()
+        total += e0.elapsed_time(e1)
+    barrier()
+    total = max_over_ranks(total)
+    clocks = sampler.stop() if rank == 0 else None
+    ms = total / args.steps
+    line = {
+        "metric": METRIC, "value": world * macs / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int64" if args.algo == "packed" else "int32", "data": "synthetic",
+        "config": {"workload": name, "algo": args.algo, "l2": "flushed before every step (256 MB memset outside the timed events)"},
+        "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
+    }
+    if muls is not None:
+        line["roofline"] = {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": imad_peak / 1e12,
+                            "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / imad_peak, "traffic": None,
+                            "kernel": "conv2d_kernel", "peak_kind": "derived: SMs x 64 lanes/clk x max SM clock"}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -442,6 +540,12 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the comparator, per-case and 2-D workloads")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--length", type=int, default=1 << 24, help="signal length of the sweep (benchmark value: 2^24)")
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"],
+                    help="c2 = 1-D sweep (default, the benchmark step); c3/c4 = one 2-D layer; c5 = the compact CNN")
+    ap.add_argument("--cases", default="", help="c2 only: comma-separated subset such as p4_K3_s,p8_K7_u (for profiling)")
+    ap.add_argument("--case-copies", type=int, default=3, help="with --cases: buffer copies per case")
+    ap.add_argument("--batch", type=int, default=0, help="c3/c4/c5: override the batch size (for profiling)")
+    ap.add_argument("--algo", default="packed", choices=["packed", "unpacked"], help="c3/c4/c5: which kernel the main line times")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
