@@ -10,7 +10,10 @@
 //   splits  y[xN+m] = ((D_x >> S m) & mask) - carry_bias[m],  m < N       (Algorithm 2's shift
 //           and mask; the per-slot bias replaces the sign-borrow increment of Eq. 29)
 // Outputs are staged per warp in shared memory and written with coalesced 16-byte stores.
+#include <cstring>
+
 #include "hikonv_cuda.cuh"
+#include "hikonv_conv1d_tc.h"
 
 namespace hikonv {
 
@@ -274,6 +277,19 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     const long long n_out = (long long)len + K - 1;
     const int y_aligned16 = ((uintptr_t)d_y % 16 == 0) ? 1 : 0;
 
+    // tune->tile > 0 selects the shuffle-based kernels below (any N, J, K); otherwise the
+    // register-resident kernels are used whenever they are instantiated for the layout
+    const bool want_tc = !(tune && tune->tile > 0);
+    Conv1dTcParams tp;
+    std::memset(&tp, 0, sizeof(tp));
+    tp.f = d_f; tp.g = d_g; tp.y = d_y; tp.len = (long long)len; tp.n_out = n_out; tp.K = K;
+    tp.g_signed = g_signed ? 1 : 0;
+    tp.aligned = (y_aligned16 && ((uintptr_t)d_f % 4 == 0)) ? 1 : 0;
+
+    if (algo == HIKONV_ALGO_UNPACKED_IMAD && want_tc && conv1d_unpacked_tc_available(K)) {
+        tp.n_tiles = (n_out + 32 * 16 - 1) / (32 * 16);
+        return launch_conv1d_unpacked_tc(tp, K, f_signed != 0, st);
+    }
     if (algo == HIKONV_ALGO_UNPACKED_IMAD) {
         Conv1dUnpackedParams up;
         up.f = d_f; up.g = d_g; up.y = d_y; up.len = (long long)len; up.n_out = n_out; up.K = K;
@@ -289,6 +305,17 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     if (rc != HIKONV_OK) return rc;
     if (L.N > kMaxN1D) return HIKONV_ERR_UNSUPPORTED;
     const SplitConsts sc = make_split_consts(L, p, q, f_signed, g_signed, K, 1);
+
+    if (want_tc && conv1d_packed_tc_available(L.N, L.J)) {
+        const int per_tile = conv1d_tc_outputs_per_tile(L.N);
+        tp.n_tiles = (n_out + per_tile - 1) / per_tile;
+        tp.S = L.S; tp.Kc = L.Kc; tp.hi_shift = L.S * L.N; tp.mask = sc.slot_mask; tp.bias = sc.bias;
+        for (int m = 0; m < kMaxN1D; ++m) {
+            tp.seg_shift[m] = m < L.N ? L.S * m : 0;
+            tp.carry_bias[m] = m < L.N ? sc.carry_bias[m] : 0;
+        }
+        return launch_conv1d_packed_tc(tp, L.N, L.J, L.signed_prod != 0, f_signed != 0, st);
+    }
 
     Conv1dParams kp;
     kp.f = d_f; kp.g = d_g; kp.y = d_y; kp.len = (long long)len; kp.n_out = n_out;

@@ -1,0 +1,33 @@
+// Interface between hikonv_conv1d.cu (argument checks, layout) and the register-resident 1-D kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "hikonv_internal.h"
+
+namespace hikonv {
+
+struct Conv1dTcParams {
+    const int8_t *f;
+    const int8_t *g;
+    int32_t *y;
+    long long len;
+    long long n_out;
+    long long n_tiles;       // warp tiles of 32 * L outputs covering n_out
+    int K, S, Kc;
+    int hi_shift;            // S * N
+    int g_signed;
+    int aligned;             // f is 4-byte aligned and y is 16-byte aligned
+    uint32_t mask;
+    uint64_t bias;
+    int seg_shift[kMaxN1D];
+    int32_t carry_bias[kMaxN1D];
+};
+
+int conv1d_tc_outputs_per_tile(int N);
+bool conv1d_packed_tc_available(int N, int J);
+int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool signed_prod, bool f_signed, cudaStream_t st);
+bool conv1d_unpacked_tc_available(int K);
+int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool f_signed, cudaStream_t st);
+
+}  // namespace hikonv

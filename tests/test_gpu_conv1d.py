@@ -39,6 +39,18 @@ def test_bitwidth_sweep_small(bits, signed, algo):
 
 @pytest.mark.parametrize("algo", ALGOS)
 @pytest.mark.parametrize("signed", [False, True])
+def test_bitwidth_sweep_shuffle_kernels(signed, algo):
+    # tile > 0 selects the general kernels (any N, J, K), which the automatic choice only uses for
+    # layouts the register-resident kernels are not instantiated for
+    for bits in range(1, 9):
+        for K in (3, 5, 7):
+            f, g = inputs.conv1d_case(40009, K, bits, bits, signed, signed, seed=bits * 10 + K)
+            assert_exact(_run(f, g, bits, bits, signed, signed, algo, tune={"tile": 4}), direct.conv1d_full(f, g),
+                         "general kernel p=%d K=%d signed=%d" % (bits, K, signed))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("signed", [False, True])
 def test_extreme_codes(signed, algo):
     for bits in range(1, 9):
         for K in (3, 5, 7):
