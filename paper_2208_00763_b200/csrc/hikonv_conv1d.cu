@@ -287,7 +287,7 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     tp.aligned = (y_aligned16 && ((uintptr_t)d_f % 4 == 0)) ? 1 : 0;
 
     if (algo == HIKONV_ALGO_UNPACKED_IMAD && want_tc && conv1d_unpacked_tc_available(K)) {
-        tp.n_tiles = (n_out + 32 * 16 - 1) / (32 * 16);
+        tp.n_tiles = (n_out + 32 * 32 - 1) / (32 * 32);
         return launch_conv1d_unpacked_tc(tp, K, f_signed != 0, st);
     }
     if (algo == HIKONV_ALGO_UNPACKED_IMAD) {

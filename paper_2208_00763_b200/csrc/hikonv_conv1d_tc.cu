@@ -18,11 +18,12 @@ constexpr int kThreadsTc = 256;
 constexpr int kWarpsTc = kThreadsTc / 32;
 
 __host__ __device__ constexpr int gcd_c(int a, int b) { return b == 0 ? a : gcd_c(b, a % b); }
-// blocks per lane: L = R N is a multiple of 4 and at least 12
+// blocks per lane: L = R N is a multiple of 4 and at least kMinRun
+constexpr int kMinRun = 24;
 __host__ __device__ constexpr int blocks_per_lane(int N) {
     const int step = 4 / gcd_c(N, 4);
     int r = step;
-    while (r * N < 12) r += step;
+    while (r * N < kMinRun) r += step;
     return r;
 }
 
@@ -89,41 +90,60 @@ __device__ __forceinline__ void store_run(int32_t *y, long long n_out, long long
     }
 }
 
-template <int N, int J, bool SP, bool FS>
+// SC > 0 fixes the slot width at compile time (shifts and masks become immediates); SC == 0 reads it
+// from the parameters.
+template <int N, int J, int SC, bool SP, bool FS>
 __global__ void __launch_bounds__(kThreadsTc) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
     constexpr int R = blocks_per_lane(N);
     constexpr int L = R * N;
     constexpr int HW = (J * N + 3) / 4;          // words in front of the run
     constexpr int NWORDS = HW + L / 4;
-    __shared__ uint32_t s_B[J];
     __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
-    if (threadIdx.x < J) {                        // pack the kernel chunk B_j (Eq. 5 on g)
+
+    const int S = SC > 0 ? SC : p.S;
+    const uint32_t mask = SC > 0 ? ((1u << (SC > 0 ? SC : 1)) - 1u) : p.mask;
+    const int hi_shift = SC > 0 ? SC * N : p.hi_shift;
+    // the kernel chunks B_j (Eq. 5 on g); every lane builds them itself from warp-uniform loads
+    uint32_t Bw[J];
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
         uint32_t b = 0;
         for (int k = 0; k < p.Kc; ++k) {
-            const int idx = threadIdx.x * p.Kc + k;
+            const int idx = j * p.Kc + k;
             if (idx < p.K) {
                 const int8_t raw = __ldg(p.g + idx);
                 const int32_t v = p.g_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
-                b += (uint32_t)v << (p.S * k);
+                b += (uint32_t)v << (S * k);
             }
         }
-        s_B[threadIdx.x] = b;
+        Bw[j] = b;
     }
-    __syncthreads();
-    uint32_t Bw[J];
-#pragma unroll
-    for (int j = 0; j < J; ++j) Bw[j] = s_B[j];
     uint32_t slot_pow[N];
 #pragma unroll
-    for (int n = 0; n < N; ++n) slot_pow[n] = 1u << (p.S * n);
+    for (int n = 0; n < N; ++n) slot_pow[n] = 1u << (S * n);
 
     const int lane = threadIdx.x & 31;
-    for (long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5); t < p.n_tiles; t += (long long)gridDim.x * kWarpsTc) {
+    const long long stride = (long long)gridDim.x * kWarpsTc;
+    long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5);
+    uint32_t wn[NWORDS];
+    bool fast_n = false;
+    if (t < p.n_tiles) {
         const long long tile0 = t * (32 * L);
-        const bool fast = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
-        const long long e0 = tile0 + lane * L;
+        fast_n = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
+        load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast_n, wn);
+    }
+    while (t < p.n_tiles) {
+        const long long tile0 = t * (32 * L);
+        const bool fast = fast_n;
         uint32_t w[NWORDS];
-        load_words<NWORDS, HW>(p.f, p.len, e0, fast, w);
+#pragma unroll
+        for (int i = 0; i < NWORDS; ++i) w[i] = wn[i];
+        t += stride;
+        if (t < p.n_tiles) {                       // next tile's codes are in flight while this one is computed
+            const long long next0 = t * (32 * L);
+            fast_n = p.aligned && next0 >= 4 * HW && next0 + 32 * L <= p.len;
+            load_words<NWORDS, HW>(p.f, p.len, next0 + lane * L, fast_n, wn);
+        }
 
         // A_x for x = -J .. R-1 (index x + J); element n of block x sits at byte 4 HW + x N + n of w
         uint32_t A[R + J];
@@ -149,10 +169,12 @@ __global__ void __launch_bounds__(kThreadsTc) conv1d_packed_tc_kernel(const Conv
             if (x >= 0) {
                 const uint64_t D = Q + (uint64_t)carry;
 #pragma unroll
-                for (int m = 0; m < N; ++m)
-                    out[x * N + m] = (int32_t)(shr64_lo(D, p.seg_shift[m]) & p.mask) - p.carry_bias[m];
+                for (int m = 0; m < N; ++m) {
+                    const int sh = SC > 0 ? SC * m : p.seg_shift[m];
+                    out[x * N + m] = (int32_t)(shr64_lo(D, sh) & mask) - p.carry_bias[m];
+                }
             }
-            carry = shr64_lo(Q, p.hi_shift);
+            carry = shr64_lo(Q, hi_shift);
         }
         store_run<L>(p.y, p.n_out, tile0, lane, fast, s_stage[threadIdx.x >> 5], out);
     }
@@ -161,26 +183,38 @@ __global__ void __launch_bounds__(kThreadsTc) conv1d_packed_tc_kernel(const Conv
 // Comparator: 16 outputs per lane, one product per 32-bit multiply-add.
 template <int K, bool FS>
 __global__ void __launch_bounds__(kThreadsTc) conv1d_unpacked_tc_kernel(const Conv1dTcParams p) {
-    constexpr int L = 16;
+    constexpr int L = 32;
     constexpr int HW = (K - 1 + 3) / 4;
     constexpr int NWORDS = HW + L / 4;
-    __shared__ int32_t s_g[K];
     __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
-    if (threadIdx.x < K) {
-        const int8_t raw = __ldg(p.g + threadIdx.x);
-        s_g[threadIdx.x] = p.g_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
-    }
-    __syncthreads();
     int32_t gk[K];
 #pragma unroll
-    for (int k = 0; k < K; ++k) gk[k] = s_g[k];
+    for (int k = 0; k < K; ++k) {
+        const int8_t raw = __ldg(p.g + k);
+        gk[k] = p.g_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+    }
     const int lane = threadIdx.x & 31;
-    for (long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5); t < p.n_tiles; t += (long long)gridDim.x * kWarpsTc) {
+    const long long stride = (long long)gridDim.x * kWarpsTc;
+    long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5);
+    uint32_t wn[NWORDS];
+    bool fast_n = false;
+    if (t < p.n_tiles) {
         const long long tile0 = t * (32 * L);
-        const bool fast = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
-        const long long e0 = tile0 + lane * L;
+        fast_n = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
+        load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast_n, wn);
+    }
+    while (t < p.n_tiles) {
+        const long long tile0 = t * (32 * L);
+        const bool fast = fast_n;
         uint32_t w[NWORDS];
-        load_words<NWORDS, HW>(p.f, p.len, e0, fast, w);
+#pragma unroll
+        for (int i = 0; i < NWORDS; ++i) w[i] = wn[i];
+        t += stride;
+        if (t < p.n_tiles) {
+            const long long next0 = t * (32 * L);
+            fast_n = p.aligned && next0 >= 4 * HW && next0 + 32 * L <= p.len;
+            load_words<NWORDS, HW>(p.f, p.len, next0 + lane * L, fast_n, wn);
+        }
         int32_t e[L + K - 1];                       // e[i] = f[e0 - (K-1) + i]
 #pragma unroll
         for (int i = 0; i < L + K - 1; ++i) {
@@ -199,12 +233,23 @@ __global__ void __launch_bounds__(kThreadsTc) conv1d_unpacked_tc_kernel(const Co
     }
 }
 
-static unsigned tc_grid(long long n_tiles) {
+// Persistent launch: as many CTAs as fit on the device at once (occupancy query, cached per kernel),
+// fewer when the problem is small; each warp then walks tiles with a grid-wide stride.
+template <typename Kernel>
+static int launch_persistent(Kernel kernel, const Conv1dTcParams &p, cudaStream_t st) {
+    static int resident = 0;                       // CTAs per SM for this kernel instantiation
+    if (resident == 0) {
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kThreadsTc, 0) != cudaSuccess || occ < 1) occ = 1;
+        resident = occ;
+    }
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long want = (n_tiles + kWarpsTc - 1) / kWarpsTc;
-    const long long cap = (long long)sms * 32;
-    return (unsigned)(want < cap ? want : cap);
+    const long long want = (p.n_tiles + kWarpsTc - 1) / kWarpsTc;
+    const long long cap = (long long)sms * resident;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    kernel<<<grid, kThreadsTc, 0, st>>>(p);
+    return launch_status();
 }
 
 int conv1d_tc_outputs_per_tile(int N) {
@@ -216,13 +261,11 @@ int conv1d_tc_outputs_per_tile(int N) {
     }
 }
 
-template <int N, int J>
-static int launch_packed_tc_nj(const Conv1dTcParams &p, bool sp, bool fs, cudaStream_t st) {
-    const unsigned grid = tc_grid(p.n_tiles);
-    if (!sp) conv1d_packed_tc_kernel<N, J, false, false><<<grid, kThreadsTc, 0, st>>>(p);
-    else if (fs) conv1d_packed_tc_kernel<N, J, true, true><<<grid, kThreadsTc, 0, st>>>(p);
-    else conv1d_packed_tc_kernel<N, J, true, false><<<grid, kThreadsTc, 0, st>>>(p);
-    return launch_status();
+template <int N, int J, int SC>
+static int launch_packed_tc_njs(const Conv1dTcParams &p, bool sp, bool fs, cudaStream_t st) {
+    if (!sp) return launch_persistent(conv1d_packed_tc_kernel<N, J, SC, false, false>, p, st);
+    if (fs) return launch_persistent(conv1d_packed_tc_kernel<N, J, SC, true, true>, p, st);
+    return launch_persistent(conv1d_packed_tc_kernel<N, J, SC, true, false>, p, st);
 }
 
 bool conv1d_packed_tc_available(int N, int J) {
@@ -234,7 +277,15 @@ bool conv1d_packed_tc_available(int N, int J) {
 }
 
 int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool sp, bool fs, cudaStream_t st) {
-#define HK_NJ(n, j) if (N == n && J == j) return launch_packed_tc_nj<n, j>(p, sp, fs, st);
+    // layouts of the p = q bitwidth sweep (K = 3, 5, 7) with the slot width as a compile-time constant
+#define HK_NJS(n, j, sc) if (N == n && J == j && p.S == sc) return launch_packed_tc_njs<n, j, sc>(p, sp, fs, st);
+    HK_NJS(11, 1, 3) HK_NJS(8, 1, 4) HK_NJS(6, 1, 6) HK_NJS(5, 1, 6) HK_NJS(5, 1, 7) HK_NJS(5, 2, 7) HK_NJS(4, 1, 8) HK_NJS(4, 2, 9)
+    HK_NJS(3, 1, 10) HK_NJS(3, 2, 11) HK_NJS(3, 3, 11) HK_NJS(3, 1, 12) HK_NJS(3, 2, 13) HK_NJS(3, 3, 13)
+    HK_NJS(2, 2, 14) HK_NJS(2, 3, 15) HK_NJS(2, 4, 15) HK_NJS(2, 2, 16) HK_NJS(2, 3, 17) HK_NJS(2, 4, 17)
+    HK_NJS(2, 2, 18) HK_NJS(2, 3, 19) HK_NJS(2, 4, 19)
+#undef HK_NJS
+    // any other layout: slot width read at run time
+#define HK_NJ(n, j) if (N == n && J == j) return launch_packed_tc_njs<n, j, 0>(p, sp, fs, st);
     HK_NJ(1, 1) HK_NJ(2, 1) HK_NJ(3, 1) HK_NJ(4, 1) HK_NJ(5, 1) HK_NJ(6, 1) HK_NJ(7, 1) HK_NJ(8, 1) HK_NJ(9, 1) HK_NJ(10, 1)
     HK_NJ(11, 1) HK_NJ(12, 1)
     HK_NJ(2, 2) HK_NJ(3, 2) HK_NJ(4, 2) HK_NJ(5, 2) HK_NJ(6, 2)
@@ -247,12 +298,10 @@ int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool sp, bool
 bool conv1d_unpacked_tc_available(int K) { return K == 3 || K == 5 || K == 7; }
 
 int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool fs, cudaStream_t st) {
-    const unsigned grid = tc_grid(p.n_tiles);
 #define HK_K(k)                                                                                   \
     if (K == k) {                                                                                 \
-        if (fs) conv1d_unpacked_tc_kernel<k, true><<<grid, kThreadsTc, 0, st>>>(p);               \
-        else conv1d_unpacked_tc_kernel<k, false><<<grid, kThreadsTc, 0, st>>>(p);                 \
-        return launch_status();                                                                   \
+        if (fs) return launch_persistent(conv1d_unpacked_tc_kernel<k, true>, p, st);              \
+        return launch_persistent(conv1d_unpacked_tc_kernel<k, false>, p, st);                     \
     }
     HK_K(3) HK_K(5) HK_K(7)
 #undef HK_K
