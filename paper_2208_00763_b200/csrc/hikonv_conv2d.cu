@@ -8,12 +8,20 @@
 //     Q = bias + sum_{ci, kh, j} A[b][ci][h+kh][xb - j] * Bw[co][ci][kh][j]
 // where A packs N neighbouring input pixels (Eq. 5) and Bw packs N (or all K) taps of the REVERSED
 // kernel row (g = W[co][ci][kh][K-1:0], Theorem 3).  Slot m < N of Q holds partial sums of pixel
-// xN + m, slot m >= N those of pixel (x+1)N + (m-N): the overlap-add of Theorem 2.  After at most
-// M accumulated (ci, kh) pairs the slots are extracted into int32 sums and Q restarts at `bias`.
+// xN + m, slot m >= N those of pixel (x+1)N + (m-N): the overlap-add of Theorem 2.
 //
 // A CTA computes TR consecutive output rows (one row segment each) times TCO output channels; it
 // is a register-tiled integer "GEMM" over packed words: each thread owns TM consecutive positions
 // times TN channels, the k dimension runs over (ci, kh, j).
+//
+// Split.  After at most M accumulated (ci, kh) pairs the accumulators are "flushed": the upper
+// slots of position i-1 are added to position i (Theorem 2 on the products, as in Section V-A), the
+// N low slots are kept, and for every m < N the 32-bit window (D >> S m) is added to an int32 sum
+//     V[m] = Y[m] + 2^S Y[m+1] + 2^(2S) Y[m+2] + ...   (mod 2^32)
+// where Y[m] is the running sum of slot m.  Nothing is masked per flush; the slots are separated
+// once at the end by back-substitution (Y[N-1] = V[N-1], Y[m] = V[m] - sum_k 2^(S k) Y[m+k]), which
+// is exact because every Y fits 32 bits.  This is Algorithm 2's shift-and-mask split with the mask
+// postponed; slots are biased (non-negative) instead of sign-corrected (Eq. 29).
 #include <algorithm>
 #include <cstring>
 #include <mutex>
@@ -22,7 +30,7 @@
 
 namespace hikonv {
 
-constexpr int kThreads2D = 256;
+constexpr int kMaxThreads2D = 256;
 constexpr int kMaxN2DSeg = 8;      // N + Kc - 1 <= 2 N <= 8
 
 struct Conv2dParams {
@@ -30,7 +38,7 @@ struct Conv2dParams {
     const uint32_t *wp;        // packed weights [Ci*K*J][CoP]
     void *out;
     int B, Ci, H, W, Co, CoP, K, pad, Ho, Wo, Hp;
-    int S, J, Kc, nhi, M;      // nhi = Kc - 1 slots above the N low ones
+    int S, J, Kc, M;
     int X;                     // output blocks per row
     int NSEG, XO, XB;          // row segments, output blocks per segment, positions per segment (XO + J)
     int TR, TMX, TNX, TCO, CK;
@@ -38,9 +46,8 @@ struct Conv2dParams {
     int b_off;                 // word offset of the weight tile in shared memory (multiple of 4: 16-byte loads)
     int requant, shift, lo, hi;
     int total_rows;            // B * Ho
-    uint32_t mask;
+    int flush_chunks;          // channel chunks accumulated between two splits (CK * K * flush_chunks <= M)
     uint64_t bias;
-    int seg_shift[kMaxN2DSeg];
     int32_t carry_bias[kMaxN2D];
 };
 
@@ -53,18 +60,34 @@ struct AccType<true> {
     typedef int32_t type;
 };
 
-// N: pixels per packed word; TM x TN: per-thread tile (positions x channels); UNPACKED: comparator
-// (N == 1, one tap per word, 32-bit multiply-add, int32 accumulators); SP: signed product;
-// XS: signed activations.
-template <int N, int TM, int TN, bool UNPACKED, bool SP, bool XS>
-__global__ void __launch_bounds__(kThreads2D) conv2d_kernel(const Conv2dParams p) {
+// One multiply-accumulate of the k loop: the packed 32x32->64 product of Eq. 9 added to the 64-bit
+// accumulator, or (comparator) one 32-bit product added to an int32 sum.
+template <bool UNPACKED, bool SP>
+__device__ __forceinline__ void mac(typename AccType<UNPACKED>::type &acc, uint32_t a, uint32_t b) {
+    if constexpr (UNPACKED) {
+        acc += (int32_t)a * (int32_t)b;
+    } else if constexpr (SP) {
+        acc += (uint64_t)((int64_t)(int32_t)a * (int64_t)(int32_t)b);
+    } else {
+        acc += (uint64_t)a * (uint64_t)b;
+    }
+}
+
+// N: pixels per packed word; SC: slot width when known at compile time (0: read from the parameters);
+// TM x TN: per-thread tile (positions x channels); UNPACKED: comparator (N == 1, one tap per word,
+// 32-bit multiply-add, int32 accumulators); SP: signed product; XS: signed activations;
+// KT, JT: kernel size and chunks per kernel row when known at compile time (0, 0: read from the
+// parameters; the (kh, j) loops are then not unrolled).
+template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, bool XS, int KT, int JT>
+__global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dParams p) {
     typedef typename AccType<UNPACKED>::type acc_t;
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t *As = smem;                                   // [CK][a_plane]
     uint32_t *Bs = As + p.b_off;                           // [CK*K*J][TCO], 16-byte aligned
     int *s_row = (int *)(Bs + p.CK * p.K * p.J * p.TCO);   // [NRmax] input offset of each staged row, -1 = zero row
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, nthreads = blockDim.x;
+    const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
     const int tn = tid % p.TNX, tm = tid / p.TNX;
     const int seg = blockIdx.x % p.NSEG;
     const int R0 = (blockIdx.x / p.NSEG) * p.TR;
@@ -76,32 +99,33 @@ __global__ void __launch_bounds__(kThreads2D) conv2d_kernel(const Conv2dParams p
     const int bl = Rlast / p.Ho;
     const int NR = (bl * p.Hp + (Rlast - bl * p.Ho) + p.K - 1) - Rp0 + 1;
     const int TP = TRe * p.XB;                              // positions of this tile
+    const int S = SC > 0 ? SC : p.S;
 
-    for (int rl = tid; rl < NR; rl += kThreads2D) {
+    for (int rl = tid; rl < NR; rl += nthreads) {
         const int rp = Rp0 + rl;
         const int b = rp / p.Hp, hi = rp - b * p.Hp - p.pad;
         s_row[rl] = (b < p.B && hi >= 0 && hi < p.H) ? (b * p.Ci * p.H + hi) * p.W : -1;
     }
 
-    // this thread's positions: smem offset of the packed word for (kh = 0, j = 0), and validity
-    int off[TM];
+    // this thread's positions: shared-memory address of the packed word for (ci = 0, kh = 0, j = 0)
+    const uint32_t *aptr[TM];
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
         const int pos = tm * TM + i;
+        int off = p.lead;                                    // idle position: reads valid memory, result dropped
         if (pos < TP) {
             const int r = pos / p.XB, xb = pos - r * p.XB;
             const int R = R0 + r;
             const int b = R / p.Ho;
-            off[i] = p.lead + ((b * p.Hp + (R - b * p.Ho)) - Rp0) * p.XB + xb;
-        } else {
-            off[i] = p.lead;                                 // idle position: reads valid memory, result dropped
+            off = p.lead + ((b * p.Hp + (R - b * p.Ho)) - Rp0) * p.XB + xb;
         }
+        aptr[i] = As + off;
     }
 
     acc_t acc[TM][TN];
-    // int32 sums kept as uint32: the biased partial sums may wrap, the final difference is exact
-    uint32_t outv[UNPACKED ? 1 : TM][UNPACKED ? 1 : N][UNPACKED ? 1 : TN];
-    uint32_t carry[UNPACKED ? 1 : N][UNPACKED ? 1 : TN];
+    // running window sums and the last position's upper-slot windows; uint32 arithmetic wraps by design
+    uint32_t V[UNPACKED ? 1 : TM][UNPACKED ? 1 : N][UNPACKED ? 1 : TN];
+    uint32_t C[UNPACKED ? 1 : N][UNPACKED ? 1 : TN];
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -112,74 +136,83 @@ __global__ void __launch_bounds__(kThreads2D) conv2d_kernel(const Conv2dParams p
 #pragma unroll
             for (int m = 0; m < N; ++m)
 #pragma unroll
-                for (int t = 0; t < TN; ++t) outv[i][m][t] = 0;
+                for (int t = 0; t < TN; ++t) V[i][m][t] = 0;
 #pragma unroll
         for (int m = 0; m < N; ++m)
 #pragma unroll
-            for (int t = 0; t < TN; ++t) carry[m][t] = 0;
+            for (int t = 0; t < TN; ++t) C[m][t] = 0;
     }
-    int cnt = 0, nflush = 0;
+    int nflush = 0, chunks_since_flush = 0;
 
-    // Split of the 64-bit accumulators (Algorithm 2's shift-and-mask on biased slots): slots
-    // 0..N-1 go to this position, slots N.. to the next position of the row (Theorem 2).
     auto flush = [&]() {
         if constexpr (!UNPACKED) {
+            const int SN = S * N;
+            const uint64_t low_mask = (1ull << SN) - 1ull;
 #pragma unroll
-        for (int t = 0; t < TN; ++t) {
+            for (int t = 0; t < TN; ++t) {
+                uint32_t upper = 0;                          // slots N.. of the previous position (fits 32 bits)
 #pragma unroll
-            for (int i = 0; i < TM; ++i) {
-                const uint64_t Q = (uint64_t)acc[i][t];
+                for (int i = 0; i < TM; ++i) {
+                    const uint64_t Q = (uint64_t)acc[i][t];
+                    uint64_t D = (i == 0) ? Q : Q + (uint64_t)upper;      // Theorem 2: carry of the block before
+                    upper = (uint32_t)(Q >> SN);
+                    D &= low_mask;
 #pragma unroll
-                for (int m = 0; m < N; ++m) outv[i][m][t] += shr64_lo(Q, p.seg_shift[m]) & p.mask;
-#pragma unroll
-                for (int m = 0; m < N; ++m) {
-                    if (m < p.nhi) {
-                        const uint32_t f = shr64_lo(Q, p.seg_shift[N + m < kMaxN2DSeg ? N + m : 0]) & p.mask;
-                        if (i + 1 < TM) outv[i + 1 < TM ? i + 1 : 0][m][t] += f;
-                        else carry[m][t] += f;
-                    }
+                    for (int m = 0; m < N; ++m) V[i][m][t] += (uint32_t)(D >> (S * m));
+                    acc[i][t] = (acc_t)p.bias;
                 }
-                acc[i][t] = (acc_t)p.bias;
+#pragma unroll
+                for (int m = 0; m < N; ++m) C[m][t] += upper >> (S * m);   // goes to the next thread's first position
             }
-        }
-        ++nflush;
+            ++nflush;
         }
     };
 
     const int HW = p.H * p.W;
     const int KJ = p.K * p.J;
-    const int words_per_plane = NR * p.XB;
     uint32_t slot_pow[N];
 #pragma unroll
-    for (int n = 0; n < N; ++n) slot_pow[n] = UNPACKED ? 1u : (1u << (p.S * n));
+    for (int n = 0; n < N; ++n) slot_pow[n] = UNPACKED ? 1u : (1u << (S * n));
     const int col_seg0 = (seg * p.XO - p.J) * N + p.K - 1 - p.pad;   // input column of slot 0 at xb = 0
+    const uint32_t *bptr = Bs + tn * TN;
 
     for (int ci0 = 0; ci0 < p.Ci; ci0 += p.CK) {
         const int ckn = min(p.CK, p.Ci - ci0);
         __syncthreads();                                             // previous chunk fully consumed (and s_row written)
-        // ---- stage the packed activation rows of ckn channels (Eq. 5, built from int8 codes)
-        for (int idx = tid; idx < ckn * words_per_plane; idx += kThreads2D) {
-            const int cl = idx / words_per_plane;
-            const int rem = idx - cl * words_per_plane;
-            const int rl = rem / p.XB, xb = rem - rl * p.XB;
+        // ---- stage the packed activation rows of ckn channels (Eq. 5, built from int8 codes): a warp per row
+        for (int r = warp; r < ckn * NR; r += nwarps) {
+            const int cl = r / NR, rl = r - cl * NR;
             const int base = s_row[rl];
-            uint32_t word = 0;
-            if (base >= 0) {
+            uint32_t *dst = As + cl * p.a_plane + p.lead + rl * p.XB;
+            if (base < 0) {
+                for (int xb = lane; xb < p.XB; xb += 32) dst[xb] = 0;
+            } else {
                 const int8_t *src = p.x + base + (ci0 + cl) * HW;
-                const int col0 = col_seg0 + xb * N;
+                for (int xb = lane; xb < p.XB; xb += 32) {
+                    const int col0 = col_seg0 + xb * N;
+                    uint32_t word = 0;
+                    if (col0 >= 0 && col0 + N <= p.W) {
 #pragma unroll
-                for (int n = 0; n < N; ++n) {
-                    const int col = col0 + n;
-                    if (col >= 0 && col < p.W) word += (uint32_t)load_code<XS>(src + col) * slot_pow[n];
+                        for (int n = 0; n < N; ++n) {
+                            const uint32_t c = (uint32_t)load_code<XS>(src + col0 + n);
+                            word = (n == 0) ? c : word + c * slot_pow[n];
+                        }
+                    } else {
+#pragma unroll
+                        for (int n = 0; n < N; ++n) {
+                            const int col = col0 + n;
+                            if (col >= 0 && col < p.W) word += (uint32_t)load_code<XS>(src + col) * slot_pow[n];
+                        }
+                    }
+                    dst[xb] = word;
                 }
             }
-            As[cl * p.a_plane + p.lead + rem] = word;
         }
         // ---- stage the packed kernel rows of the same channels for TCO output channels
         {
             const int tco4 = p.TCO / 4;
             const int rows = ckn * KJ;
-            for (int idx = tid; idx < rows * tco4; idx += kThreads2D) {
+            for (int idx = tid; idx < rows * tco4; idx += nthreads) {
                 const int kr = idx / tco4, c4 = idx - kr * tco4;
                 const int co = co0 + c4 * 4;
                 uint4 v = make_uint4(0, 0, 0, 0);
@@ -189,51 +222,76 @@ __global__ void __launch_bounds__(kThreads2D) conv2d_kernel(const Conv2dParams p
         }
         __syncthreads();
         // ---- multiply-accumulate over (ci, kh, j)
-        for (int cl = 0; cl < ckn; ++cl) {
-            for (int kh = 0; kh < p.K; ++kh) {
-                for (int j = 0; j < p.J; ++j) {
-                    const uint32_t *arow = As + cl * p.a_plane + kh * p.XB - j;
-                    const uint32_t *brow = Bs + ((cl * p.K + kh) * p.J + j) * p.TCO + tn * TN;
-                    uint32_t a[TM], b[TN];
+        if constexpr (KT > 0) {
+            for (int cl = 0; cl < ckn; ++cl) {
+                const int abase = cl * p.a_plane;
+                const int bbase = cl * (KT * JT) * p.TCO;
 #pragma unroll
-                    for (int i = 0; i < TM; ++i) a[i] = arow[off[i]];
+                for (int kh = 0; kh < KT; ++kh) {
 #pragma unroll
-                    for (int t = 0; t < TN; t += 4) {
-                        const uint4 v = *reinterpret_cast<const uint4 *>(brow + t);
-                        b[t] = v.x; b[t + 1] = v.y; b[t + 2] = v.z; b[t + 3] = v.w;
-                    }
+                    for (int j = 0; j < JT; ++j) {
+                        const int aoff = abase + kh * p.XB - j;
+                        const uint32_t *brow = bptr + bbase + (kh * JT + j) * p.TCO;
+                        uint32_t a[TM], b[TN];
 #pragma unroll
-                    for (int i = 0; i < TM; ++i)
+                        for (int i = 0; i < TM; ++i) a[i] = aptr[i][aoff];
 #pragma unroll
-                        for (int t = 0; t < TN; ++t) {
-                            if (UNPACKED) acc[i][t] = (acc_t)((int32_t)acc[i][t] + (int32_t)a[i] * (int32_t)b[t]);
-                            else { uint64_t q = (uint64_t)acc[i][t]; mad_wide<SP>(q, a[i], b[t]); acc[i][t] = (acc_t)q; }
+                        for (int t = 0; t < TN; t += 4) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(brow + t);
+                            b[t] = v.x; b[t + 1] = v.y; b[t + 2] = v.z; b[t + 3] = v.w;
                         }
+#pragma unroll
+                        for (int i = 0; i < TM; ++i)
+#pragma unroll
+                            for (int t = 0; t < TN; ++t) mac<UNPACKED, SP>(acc[i][t], a[i], b[t]);
+                    }
                 }
-                if (!UNPACKED && ++cnt == p.M) { flush(); cnt = 0; }
+            }
+        } else {
+            for (int cl = 0; cl < ckn; ++cl) {
+                for (int kh = 0; kh < p.K; ++kh) {
+                    for (int j = 0; j < p.J; ++j) {
+                        const int aoff = cl * p.a_plane + kh * p.XB - j;
+                        const uint32_t *brow = bptr + ((cl * p.K + kh) * p.J + j) * p.TCO;
+                        uint32_t a[TM], b[TN];
+#pragma unroll
+                        for (int i = 0; i < TM; ++i) a[i] = aptr[i][aoff];
+#pragma unroll
+                        for (int t = 0; t < TN; t += 4) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(brow + t);
+                            b[t] = v.x; b[t + 1] = v.y; b[t + 2] = v.z; b[t + 3] = v.w;
+                        }
+#pragma unroll
+                        for (int i = 0; i < TM; ++i)
+#pragma unroll
+                            for (int t = 0; t < TN; ++t) mac<UNPACKED, SP>(acc[i][t], a[i], b[t]);
+                    }
+                }
             }
         }
+        // a chunk never holds more than M (ci, kh) pairs; split before the next one might not fit
+        if (!UNPACKED && ++chunks_since_flush == p.flush_chunks) { flush(); chunks_since_flush = 0; }
     }
-    if (!UNPACKED && cnt > 0) flush();
+    if (!UNPACKED && chunks_since_flush > 0) flush();
 
-    // ---- hand the slots that belong to the next thread's first position across (Theorem 2 at thread borders)
+    // ---- hand the last position's upper-slot windows to the next thread's first position
     if constexpr (!UNPACKED) {
         __syncthreads();
-        uint32_t *xch = smem;                              // [TMX][N][TCO]
+        uint32_t *xch = smem;                                        // [TMX][N][TCO]
 #pragma unroll
         for (int m = 0; m < N; ++m)
 #pragma unroll
-            for (int t = 0; t < TN; ++t) xch[(tm * N + m) * p.TCO + tn * TN + t] = carry[m][t];
+            for (int t = 0; t < TN; ++t) xch[(tm * N + m) * p.TCO + tn * TN + t] = C[m][t];
         __syncthreads();
         if (tm > 0) {
 #pragma unroll
             for (int m = 0; m < N; ++m)
 #pragma unroll
-                for (int t = 0; t < TN; ++t) outv[0][m][t] += xch[((tm - 1) * N + m) * p.TCO + tn * TN + t];
+                for (int t = 0; t < TN; ++t) V[0][m][t] += xch[((tm - 1) * N + m) * p.TCO + tn * TN + t];
         }
     }
 
-    // ---- bias removal, optional requantisation (arithmetic shift, clamp), store
+    // ---- separate the slots, remove the bias, optional requantisation (arithmetic shift, clamp), store
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
         const int pos = tm * TM + i;
@@ -249,13 +307,24 @@ __global__ void __launch_bounds__(kThreads2D) conv2d_kernel(const Conv2dParams p
             const int co = co0 + tn * TN + t;
             if (co >= p.Co) continue;
             const size_t row_off = (((size_t)b * p.Co + co) * p.Ho + h) * p.Wo;
+            uint32_t Y[N];
+            if constexpr (!UNPACKED) {
+#pragma unroll
+                for (int m = N - 1; m >= 0; --m) {
+                    uint32_t y = V[i][m][t];
+#pragma unroll
+                    for (int k = 1; k < N; ++k)
+                        if (m + k < N && S * k < 32) y -= Y[m + k < N ? m + k : 0] << (S * k);
+                    Y[m] = y;
+                }
+            }
 #pragma unroll
             for (int m = 0; m < N; ++m) {
                 const int w = xg * N + m;
                 if (w >= p.Wo) continue;
                 int32_t v;
-                if (UNPACKED) v = (int32_t)acc[i][t];
-                else v = (int32_t)(outv[UNPACKED ? 0 : i][UNPACKED ? 0 : m][UNPACKED ? 0 : t] - (uint32_t)nflush * (uint32_t)p.carry_bias[m]);
+                if constexpr (UNPACKED) v = (int32_t)acc[i][t];
+                else v = (int32_t)(Y[m] - (uint32_t)nflush * (uint32_t)p.carry_bias[m]);
                 if (p.requant) {
                     v >>= p.shift;
                     v = max(p.lo, min(p.hi, v));
@@ -320,9 +389,9 @@ __global__ void __launch_bounds__(256) maxpool2x2_kernel(const int8_t *__restric
 struct Conv2dSetup {
     hikonv_layout_t L;
     Conv2dParams kp;
-    int variant;          // index into the launch table
     size_t smem_bytes;
     dim3 grid;
+    int threads;
     bool unpacked;
 };
 
@@ -332,14 +401,14 @@ static int sm_count() {
     return sms;
 }
 
-template <int N, int TM, int TN, bool UNPACKED>
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT>
 static int launch_variant(const Conv2dSetup &s, bool sp, bool xs, cudaStream_t st) {
 #define HK_LAUNCH(SPV, XSV)                                                                                      \
     do {                                                                                                         \
-        auto kern = conv2d_kernel<N, TM, TN, UNPACKED, SPV, XSV>;                                                \
+        auto kern = conv2d_kernel<N, SC, TM, TN, UNPACKED, SPV, XSV, KT, JT>;                                    \
         if (s.smem_bytes > 48 * 1024)                                                                            \
             HIKONV_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem_bytes)); \
-        kern<<<s.grid, kThreads2D, s.smem_bytes, st>>>(s.kp);                                                    \
+        kern<<<s.grid, s.threads, s.smem_bytes, st>>>(s.kp);                                                     \
     } while (0)
     if (!sp) HK_LAUNCH(false, false);
     else if (xs) HK_LAUNCH(true, true);
@@ -350,6 +419,57 @@ static int launch_variant(const Conv2dSetup &s, bool sp, bool xs, cudaStream_t s
 
 constexpr int kTM = 4, kTN = 4;          // per-thread tile of the packed kernels
 constexpr int kTMU = 8, kTNU = 4;        // per-thread tile of the comparator
+
+// Tile shape of one candidate and its modelled cost.
+struct TileChoice {
+    int TNX, TMX, TR, NSEG, XO, XB;
+    double cost;
+};
+
+// Chooses channels per CTA (TNX * TN), rows per CTA (TR) and row segments so that the device is
+// evenly loaded.  The model charges each "wave" of resident CTAs max(resident threads, 256) per SM
+// (an SM with fewer threads than that cannot fill the multiply pipe), adds the staging work of a
+// tile relative to its multiply work, and divides by the useful work.
+static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int J, int Co, int TM, int TN, int sms,
+                               int force_tr) {
+    TileChoice best;
+    best.cost = -1.0;
+    for (int TNX = 1; TNX <= 16; TNX *= 2) {
+        const int TCO = TNX * TN;
+        if (TNX > 1 && TCO / 2 >= Co) break;                       // more channel lanes than channels
+        const int gy = ceil_div(Co, TCO);
+        const int max_tmx = kMaxThreads2D / TNX;
+        const int maxpos = max_tmx * TM;
+        int NSEG = 1;
+        while (ceil_div(X, NSEG) + J > maxpos) ++NSEG;
+        const int XO = ceil_div(X, NSEG), XB = XO + J;
+        const int tr_hi = std::max(1, std::min(maxpos / XB, total_rows));
+        const int tr_lo = force_tr > 0 ? std::min(force_tr, tr_hi) : 1;
+        const int tr_end = force_tr > 0 ? tr_lo : tr_hi;
+        for (int TR = tr_lo; TR <= tr_end; ++TR) {
+            int TMX = ceil_div(TR * XB, TM);
+            int threads = (TMX * TNX + 31) / 32 * 32;               // whole warps
+            if (threads > kMaxThreads2D) continue;
+            TMX = threads / TNX;
+            const long long tiles = (long long)ceil_div(total_rows, TR) * NSEG * gy;
+            const int per_sm = std::max(1, std::min(2048 / threads, 65536 / (threads * 128)));
+            const long long slots = (long long)per_sm * sms;
+            const long long full_waves = tiles / slots;
+            const long long rest = tiles - full_waves * slots;
+            double time = (double)full_waves * std::max(per_sm * threads, 256);
+            if (rest > 0) time += std::max((int)((rest + sms - 1) / sms) * threads, 256);
+            const int span = (TR + Ho - 2) / Ho + 1;
+            const double NR = TR + (K - 1) * span;
+            const double work = (double)K * J * (TM * TN + 8) * threads;
+            const double stage = NR * XB * (4.0 * N + 10.0) + (double)K * J * TCO;
+            time *= 1.0 + stage / work;
+            const double useful = (double)total_rows * X * Co;     // output blocks x channels
+            const double cost = time * sms / useful;
+            if (best.cost < 0 || cost < best.cost - 1e-12) best = {TNX, TMX, TR, NSEG, XO, XB, cost};
+        }
+    }
+    return best;
+}
 
 static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, int pad, int p, int q, int xs, int ws,
                       int requant, int shift, int lo, int hi, int algo, const hikonv_tuning_t *tune, Conv2dSetup *s) {
@@ -382,38 +502,32 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         if (L.N > kMaxN2D || L.segments > kMaxN2DSeg) return HIKONV_ERR_UNSUPPORTED;
         TM = kTM; TN = kTN; N = L.N;
         const SplitConsts sc = make_split_consts(L, p, q, xs, ws, K, L.M);
-        kp.mask = sc.slot_mask;
         kp.bias = sc.bias;
-        for (int m = 0; m < kMaxN2DSeg; ++m) kp.seg_shift[m] = m < L.segments ? L.S * m : 0;
         for (int m = 0; m < kMaxN2D; ++m) kp.carry_bias[m] = m < L.N ? sc.carry_bias[m] : 0;
     }
     kp.B = B; kp.Ci = Ci; kp.H = H; kp.W = W; kp.Co = Co; kp.K = K; kp.pad = pad; kp.Ho = Ho; kp.Wo = Wo; kp.Hp = Ho + K - 1;
     kp.CoP = (Co + 3) / 4 * 4;
-    kp.S = L.S; kp.J = L.J; kp.Kc = L.Kc; kp.nhi = L.segments - L.N; kp.M = L.M;
+    kp.S = L.S; kp.J = L.J; kp.Kc = L.Kc; kp.M = L.M;
     kp.requant = requant ? 1 : 0; kp.shift = shift; kp.lo = lo; kp.hi = hi;
     kp.total_rows = B * Ho;
     kp.X = ceil_div(Wo, N);
-    // channels per CTA: up to 64, thread grid TMX x TNX = 256
-    int TNX = 1;
-    while (TNX * TN < Co && TNX * TN < 64) TNX *= 2;
-    kp.TNX = TNX; kp.TMX = kThreads2D / TNX; kp.TCO = TNX * TN;
-    const int maxpos = kp.TMX * TM;
-    // rows wider than a tile are cut into segments, each with its own J halo positions
-    kp.NSEG = 1;
-    while (ceil_div(kp.X, kp.NSEG) + L.J > maxpos) ++kp.NSEG;
-    kp.XO = ceil_div(kp.X, kp.NSEG);
-    kp.XB = kp.XO + L.J;
-    int TR = maxpos / kp.XB;
-    if (tune && tune->tile > 0 && tune->tile < TR) TR = tune->tile;
-    if (TR > kp.total_rows) TR = kp.total_rows;
-    kp.TR = TR;
-    const int span = (TR + Ho - 2) / Ho + 1;                 // images a tile can touch
-    kp.NRmax = TR + (K - 1) * span;
+    const TileChoice tc = choose_tiles(kp.total_rows, Ho, kp.X, N, K, L.J, Co, TM, TN, sm_count(), tune ? tune->tile : 0);
+    if (tc.cost < 0) return HIKONV_ERR_UNSUPPORTED;
+    kp.TNX = tc.TNX; kp.TMX = tc.TMX; kp.TCO = tc.TNX * TN;
+    kp.NSEG = tc.NSEG; kp.XO = tc.XO; kp.XB = tc.XB; kp.TR = tc.TR;
+    s->threads = tc.TMX * tc.TNX;
+    const int span = (kp.TR + Ho - 2) / Ho + 1;              // images a tile can touch
+    kp.NRmax = kp.TR + (K - 1) * span;
     kp.lead = L.J;                                           // room for the xb - j reads at the front
     kp.a_plane = kp.NRmax * kp.XB + kp.lead;
-    // channels per stage: a multiple of the split period when that is short, about 8 otherwise
+    // channels per stage: a chunk holds at most M (ci, kh) pairs so that splits fall on chunk borders
     int CK = 8;
-    if (!s->unpacked && L.M < Ci * K) CK = std::max(1, std::min(8, L.M / K));
+    kp.flush_chunks = 1 << 30;
+    if (!s->unpacked && L.M < Ci * K) {
+        if (L.M < K) return HIKONV_ERR_NO_FIT;               // not even one channel's kernel rows between two splits
+        CK = std::max(1, std::min(8, L.M / K));
+        kp.flush_chunks = std::max(1, L.M / (CK * K));
+    }
     if (CK > Ci) CK = Ci;
     kp.CK = CK;
     kp.b_off = (CK * kp.a_plane + 3) / 4 * 4;
@@ -421,7 +535,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
     s->smem_bytes = std::max(words + (size_t)kp.NRmax, xch_words) * 4 + 16;
     if (s->smem_bytes > 200 * 1024) return HIKONV_ERR_UNSUPPORTED;
-    const long long row_tiles = ((long long)kp.total_rows + TR - 1) / TR;
+    const long long row_tiles = ((long long)kp.total_rows + kp.TR - 1) / kp.TR;
     const long long gx = row_tiles * kp.NSEG;
     const int gy = ceil_div(Co, kp.TCO);
     if (gx > 0x7FFFFFFFLL || gy > 65535) return HIKONV_ERR_UNSUPPORTED;
@@ -431,12 +545,22 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
 
 static int launch_conv2d(const Conv2dSetup &s, bool xs, cudaStream_t st) {
     const bool sp = s.L.signed_prod != 0;
-    if (s.unpacked) return launch_variant<1, kTMU, kTNU, true>(s, sp, xs, st);
+    const int K = s.kp.K, J = s.L.J;
+    if (s.unpacked) {
+        if (K == 3) return launch_variant<1, 0, kTMU, kTNU, true, 3, 3>(s, sp, xs, st);
+        if (K == 1) return launch_variant<1, 0, kTMU, kTNU, true, 1, 1>(s, sp, xs, st);
+        return launch_variant<1, 0, kTMU, kTNU, true, 0, 0>(s, sp, xs, st);
+    }
+    // the layouts of 3x3 and 1x1 layers with the slot width and loop bounds as compile-time constants
+    if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1>(s, sp, xs, st);
+    if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, xs, st);
+    if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, xs, st);
+    if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, xs, st);
     switch (s.L.N) {
-        case 1: return launch_variant<1, kTM, kTN, false>(s, sp, xs, st);
-        case 2: return launch_variant<2, kTM, kTN, false>(s, sp, xs, st);
-        case 3: return launch_variant<3, kTM, kTN, false>(s, sp, xs, st);
-        case 4: return launch_variant<4, kTM, kTN, false>(s, sp, xs, st);
+        case 1: return launch_variant<1, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
+        case 2: return launch_variant<2, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
+        case 3: return launch_variant<3, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
+        case 4: return launch_variant<4, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
         default: return HIKONV_ERR_UNSUPPORTED;
     }
 }

@@ -177,7 +177,7 @@ int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, 
             // row into several chunks: score every feasible (N, S)
             for (int S = forceS ? forceS : 31; S >= (forceS ? forceS : 1); --S) {
                 hikonv_layout_t c;
-                if (!check_candidate(p, q, fs, gs, K, N, S, false, total_terms, &c)) continue;
+                if (!check_candidate(p, q, fs, gs, K, N, S, true, total_terms, &c)) continue;
                 const double blocks = (double)(ceil_div(wo, N) + c.J);   // words per output row, halo included
                 const double per_mul = cm.mul_cycles + cm.split_cycles_per_seg * c.segments / (double)c.M;
                 const double cost = blocks * c.J * per_mul / (double)wo; // cycles per output pixel and (ci, kh)
