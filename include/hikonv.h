@@ -74,6 +74,8 @@ typedef struct {
     int M;           /* products that may be summed in the 64-bit accumulator before a split  */
     int signed_prod; /* 1 when either operand is signed (signed multiply, biased split)       */
     int S_paper;     /* Eq. 6 with the mode's guard bits, for reference                       */
+    int carry_bits;  /* 2-D: every M products the slot bits above this many low bits move to a
+                        second packed accumulator (0: never, M covers the whole layer; 1-D: 0)   */
 } hikonv_layout_t;
 
 /* Optional overrides for experiments and tests; zero in a field means "choose automatically".

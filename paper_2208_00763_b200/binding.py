@@ -31,7 +31,7 @@ class PlanT(ctypes.Structure):
 
 
 class LayoutT(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("N", "S", "Kc", "J", "segments", "top_bits", "M", "signed_prod", "S_paper")]
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "S", "Kc", "J", "segments", "top_bits", "M", "signed_prod", "S_paper", "carry_bits")]
 
 
 class TuningT(ctypes.Structure):

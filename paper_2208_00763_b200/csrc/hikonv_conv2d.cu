@@ -14,14 +14,15 @@
 // is a register-tiled integer "GEMM" over packed words: each thread owns TM consecutive positions
 // times TN channels, the k dimension runs over (ci, kh, j).
 //
-// Split.  After at most M accumulated (ci, kh) pairs the accumulators are "flushed": the upper
-// slots of position i-1 are added to position i (Theorem 2 on the products, as in Section V-A), the
-// N low slots are kept, and for every m < N the 32-bit window (D >> S m) is added to an int32 sum
-//     V[m] = Y[m] + 2^S Y[m+1] + 2^(2S) Y[m+2] + ...   (mod 2^32)
-// where Y[m] is the running sum of slot m.  Nothing is masked per flush; the slots are separated
-// once at the end by back-substitution (Y[N-1] = V[N-1], Y[m] = V[m] - sum_k 2^(S k) Y[m+k]), which
-// is exact because every Y fits 32 bits.  This is Algorithm 2's shift-and-mask split with the mask
-// postponed; slots are biased (non-negative) instead of sign-corrected (Eq. 29).
+// Split.  Every slot starts at a bias that makes its running sum non-negative, so slots never borrow
+// from each other (this replaces the sign-borrow increment of Eq. 29).  After at most M accumulated
+// (ci, kh) pairs a slot would overflow; instead of splitting all slots into int32 sums there (the
+// shift-and-mask of Algorithm 2, N + K - 1 extractions per accumulator), the kernel moves the bits of
+// every slot above its low h bits into a SECOND packed accumulator with the same slot layout,
+//     E += (Q >> h) & mask_high;      Q = (Q & mask_low) | bias;
+// eight logic/shift/add instructions per accumulator whatever N is.  E can take 2^h such moves.  The
+// slots are extracted once, at the end: slot m holds 2^h E_m + Q_m - (moves + 1) bias_m, the low N
+// slots belong to this block and the upper ones are added to the next block of the row (Theorem 2).
 #include <algorithm>
 #include <cstring>
 #include <mutex>
@@ -47,8 +48,10 @@ struct Conv2dParams {
     int requant, shift, lo, hi;
     int total_rows;            // B * Ho
     int flush_chunks;          // channel chunks accumulated between two splits (CK * K * flush_chunks <= M)
-    uint64_t bias;
-    int32_t carry_bias[kMaxN2D];
+    int hbits, nslots;         // carry-save: low bits kept per slot; number of slots N + Kc - 1
+    uint64_t bias, mask_low, mask_high;
+    uint32_t slot_mask, top_mask;
+    int32_t slot_bias[kMaxN2DSeg];
 };
 
 template <bool UNPACKED>
@@ -123,9 +126,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
 
     acc_t acc[TM][TN];
-    // running window sums and the last position's upper-slot windows; uint32 arithmetic wraps by design
-    uint32_t V[UNPACKED ? 1 : TM][UNPACKED ? 1 : N][UNPACKED ? 1 : TN];
-    uint32_t C[UNPACKED ? 1 : N][UNPACKED ? 1 : TN];
+    acc_t E[UNPACKED ? 1 : TM][UNPACKED ? 1 : TN];     // second packed accumulator (upper slot bits)
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
@@ -134,37 +135,24 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
         for (int i = 0; i < TM; ++i)
 #pragma unroll
-            for (int m = 0; m < N; ++m)
-#pragma unroll
-                for (int t = 0; t < TN; ++t) V[i][m][t] = 0;
-#pragma unroll
-        for (int m = 0; m < N; ++m)
-#pragma unroll
-            for (int t = 0; t < TN; ++t) C[m][t] = 0;
+            for (int t = 0; t < TN; ++t) E[i][t] = 0;
     }
-    int nflush = 0, chunks_since_flush = 0;
+    int nmoves = 0, chunks_since_move = 0;
 
-    auto flush = [&]() {
+    // move the upper bits of every slot to E and restart the slots at their bias
+    auto carry_save = [&]() {
         if constexpr (!UNPACKED) {
-            const int SN = S * N;
-            const uint64_t low_mask = (1ull << SN) - 1ull;
+            const uint64_t mask_high = p.mask_high, mask_low = p.mask_low, bias = p.bias;
+            const int h = p.hbits;
 #pragma unroll
-            for (int t = 0; t < TN; ++t) {
-                uint32_t upper = 0;                          // slots N.. of the previous position (fits 32 bits)
+            for (int i = 0; i < TM; ++i)
 #pragma unroll
-                for (int i = 0; i < TM; ++i) {
+                for (int t = 0; t < TN; ++t) {
                     const uint64_t Q = (uint64_t)acc[i][t];
-                    uint64_t D = (i == 0) ? Q : Q + (uint64_t)upper;      // Theorem 2: carry of the block before
-                    upper = (uint32_t)(Q >> SN);
-                    D &= low_mask;
-#pragma unroll
-                    for (int m = 0; m < N; ++m) V[i][m][t] += (uint32_t)(D >> (S * m));
-                    acc[i][t] = (acc_t)p.bias;
+                    E[i][t] += (Q >> h) & mask_high;
+                    acc[i][t] = (acc_t)((Q & mask_low) | bias);
                 }
-#pragma unroll
-                for (int m = 0; m < N; ++m) C[m][t] += upper >> (S * m);   // goes to the next thread's first position
-            }
-            ++nflush;
+            ++nmoves;
         }
     };
 
@@ -269,62 +257,66 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 }
             }
         }
-        // a chunk never holds more than M (ci, kh) pairs; split before the next one might not fit
-        if (!UNPACKED && ++chunks_since_flush == p.flush_chunks) { flush(); chunks_since_flush = 0; }
+        // at most M (ci, kh) pairs between two moves; none is needed after the last stage
+        if (!UNPACKED && ++chunks_since_move == p.flush_chunks && ci0 + p.CK < p.Ci) { carry_save(); chunks_since_move = 0; }
     }
-    if (!UNPACKED && chunks_since_flush > 0) flush();
 
-    // ---- hand the last position's upper-slot windows to the next thread's first position
+    // ---- extract the slots: slot m holds 2^h E_m + Q_m - (moves + 1) bias_m (uint32 arithmetic wraps by design)
+    const uint32_t nb = (uint32_t)nmoves + 1u;
+    auto slot_value = [&](uint64_t Q, uint64_t Ev, int m) -> uint32_t {
+        const uint32_t msk = (m == p.nslots - 1) ? p.top_mask : p.slot_mask;
+        const uint32_t qv = (uint32_t)(Q >> (S * m)) & msk;
+        const uint32_t ev = (uint32_t)(Ev >> (S * m)) & msk;
+        return (ev << p.hbits) + qv - nb * (uint32_t)p.slot_bias[m];
+    };
+    // the upper slots of a thread's last position belong to the next thread's first position (Theorem 2)
     if constexpr (!UNPACKED) {
         __syncthreads();
         uint32_t *xch = smem;                                        // [TMX][N][TCO]
 #pragma unroll
         for (int m = 0; m < N; ++m)
 #pragma unroll
-            for (int t = 0; t < TN; ++t) xch[(tm * N + m) * p.TCO + tn * TN + t] = C[m][t];
+            for (int t = 0; t < TN; ++t)
+                xch[(tm * N + m) * p.TCO + tn * TN + t] =
+                    (N + m < p.nslots) ? slot_value((uint64_t)acc[TM - 1][t], (uint64_t)E[TM - 1][t], N + m) : 0u;
         __syncthreads();
-        if (tm > 0) {
-#pragma unroll
-            for (int m = 0; m < N; ++m)
-#pragma unroll
-                for (int t = 0; t < TN; ++t) V[0][m][t] += xch[((tm - 1) * N + m) * p.TCO + tn * TN + t];
-        }
     }
 
-    // ---- separate the slots, remove the bias, optional requantisation (arithmetic shift, clamp), store
+    // ---- overlap-add, optional requantisation (arithmetic shift, clamp), store
 #pragma unroll
-    for (int i = 0; i < TM; ++i) {
-        const int pos = tm * TM + i;
-        if (pos >= TP) continue;
-        const int r = pos / p.XB, xbl = pos - r * p.XB;
-        if (xbl < p.J) continue;                                     // halo positions produce no pixels
-        const int xg = seg * p.XO + xbl - p.J;                       // output block in the row
-        if (xg >= p.X) continue;
-        const int R = R0 + r;
-        const int b = R / p.Ho, h = R - b * p.Ho;
+    for (int t = 0; t < TN; ++t) {
+        const int co = co0 + tn * TN + t;
+        uint32_t upper[N];                                           // upper slots of the previous position
+        if constexpr (!UNPACKED) {
 #pragma unroll
-        for (int t = 0; t < TN; ++t) {
-            const int co = co0 + tn * TN + t;
-            if (co >= p.Co) continue;
-            const size_t row_off = (((size_t)b * p.Co + co) * p.Ho + h) * p.Wo;
+            for (int m = 0; m < N; ++m) upper[m] = (tm > 0) ? smem[((tm - 1) * N + m) * p.TCO + tn * TN + t] : 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < TM; ++i) {
             uint32_t Y[N];
             if constexpr (!UNPACKED) {
 #pragma unroll
-                for (int m = N - 1; m >= 0; --m) {
-                    uint32_t y = V[i][m][t];
+                for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], (uint64_t)E[i][t], m) + upper[m];
 #pragma unroll
-                    for (int k = 1; k < N; ++k)
-                        if (m + k < N && S * k < 32) y -= Y[m + k < N ? m + k : 0] << (S * k);
-                    Y[m] = y;
-                }
+                for (int m = 0; m < N; ++m)
+                    upper[m] = (N + m < p.nslots) ? slot_value((uint64_t)acc[i][t], (uint64_t)E[i][t], N + m) : 0u;
+            } else {
+                Y[0] = (uint32_t)acc[i][t];
             }
+            const int pos = tm * TM + i;
+            if (pos >= TP || co >= p.Co) continue;
+            const int r = pos / p.XB, xbl = pos - r * p.XB;
+            if (xbl < p.J) continue;                                 // halo positions produce no pixels
+            const int xg = seg * p.XO + xbl - p.J;                   // output block in the row
+            if (xg >= p.X) continue;
+            const int R = R0 + r;
+            const int b = R / p.Ho, h = R - b * p.Ho;
+            const size_t row_off = (((size_t)b * p.Co + co) * p.Ho + h) * p.Wo;
 #pragma unroll
             for (int m = 0; m < N; ++m) {
                 const int w = xg * N + m;
                 if (w >= p.Wo) continue;
-                int32_t v;
-                if constexpr (UNPACKED) v = (int32_t)acc[i][t];
-                else v = (int32_t)(Y[m] - (uint32_t)nflush * (uint32_t)p.carry_bias[m]);
+                int32_t v = (int32_t)Y[m];
                 if (p.requant) {
                     v >>= p.shift;
                     v = max(p.lo, min(p.hi, v));
@@ -502,8 +494,11 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         if (L.N > kMaxN2D || L.segments > kMaxN2DSeg) return HIKONV_ERR_UNSUPPORTED;
         TM = kTM; TN = kTN; N = L.N;
         const SplitConsts sc = make_split_consts(L, p, q, xs, ws, K, L.M);
-        kp.bias = sc.bias;
-        for (int m = 0; m < kMaxN2D; ++m) kp.carry_bias[m] = m < L.N ? sc.carry_bias[m] : 0;
+        kp.bias = sc.bias; kp.mask_low = sc.mask_low; kp.mask_high = sc.mask_high;
+        kp.hbits = L.carry_bits; kp.nslots = L.segments;
+        kp.slot_mask = sc.slot_mask;
+        kp.top_mask = (L.top_bits >= 32) ? 0xFFFFFFFFu : ((1u << L.top_bits) - 1u);
+        for (int m = 0; m < kMaxN2DSeg; ++m) kp.slot_bias[m] = m < L.segments ? sc.seg_bias[m] : 0;
     }
     kp.B = B; kp.Ci = Ci; kp.H = H; kp.W = W; kp.Co = Co; kp.K = K; kp.pad = pad; kp.Ho = Ho; kp.Wo = Wo; kp.Hp = Ho + K - 1;
     kp.CoP = (Co + 3) / 4 * 4;
@@ -520,15 +515,16 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.NRmax = kp.TR + (K - 1) * span;
     kp.lead = L.J;                                           // room for the xb - j reads at the front
     kp.a_plane = kp.NRmax * kp.XB + kp.lead;
-    // channels per stage: a chunk holds at most M (ci, kh) pairs so that splits fall on chunk borders
-    int CK = 8;
+    // channels per stage and stages between two carry-save moves (at most M (ci, kh) pairs)
+    int CK = std::min(8, Ci);
     kp.flush_chunks = 1 << 30;
     if (!s->unpacked && L.M < Ci * K) {
-        if (L.M < K) return HIKONV_ERR_NO_FIT;               // not even one channel's kernel rows between two splits
-        CK = std::max(1, std::min(8, L.M / K));
-        kp.flush_chunks = std::max(1, L.M / (CK * K));
+        if (L.M < K) return HIKONV_ERR_NO_FIT;               // not even one channel's kernel rows between two moves
+        int fc = 1;
+        const int eff = pick_chunking(L.M / K, Ci, &CK, &fc);
+        if (ceil_div(Ci, eff) > (1 << L.carry_bits)) return HIKONV_ERR_NO_FIT;
+        kp.flush_chunks = fc;
     }
-    if (CK > Ci) CK = Ci;
     kp.CK = CK;
     kp.b_off = (CK * kp.a_plane + 3) / 4 * 4;
     size_t words = (size_t)kp.b_off + (size_t)CK * K * L.J * kp.TCO;

@@ -22,12 +22,14 @@ struct SplitConsts {
     int32_t seg_bias[kMaxSegments];     // per product slot
     int32_t carry_bias[kMaxSegments];   // slot m of (product + carry of the previous block), m < N
     uint32_t slot_mask;                 // 2^S - 1
+    uint64_t mask_low;                  // the low h bits of every slot (h = carry_bits)
+    uint64_t mask_high;                 // the remaining bits of every slot, moved down by h
 };
 
 // Cost-model constants for the 2-D planner, in scheduler cycles per warp instruction.
 struct CostModel {
-    double mul_cycles = 2.0;        // one 32x32->64 multiply-accumulate
-    double split_cycles_per_seg = 5.0;
+    double mul_cycles = 4.0;        // one 32x32->64 multiply-accumulate (half the rate of a 32-bit one)
+    double carry_save_cycles = 10.0; // moving the upper slot bits to the second accumulator, per accumulator
 };
 
 int validate_codes(int p, int q);
@@ -38,6 +40,31 @@ int make_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int t
 SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int f_signed, int g_signed, int K, int M);
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// 2-D kernels stage CK input channels at a time and move the upper slot bits to the second
+// accumulator every `fc` stages.  Given the number of channels CF that may be accumulated between two
+// such moves, picks CK <= 8 and fc with CK * fc <= CF as large as possible (stages of fewer than
+// three channels are avoided when something close is available).  Returns CK * fc.
+inline int pick_chunking(int CF, int Ci, int *CK, int *fc) {
+    if (CF >= Ci) {
+        *CK = Ci < 8 ? Ci : 8;
+        *fc = 1 << 30;
+        return Ci;
+    }
+    int best = 0;
+    double best_score = -1.0;
+    for (int ck = (CF < 8 ? CF : 8); ck >= 1; --ck) {
+        const int f = CF / ck, eff = ck * f;
+        const double score = ck >= 3 ? eff : 0.7 * eff;
+        if (score > best_score) {
+            best_score = score;
+            best = eff;
+            *CK = ck;
+            *fc = f;
+        }
+    }
+    return best;
+}
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace hikonv

@@ -76,9 +76,13 @@ static bool slot_fits(i128 lo, i128 hi, int w) {
 }
 
 // Checks one candidate (N, S) and fills Kc, J, segments, top_bits and the largest M (capped).
-// `packed_overlap`: the carry of block x-1 is added to block x's product before the split.
+// `packed_overlap`: the carry of block x-1 is added to block x's product before the split (1-D).
+// `carry_save_total` > 0 selects the 2-D rule: after every M accumulated products the part of each
+// slot above its low h bits is moved to a second packed accumulator, so a slot must hold
+// (2^h - 1) + bias + M T pmax with the bias a multiple of 2^h, and the second accumulator must
+// survive ceil(total / M) such moves (at most 2^h of them).
 static bool check_candidate(int p, int q, int fs, int gs, int K, int N, int S, bool packed_overlap,
-                            long long M_cap, hikonv_layout_t *L) {
+                            long long M_cap, long long carry_save_total, long long force_M, hikonv_layout_t *L) {
     if (S < 1 || S > 31 || N < 1) return false;
     const bool sp = fs || gs;
     const Range fr = code_range(p, fs), gr = code_range(q, gs);
@@ -120,11 +124,50 @@ static bool check_candidate(int p, int q, int fs, int gs, int K, int N, int S, b
         }
         return true;
     };
-    if (!fits_with(1)) return false;
-    long long lo = 1, hi = std::max(1LL, M_cap);   // largest M in [1, M_cap] that fits (monotone)
-    while (lo < hi) {
-        const long long mid = (lo + hi + 1) / 2;
-        if (fits_with(mid)) lo = mid; else hi = mid - 1;
+    long long lo = 1;
+    int carry_bits = 0;
+    if (carry_save_total > 0) {
+        auto fits_cs = [&](long long M, int h) {
+            for (int m = 0; m < NS; ++m) {
+                const int w = (m == NS - 1) ? top_bits : S;
+                if (h >= w) return false;
+                const i128 unit = (i128)1 << h;
+                i128 bias = (i128)M * T[m] * (-pmin);
+                bias = (bias + unit - 1) / unit * unit;
+                const i128 low = (h > 0 && M < carry_save_total) ? unit - 1 : 0;
+                if (low + bias + (i128)M * T[m] * pmax > ((i128)1 << w) - 1) return false;
+            }
+            return true;
+        };
+        long long bestM = 0;
+        for (int h = 0; h < S; ++h) {
+            long long a = 1, b = force_M > 0 ? force_M : std::max(1LL, M_cap);
+            if (force_M > 0) a = force_M;
+            if (!fits_cs(a, h)) continue;
+            while (a < b) {
+                const long long mid = (a + b + 1) / 2;
+                if (fits_cs(mid, h)) a = mid; else b = mid - 1;
+            }
+            if (a < carry_save_total) {
+                // the kernel moves bits at channel-stage borders: whole channels, in the staging it can realise
+                const int Ci = (int)(carry_save_total / K);
+                if (a < K) continue;
+                int ck, fc;
+                const int eff = pick_chunking((int)(a / K), Ci, &ck, &fc);
+                if (ceil_div(Ci, eff) > (1LL << h)) continue;
+                a = (long long)eff * K;
+            }
+            if (a > bestM) { bestM = a; carry_bits = h; }
+        }
+        if (bestM < 1) return false;
+        lo = bestM;
+    } else {
+        if (!fits_with(1)) return false;
+        long long hi = std::max(1LL, M_cap);           // largest M in [1, M_cap] that fits (monotone)
+        while (lo < hi) {
+            const long long mid = (lo + hi + 1) / 2;
+            if (fits_with(mid)) lo = mid; else hi = mid - 1;
+        }
     }
     L->N = N;
     L->S = S;
@@ -134,6 +177,7 @@ static bool check_candidate(int p, int q, int fs, int gs, int K, int N, int S, b
     L->top_bits = top_bits;
     L->M = (int)lo;
     L->signed_prod = sp ? 1 : 0;
+    L->carry_bits = carry_bits;
     return true;
 }
 
@@ -156,7 +200,7 @@ int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, 
             double best_rate = 0.0;
             for (int N = forceN ? forceN : 1; N <= maxN; ++N) {
                 hikonv_layout_t c;
-                if (!check_candidate(p, q, fs, gs, K, N, S, true, 1, &c)) continue;
+                if (!check_candidate(p, q, fs, gs, K, N, S, true, 1, 0, 0, &c)) continue;
                 const double rate = (double)c.N / c.J;   // outputs per multiply
                 if (rate > best_rate + 1e-9) {
                     best_rate = rate;
@@ -177,9 +221,9 @@ int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, 
             // row into several chunks: score every feasible (N, S)
             for (int S = forceS ? forceS : 31; S >= (forceS ? forceS : 1); --S) {
                 hikonv_layout_t c;
-                if (!check_candidate(p, q, fs, gs, K, N, S, true, total_terms, &c)) continue;
+                if (!check_candidate(p, q, fs, gs, K, N, S, false, total_terms, total_terms, forceM, &c)) continue;
                 const double blocks = (double)(ceil_div(wo, N) + c.J);   // words per output row, halo included
-                const double per_mul = cm.mul_cycles + cm.split_cycles_per_seg * c.segments / (double)c.M;
+                const double per_mul = cm.mul_cycles + cm.carry_save_cycles / (double)c.M;
                 const double cost = blocks * c.J * per_mul / (double)wo; // cycles per output pixel and (ci, kh)
                 if (!found || cost <= best_cost + 1e-12) {      // ties: the narrower slot
                     best_cost = cost;
@@ -194,7 +238,7 @@ int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, 
         }
     }
     if (!found) return HIKONV_ERR_NO_FIT;
-    if (forceM) {
+    if (forceM && dims == 1) {
         if (forceM > best.M) return HIKONV_ERR_NO_FIT;
         best.M = forceM;
     }
@@ -221,10 +265,16 @@ SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int fs, in
     const long long pmin = *std::min_element(prods, prods + 4);
     int T[kMaxSegments];
     term_counts(L, K, T);
+    const int h = L.carry_bits;
+    const long long unit = 1LL << h;
     for (int m = 0; m < L.segments; ++m) {
-        const long long b = -(long long)M * T[m] * pmin;      // >= 0: lifts the most negative sum to 0
+        long long b = -(long long)M * T[m] * pmin;            // >= 0: lifts the most negative sum to 0
+        b = (b + unit - 1) / unit * unit;                     // a multiple of 2^h (2-D carry-save; h = 0 otherwise)
+        const int w = (m == L.segments - 1) ? L.top_bits : L.S;
         c.seg_bias[m] = (int32_t)b;
         c.bias += (uint64_t)b << (L.S * m);
+        c.mask_low += (uint64_t)(unit - 1) << (L.S * m);
+        c.mask_high += (uint64_t)((1LL << (w - h)) - 1) << (L.S * m);
     }
     for (int m = 0; m < L.N; ++m)
         c.carry_bias[m] = c.seg_bias[m] + (m + L.N < L.segments ? c.seg_bias[m + L.N] : 0);
