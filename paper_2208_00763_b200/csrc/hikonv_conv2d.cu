@@ -44,7 +44,11 @@ struct Conv2dParams {
     int NSEG, XO, XB;          // row segments, output blocks per segment, positions per segment (XO + J)
     int TR, TMX, TNX, TCO, CK;
     int NRmax, a_plane, lead;
-    int b_off;                 // word offset of the weight tile in shared memory (multiple of 4: 16-byte loads)
+    int b_off;                 // word offset of the two weight tiles in shared memory (multiple of 4: 16-byte loads)
+    int b_words;               // words per weight tile (CK * K * J * TCO)
+    int raw_off, RPW;          // word offset of the raw activation rows, and their pitch in words
+    int async_ok;              // x is 4-byte aligned: rows can be fetched with 4-byte asynchronous copies
+    int x_bytes;               // B * Ci * H * W
     int requant, shift, lo, hi;
     int total_rows;            // B * Ho
     int flush_chunks;          // channel chunks accumulated between two splits (CK * K * flush_chunks <= M)
@@ -86,8 +90,9 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     typedef typename AccType<UNPACKED>::type acc_t;
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t *As = smem;                                   // [CK][a_plane]
-    uint32_t *Bs = As + p.b_off;                           // [CK*K*J][TCO], 16-byte aligned
-    int *s_row = (int *)(Bs + p.CK * p.K * p.J * p.TCO);   // [NRmax] input offset of each staged row, -1 = zero row
+    uint32_t *Bs = As + p.b_off;                           // two tiles [CK*K*J][TCO], 16-byte aligned
+    uint32_t *raw = As + p.raw_off;                        // [CK][NR][RPW] input rows as fetched (bytes, 4-byte granules)
+    int *s_row = (int *)(raw + p.CK * p.NRmax * p.RPW);    // [NRmax] input offset of each staged row, -1 = zero row
 
     const int tid = threadIdx.x, nthreads = blockDim.x;
     const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
@@ -162,53 +167,99 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
     for (int n = 0; n < N; ++n) slot_pow[n] = UNPACKED ? 1u : (1u << (S * n));
     const int col_seg0 = (seg * p.XO - p.J) * N + p.K - 1 - p.pad;   // input column of slot 0 at xb = 0
-    const uint32_t *bptr = Bs + tn * TN;
+    const int c_lo = max(col_seg0, 0), c_hi = min(p.W, col_seg0 + p.XB * N);   // input columns this row segment reads
+    const unsigned long long xaddr = (unsigned long long)p.x;
 
-    for (int ci0 = 0; ci0 < p.Ci; ci0 += p.CK) {
-        const int ckn = min(p.CK, p.Ci - ci0);
-        __syncthreads();                                             // previous chunk fully consumed (and s_row written)
-        // ---- stage the packed activation rows of ckn channels (Eq. 5, built from int8 codes): a warp per row
-        for (int r = warp; r < ckn * NR; r += nwarps) {
-            const int cl = r / NR, rl = r - cl * NR;
-            const int base = s_row[rl];
-            uint32_t *dst = As + cl * p.a_plane + p.lead + rl * p.XB;
-            if (base < 0) {
-                for (int xb = lane; xb < p.XB; xb += 32) dst[xb] = 0;
-            } else {
-                const int8_t *src = p.x + base + (ci0 + cl) * HW;
+    // Asynchronous fetch of one stage: the input rows of ckn channels as they are (4-byte granules that
+    // cover the needed columns, whatever the row's alignment) and the packed kernel rows for TCO channels.
+    auto fetch = [&](int ci0, int ckn, uint32_t *Bdst) {
+        if (c_hi > c_lo) {
+            for (int cl = 0; cl < ckn; ++cl) {
+                for (int rl = warp; rl < NR; rl += nwarps) {
+                    const int base = s_row[rl];
+                    if (base < 0) continue;
+                    const int first = base + (ci0 + cl) * HW + c_lo;          // byte offset of the first needed code
+                    const int phase = (int)((xaddr + (unsigned long long)first) & 3ull);
+                    const int nwords = (phase + (c_hi - c_lo) + 3) >> 2;
+                    uint32_t *dst = raw + (cl * NR + rl) * p.RPW;
+                    if (p.async_ok) {
+                        const int8_t *src = p.x + (first - phase);
+                        for (int wd = lane; wd < nwords; wd += 32) {
+                            const int left = p.x_bytes - (first - phase + 4 * wd);  // bytes up to the end of the tensor
+                            cp_async_4(dst + wd, src + 4 * wd, left >= 4 ? 4 : left);
+                        }
+                    } else {
+                        for (int wd = lane; wd < nwords; wd += 32) {
+                            uint32_t v = 0;
+#pragma unroll
+                            for (int bb = 0; bb < 4; ++bb) {
+                                const int off = first - phase + 4 * wd + bb;
+                                if (off >= 0 && off < p.x_bytes) v |= (uint32_t)(uint8_t)__ldg(p.x + off) << (8 * bb);
+                            }
+                            dst[wd] = v;
+                        }
+                    }
+                }
+            }
+        }
+        const int tco4 = p.TCO / 4;
+        const int rows = ckn * KJ;
+        for (int idx = tid; idx < rows * tco4; idx += nthreads) {
+            const int kr = idx / tco4, c4 = idx - kr * tco4;
+            const int co = co0 + c4 * 4;
+            uint32_t *dst = Bdst + (kr * tco4 + c4) * 4;
+            if (co < p.CoP) cp_async_16(dst, p.wp + (size_t)(ci0 * KJ + kr) * p.CoP + co);
+            else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
+        }
+        cp_async_commit();
+    };
+
+    // Packs the fetched rows into A words (Eq. 5): a warp per row, a lane per word.
+    auto pack_rows = [&](int ci0, int ckn) {
+        for (int cl = 0; cl < ckn; ++cl) {
+            for (int rl = warp; rl < NR; rl += nwarps) {
+                const int base = s_row[rl];
+                uint32_t *dst = As + cl * p.a_plane + p.lead + rl * p.XB;
+                if (base < 0 || c_hi <= c_lo) {
+                    for (int xb = lane; xb < p.XB; xb += 32) dst[xb] = 0;
+                    continue;
+                }
+                const int first = base + (ci0 + cl) * HW + c_lo;
+                const int phase = (int)((xaddr + (unsigned long long)first) & 3ull);
+                const int8_t *rb = reinterpret_cast<const int8_t *>(raw + (cl * NR + rl) * p.RPW) + phase - c_lo;   // rb[col]
                 for (int xb = lane; xb < p.XB; xb += 32) {
                     const int col0 = col_seg0 + xb * N;
                     uint32_t word = 0;
-                    if (col0 >= 0 && col0 + N <= p.W) {
+                    if (col0 >= c_lo && col0 + N <= c_hi) {
 #pragma unroll
                         for (int n = 0; n < N; ++n) {
-                            const uint32_t c = (uint32_t)load_code<XS>(src + col0 + n);
+                            const uint32_t c = (uint32_t)code_value<XS>(rb[col0 + n]);
                             word = (n == 0) ? c : word + c * slot_pow[n];
                         }
                     } else {
 #pragma unroll
                         for (int n = 0; n < N; ++n) {
                             const int col = col0 + n;
-                            if (col >= 0 && col < p.W) word += (uint32_t)load_code<XS>(src + col) * slot_pow[n];
+                            if (col >= c_lo && col < c_hi) word += (uint32_t)code_value<XS>(rb[col]) * slot_pow[n];
                         }
                     }
                     dst[xb] = word;
                 }
             }
         }
-        // ---- stage the packed kernel rows of the same channels for TCO output channels
-        {
-            const int tco4 = p.TCO / 4;
-            const int rows = ckn * KJ;
-            for (int idx = tid; idx < rows * tco4; idx += nthreads) {
-                const int kr = idx / tco4, c4 = idx - kr * tco4;
-                const int co = co0 + c4 * 4;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (co < p.CoP) v = __ldg(reinterpret_cast<const uint4 *>(p.wp + (size_t)(ci0 * KJ + kr) * p.CoP + co));
-                reinterpret_cast<uint4 *>(Bs)[kr * tco4 + c4] = v;
-            }
-        }
-        __syncthreads();
+    };
+
+    __syncthreads();                                                 // s_row is written
+    fetch(0, min(p.CK, p.Ci), Bs);
+    int stage = 0;
+    for (int ci0 = 0; ci0 < p.Ci; ci0 += p.CK, stage ^= 1) {
+        const int ckn = min(p.CK, p.Ci - ci0);
+        cp_async_wait_all();
+        __syncthreads();                                             // this stage has landed; the previous one is fully consumed
+        pack_rows(ci0, ckn);
+        __syncthreads();                                             // A words ready; the raw rows may be overwritten
+        if (ci0 + p.CK < p.Ci) fetch(ci0 + p.CK, min(p.CK, p.Ci - ci0 - p.CK), Bs + (stage ^ 1) * p.b_words);
+        const uint32_t *bptr = Bs + stage * p.b_words + tn * TN;
         // ---- multiply-accumulate over (ci, kh, j)
         if constexpr (KT > 0) {
             for (int cl = 0; cl < ckn; ++cl) {
@@ -527,9 +578,13 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     }
     kp.CK = CK;
     kp.b_off = (CK * kp.a_plane + 3) / 4 * 4;
-    size_t words = (size_t)kp.b_off + (size_t)CK * K * L.J * kp.TCO;
+    kp.b_words = CK * K * L.J * kp.TCO;
+    kp.raw_off = kp.b_off + 2 * kp.b_words;
+    kp.RPW = (std::min(W, kp.XB * N) + 6) / 4 + 1;
+    kp.x_bytes = B * Ci * H * W;
+    size_t words = (size_t)kp.raw_off + (size_t)CK * kp.NRmax * kp.RPW + (size_t)kp.NRmax;
     size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
-    s->smem_bytes = std::max(words + (size_t)kp.NRmax, xch_words) * 4 + 16;
+    s->smem_bytes = std::max(words, xch_words) * 4 + 16;
     if (s->smem_bytes > 200 * 1024) return HIKONV_ERR_UNSUPPORTED;
     const long long row_tiles = ((long long)kp.total_rows + kp.TR - 1) / kp.TR;
     const long long gx = row_tiles * kp.NSEG;
@@ -585,6 +640,7 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
         return HIKONV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     s.kp.x = d_x;
+    s.kp.async_ok = ((uintptr_t)d_x % 4 == 0) ? 1 : 0;
     s.kp.wp = (const uint32_t *)d_workspace;
     s.kp.out = d_out;
     const int total = Ci * K * s.L.J * s.kp.CoP;

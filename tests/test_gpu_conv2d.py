@@ -81,6 +81,19 @@ def test_extreme_codes(algo):
 
 
 @pytest.mark.parametrize("algo", ALGOS)
+def test_unaligned_input_pointer(algo):
+    # an input that does not start on a 4-byte boundary takes the byte-wise row fetch
+    x, w = inputs.conv2d_case(2, 9, 7, 13, 8, 3, 4, 4, True, True, seed=91)
+    ref = direct.conv2d_nchw(x, w, 1)
+    flat = torch.zeros(x.size + 8, dtype=torch.int8, device="cuda")
+    for shift in (1, 2, 3):
+        flat[shift:shift + x.size] = dev(x).reshape(-1)
+        view = flat[shift:shift + x.size].view(2, 9, 7, 13)
+        assert view.data_ptr() % 4 == shift
+        assert_exact(hk.conv2d(view, dev(w), 1, 4, 4, True, True, algo=algo), ref, "offset %d" % shift)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
 def test_requantize(algo):
     x, w = inputs.conv2d_case(2, 32, 10, 12, 16, 3, 4, 4, True, True, seed=77)
     acc = direct.conv2d_nchw(x, w, 1)
