@@ -360,7 +360,8 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
         x, w = inputs.layer_case(shape)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         d_w = torch.from_numpy(inputs.to_storage(w)).to(dev)
-        ws = torch.empty(hk.conv2d_workspace_bytes(shape["Ci"], shape["Co"], shape["K"]), dtype=torch.uint8, device=dev)
+        ws = torch.empty(hk.conv2d_workspace_bytes(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"]),
+                         dtype=torch.uint8, device=dev)
         rq = (shape["shift"], shape["lo"], shape["hi"]) if shape["requant"] else None
         Ho = shape["H"] + 2 * shape["pad"] - shape["K"] + 1
         Wo = shape["W"] + 2 * shape["pad"] - shape["K"] + 1
@@ -372,7 +373,7 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
         def step():
             hk.conv2d(d_x, d_w, shape["pad"], shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], requant=rq,
                       algo=algo, workspace=ws, out=o)
-        launches_per_step = 2
+        launches_per_step = 3
         name = "%s: 2-D layer %dx%dx%dx%d -> %d channels, %dx%d, pad %d, p=%d q=%d" % (
             args.workload, shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["K"], shape["pad"],
             shape["p"], shape["q"])
@@ -393,7 +394,7 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
 
         def step():
             net.forward(d_x, algo=algo)
-        launches_per_step = 2 * 9 + 4
+        launches_per_step = 3 * 9 + 4
         name = "c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head" % x.shape[0]
         h2d = d_x.numel()
         d2h = x.shape[0] * 36 * H * W * 4
@@ -491,7 +492,8 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
         x, w = inputs.layer_case(shape)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         d_w = torch.from_numpy(inputs.to_storage(w)).to(dev)
-        ws = torch.empty(hk.conv2d_workspace_bytes(shape["Ci"], shape["Co"], shape["K"]), dtype=torch.uint8, device=dev)
+        ws = torch.empty(hk.conv2d_workspace_bytes(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"]),
+                         dtype=torch.uint8, device=dev)
         rq = (shape["shift"], shape["lo"], shape["hi"]) if shape["requant"] else None
         Ho = shape["H"] + 2 * shape["pad"] - shape["K"] + 1
         Wo = shape["W"] + 2 * shape["pad"] - shape["K"] + 1

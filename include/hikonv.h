@@ -155,9 +155,11 @@ int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, 
  *   requant != 0: d_out is int8, clamp(sum >> shift, lo, hi) with an arithmetic (floor) shift,
  *                 0 <= shift <= 31, -128 <= lo <= hi <= 255 (values above 127 are stored as the
  *                 byte of the unsigned code).
- * The packed path first writes the reversed, packed kernel rows (g = W[co][ci][kh][K-1:0], Theorem 3)
- * to d_workspace (hikonv_conv2d_workspace_bytes bytes, 256-byte aligned), then runs the layer; both
- * on `stream`.  The unpacked comparator uses the workspace for int32 copies of the weights.
+ * Three kernels run on `stream`: the reversed kernel rows (g = W[co][ci][kh][K-1:0], Theorem 3) and the
+ * activation rows are packed (Eq. 5) into d_workspace, then the layer kernel streams the packed words.
+ * d_workspace: hikonv_conv2d_workspace_bytes(...) bytes of device memory, 256-byte aligned; the call
+ * overwrites it and needs nothing from it afterwards.  The unpacked comparator uses the same workspace for
+ * int32 copies of the weights and codes.
  * stride must be 1 and 0 <= pad < K.
  */
 int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,
@@ -165,7 +167,8 @@ int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *
                   int requant, int shift, int lo, int hi, void *d_workspace, size_t workspace_bytes,
                   int algo, const hikonv_tuning_t *tune, void *stream);
 
-size_t hikonv_conv2d_workspace_bytes(int Ci, int Co, int K);
+/* Workspace needed by hikonv_conv2d for this layer shape (an upper bound over all layouts and both algorithms). */
+size_t hikonv_conv2d_workspace_bytes(int B, int Ci, int H, int W, int Co, int K, int pad);
 
 /*
  * hikonv_conv2d_static_scratch - hikonv_conv2d for callers that cannot provide device scratch.
@@ -174,12 +177,12 @@ size_t hikonv_conv2d_workspace_bytes(int Ci, int Co, int K);
  * Some callers cannot allocate device memory at the point where they run a layer: code that runs
  * inside a memory-capped serving process whose pool is owned by another component, plug-ins that are
  * handed input and output tensors only, and real-time loops where cudaMalloc (which synchronises the
- * device and can fail late) is forbidden after start-up.  For them the packed kernel rows go to a
- * fixed buffer of HIKONV_STATIC_SCRATCH_BYTES that lives inside the library image on every GPU that
+ * device and can fail late) is forbidden after start-up.  For them the packed kernel and activation rows
+ * go to a fixed buffer of HIKONV_STATIC_SCRATCH_BYTES that lives inside the library image on every GPU that
  * loads it, from load until the process exits.  Arguments are those of hikonv_conv2d without the
  * workspace pair; results are identical.
  *
- *   - Limit: hikonv_conv2d_workspace_bytes(Ci, Co, K) must not exceed HIKONV_STATIC_SCRATCH_BYTES,
+ *   - Limit: hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad) must not exceed HIKONV_STATIC_SCRATCH_BYTES,
  *     otherwise HIKONV_ERR_TOO_LARGE is returned and nothing is launched.
  *   - The function calls no cudaMalloc/cudaFree and no allocating library routine.
  *   - The first call on each device looks up the buffer's device address (once per device, with that

@@ -51,7 +51,7 @@ _SIGNATURES = {
     "hikonv_conv1d_host": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _i, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz, _i,
                            ctypes.POINTER(TuningT), _vp]),
-    "hikonv_conv2d_workspace_bytes": (_sz, [_i, _i, _i]),
+    "hikonv_conv2d_workspace_bytes": (_sz, [_i] * 7),
     "hikonv_conv2d_static_scratch": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i,
                                           ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d_host_workspace_bytes": (_sz, [_i] * 8),
@@ -162,8 +162,8 @@ def conv1d_host(h_f: torch.Tensor, h_g: torch.Tensor, p, q, f_signed, g_signed, 
                                     algo, _tune(tune), _stream(stream)), "hikonv_conv1d_host")
 
 
-def conv2d_workspace_bytes(Ci: int, Co: int, K: int) -> int:
-    return int(lib().hikonv_conv2d_workspace_bytes(Ci, Co, K))
+def conv2d_workspace_bytes(B: int, Ci: int, H: int, W: int, Co: int, K: int, pad: int) -> int:
+    return int(lib().hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad))
 
 
 def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_signed: bool, w_signed: bool,
@@ -176,7 +176,7 @@ def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_sig
         raise ValueError("weight shape does not match the input")
     Ho, Wo = H + 2 * pad - K + 1, W + 2 * pad - K + 1
     if workspace is None:
-        workspace = torch.empty(conv2d_workspace_bytes(Ci, Co, K), dtype=torch.uint8, device=d_x.device)
+        workspace = torch.empty(conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad), dtype=torch.uint8, device=d_x.device)
     if out is None:
         out = torch.empty((B, Co, max(Ho, 0), max(Wo, 0)), dtype=torch.int8 if requant else torch.int32, device=d_x.device)
     shift, lo, hi = requant if requant else (0, 0, 0)
@@ -190,11 +190,11 @@ def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_sig
 def conv2d_static_scratch(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_signed: bool, w_signed: bool,
                           out: torch.Tensor, requant: Optional[tuple] = None, algo: int = ALGO_PACKED32, tune=None,
                           stride: int = 1, stream=None) -> torch.Tensor:
-    """``conv2d`` without a workspace: the packed kernel rows go to the library's built-in device buffer.
+    """``conv2d`` without a workspace: the packed kernel and activation rows go to the library's built-in device buffer.
 
     For callers that may not allocate device memory when the layer runs (they own only the input and
     output tensors, or allocation is forbidden after start-up).  ``out`` must be preallocated by the
-    caller.  Layers whose packed weights exceed ``STATIC_SCRATCH_BYTES`` raise ``ERR_TOO_LARGE``; calls
+    caller.  Layers whose packed rows exceed ``STATIC_SCRATCH_BYTES`` raise ``ERR_TOO_LARGE``; calls
     that may overlap on the GPU must be ordered by the caller, since they share the buffer.
     """
     B, Ci, H, W = d_x.shape

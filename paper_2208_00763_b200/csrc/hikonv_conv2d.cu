@@ -10,6 +10,10 @@
 // kernel row (g = W[co][ci][kh][K-1:0], Theorem 3).  Slot m < N of Q holds partial sums of pixel
 // xN + m, slot m >= N those of pixel (x+1)N + (m-N): the overlap-add of Theorem 2.
 //
+// Activations are packed once per layer by pack_activations_kernel into Ap[ci][b*Hp + hp][xb] (zero padding
+// rows and halo words materialised), weights by pack_weights_kernel into Bw[(ci,kh,j)][co]; the layer
+// kernel streams both with 16-byte asynchronous copies into double-buffered shared memory.
+//
 // A CTA computes TR consecutive output rows (one row segment each) times TCO output channels; it
 // is a register-tiled integer "GEMM" over packed words: each thread owns TM consecutive positions
 // times TN channels, the k dimension runs over (ci, kh, j).
@@ -36,22 +40,23 @@ constexpr int kMaxN2DSeg = 8;      // N + Kc - 1 <= 2 N <= 8
 
 struct Conv2dParams {
     const int8_t *x;
+    const uint32_t *ap;        // packed activations [Ci][B*Hp][XBT]
     const uint32_t *wp;        // packed weights [Ci*K*J][CoP]
     void *out;
     int B, Ci, H, W, Co, CoP, K, pad, Ho, Wo, Hp;
     int S, J, Kc, M;
     int X;                     // output blocks per row
-    int NSEG, XO, XB;          // row segments, output blocks per segment, positions per segment (XO + J)
+    int XBT;                   // words per packed activation row (halo + blocks, rounded up so that every tile row can be read in 16-byte pieces)
+    int NSEG, XO, XB;          // row segments, output blocks per segment (a multiple of 4 when NSEG > 1), positions per segment (XO + J)
+    int XBS;                   // words per activation row in shared memory (XB rounded up to a multiple of 4)
     int TR, TMX, TNX, TCO, CK;
-    int NRmax, a_plane, lead;
-    int b_off;                 // word offset of the two weight tiles in shared memory (multiple of 4: 16-byte loads)
+    int NRmax, a_plane, lead;  // staged rows per channel; words per channel in shared memory; words before the first row
+    int a_words;               // words per activation tile (CK * a_plane)
+    int b_off;                 // word offset of the first weight tile in shared memory
     int b_words;               // words per weight tile (CK * K * J * TCO)
-    int raw_off, RPW;          // word offset of the raw activation rows, and their pitch in words
-    int async_ok;              // x is 4-byte aligned: rows can be fetched with 4-byte asynchronous copies
-    int x_bytes;               // B * Ci * H * W
     int requant, shift, lo, hi;
     int total_rows;            // B * Ho
-    int flush_chunks;          // channel chunks accumulated between two splits (CK * K * flush_chunks <= M)
+    int flush_chunks;          // channel stages accumulated between two carry-save moves (CK * K * flush_chunks <= M)
     int hbits, nslots;         // carry-save: low bits kept per slot; number of slots N + Kc - 1
     uint64_t bias, mask_low, mask_high;
     uint32_t slot_mask, top_mask;
@@ -89,13 +94,10 @@ template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, bool XS, int KT
 __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dParams p) {
     typedef typename AccType<UNPACKED>::type acc_t;
     extern __shared__ __align__(16) uint32_t smem[];
-    uint32_t *As = smem;                                   // [CK][a_plane]
-    uint32_t *Bs = As + p.b_off;                           // two tiles [CK*K*J][TCO], 16-byte aligned
-    uint32_t *raw = As + p.raw_off;                        // [CK][NR][RPW] input rows as fetched (bytes, 4-byte granules)
-    int *s_row = (int *)(raw + p.CK * p.NRmax * p.RPW);    // [NRmax] input offset of each staged row, -1 = zero row
+    uint32_t *As = smem;                                   // two tiles [CK][a_plane]
+    uint32_t *Bs = smem + p.b_off;                         // two tiles [CK*K*J][TCO]
 
     const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
     const int tn = tid % p.TNX, tm = tid / p.TNX;
     const int seg = blockIdx.x % p.NSEG;
     const int R0 = (blockIdx.x / p.NSEG) * p.TR;
@@ -109,12 +111,6 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     const int TP = TRe * p.XB;                              // positions of this tile
     const int S = SC > 0 ? SC : p.S;
 
-    for (int rl = tid; rl < NR; rl += nthreads) {
-        const int rp = Rp0 + rl;
-        const int b = rp / p.Hp, hi = rp - b * p.Hp - p.pad;
-        s_row[rl] = (b < p.B && hi >= 0 && hi < p.H) ? (b * p.Ci * p.H + hi) * p.W : -1;
-    }
-
     // this thread's positions: shared-memory address of the packed word for (ci = 0, kh = 0, j = 0)
     const uint32_t *aptr[TM];
 #pragma unroll
@@ -125,7 +121,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             const int r = pos / p.XB, xb = pos - r * p.XB;
             const int R = R0 + r;
             const int b = R / p.Ho;
-            off = p.lead + ((b * p.Hp + (R - b * p.Ho)) - Rp0) * p.XB + xb;
+            off = p.lead + ((b * p.Hp + (R - b * p.Ho)) - Rp0) * p.XBS + xb;
         }
         aptr[i] = As + off;
     }
@@ -161,45 +157,21 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         }
     };
 
-    const int HW = p.H * p.W;
     const int KJ = p.K * p.J;
-    uint32_t slot_pow[N];
-#pragma unroll
-    for (int n = 0; n < N; ++n) slot_pow[n] = UNPACKED ? 1u : (1u << (S * n));
-    const int col_seg0 = (seg * p.XO - p.J) * N + p.K - 1 - p.pad;   // input column of slot 0 at xb = 0
-    const int c_lo = max(col_seg0, 0), c_hi = min(p.W, col_seg0 + p.XB * N);   // input columns this row segment reads
-    const unsigned long long xaddr = (unsigned long long)p.x;
+    const int xq = p.XBS / 4;                                        // 16-byte pieces per activation row
+    const size_t ap_plane = (size_t)p.B * p.Hp * p.XBT;              // words per channel of Ap
+    const uint32_t *ap_tile = p.ap + (size_t)Rp0 * p.XBT + seg * p.XO;   // first word this tile reads (16-byte aligned)
 
-    // Asynchronous fetch of one stage: the input rows of ckn channels as they are (4-byte granules that
-    // cover the needed columns, whatever the row's alignment) and the packed kernel rows for TCO channels.
-    auto fetch = [&](int ci0, int ckn, uint32_t *Bdst) {
-        if (c_hi > c_lo) {
-            for (int cl = 0; cl < ckn; ++cl) {
-                for (int rl = warp; rl < NR; rl += nwarps) {
-                    const int base = s_row[rl];
-                    if (base < 0) continue;
-                    const int first = base + (ci0 + cl) * HW + c_lo;          // byte offset of the first needed code
-                    const int phase = (int)((xaddr + (unsigned long long)first) & 3ull);
-                    const int nwords = (phase + (c_hi - c_lo) + 3) >> 2;
-                    uint32_t *dst = raw + (cl * NR + rl) * p.RPW;
-                    if (p.async_ok) {
-                        const int8_t *src = p.x + (first - phase);
-                        for (int wd = lane; wd < nwords; wd += 32) {
-                            const int left = p.x_bytes - (first - phase + 4 * wd);  // bytes up to the end of the tensor
-                            cp_async_4(dst + wd, src + 4 * wd, left >= 4 ? 4 : left);
-                        }
-                    } else {
-                        for (int wd = lane; wd < nwords; wd += 32) {
-                            uint32_t v = 0;
-#pragma unroll
-                            for (int bb = 0; bb < 4; ++bb) {
-                                const int off = first - phase + 4 * wd + bb;
-                                if (off >= 0 && off < p.x_bytes) v |= (uint32_t)(uint8_t)__ldg(p.x + off) << (8 * bb);
-                            }
-                            dst[wd] = v;
-                        }
-                    }
-                }
+    // Asynchronous fetch of one stage: NR packed rows of ckn channels and the packed kernel rows of the
+    // same channels for TCO output channels, all in 16-byte pieces.
+    auto fetch = [&](int ci0, int ckn, uint32_t *Adst, uint32_t *Bdst) {
+        const int per_ch = NR * xq;
+        for (int cl = 0; cl < ckn; ++cl) {
+            const uint32_t *src = ap_tile + (size_t)(ci0 + cl) * ap_plane;
+            uint32_t *dst = Adst + cl * p.a_plane + p.lead;
+            for (int idx = tid; idx < per_ch; idx += nthreads) {
+                const int rl = idx / xq, qd = idx - rl * xq;
+                cp_async_16(dst + rl * p.XBS + 4 * qd, src + (size_t)rl * p.XBT + 4 * qd);
             }
         }
         const int tco4 = p.TCO / 4;
@@ -214,62 +186,26 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         cp_async_commit();
     };
 
-    // Packs the fetched rows into A words (Eq. 5): a warp per row, a lane per word.
-    auto pack_rows = [&](int ci0, int ckn) {
-        for (int cl = 0; cl < ckn; ++cl) {
-            for (int rl = warp; rl < NR; rl += nwarps) {
-                const int base = s_row[rl];
-                uint32_t *dst = As + cl * p.a_plane + p.lead + rl * p.XB;
-                if (base < 0 || c_hi <= c_lo) {
-                    for (int xb = lane; xb < p.XB; xb += 32) dst[xb] = 0;
-                    continue;
-                }
-                const int first = base + (ci0 + cl) * HW + c_lo;
-                const int phase = (int)((xaddr + (unsigned long long)first) & 3ull);
-                const int8_t *rb = reinterpret_cast<const int8_t *>(raw + (cl * NR + rl) * p.RPW) + phase - c_lo;   // rb[col]
-                for (int xb = lane; xb < p.XB; xb += 32) {
-                    const int col0 = col_seg0 + xb * N;
-                    uint32_t word = 0;
-                    if (col0 >= c_lo && col0 + N <= c_hi) {
-#pragma unroll
-                        for (int n = 0; n < N; ++n) {
-                            const uint32_t c = (uint32_t)code_value<XS>(rb[col0 + n]);
-                            word = (n == 0) ? c : word + c * slot_pow[n];
-                        }
-                    } else {
-#pragma unroll
-                        for (int n = 0; n < N; ++n) {
-                            const int col = col0 + n;
-                            if (col >= c_lo && col < c_hi) word += (uint32_t)code_value<XS>(rb[col]) * slot_pow[n];
-                        }
-                    }
-                    dst[xb] = word;
-                }
-            }
-        }
-    };
-
-    __syncthreads();                                                 // s_row is written
-    fetch(0, min(p.CK, p.Ci), Bs);
+    fetch(0, min(p.CK, p.Ci), As, Bs);
     int stage = 0;
     for (int ci0 = 0; ci0 < p.Ci; ci0 += p.CK, stage ^= 1) {
         const int ckn = min(p.CK, p.Ci - ci0);
         cp_async_wait_all();
         __syncthreads();                                             // this stage has landed; the previous one is fully consumed
-        pack_rows(ci0, ckn);
-        __syncthreads();                                             // A words ready; the raw rows may be overwritten
-        if (ci0 + p.CK < p.Ci) fetch(ci0 + p.CK, min(p.CK, p.Ci - ci0 - p.CK), Bs + (stage ^ 1) * p.b_words);
+        if (ci0 + p.CK < p.Ci)
+            fetch(ci0 + p.CK, min(p.CK, p.Ci - ci0 - p.CK), As + (stage ^ 1) * p.a_words, Bs + (stage ^ 1) * p.b_words);
+        const int astage = stage * p.a_words;
         const uint32_t *bptr = Bs + stage * p.b_words + tn * TN;
         // ---- multiply-accumulate over (ci, kh, j)
         if constexpr (KT > 0) {
             for (int cl = 0; cl < ckn; ++cl) {
-                const int abase = cl * p.a_plane;
+                const int abase = astage + cl * p.a_plane;
                 const int bbase = cl * (KT * JT) * p.TCO;
 #pragma unroll
                 for (int kh = 0; kh < KT; ++kh) {
 #pragma unroll
                     for (int j = 0; j < JT; ++j) {
-                        const int aoff = abase + kh * p.XB - j;
+                        const int aoff = abase + kh * p.XBS - j;
                         const uint32_t *brow = bptr + bbase + (kh * JT + j) * p.TCO;
                         uint32_t a[TM], b[TN];
 #pragma unroll
@@ -290,7 +226,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             for (int cl = 0; cl < ckn; ++cl) {
                 for (int kh = 0; kh < p.K; ++kh) {
                     for (int j = 0; j < p.J; ++j) {
-                        const int aoff = cl * p.a_plane + kh * p.XB - j;
+                        const int aoff = astage + cl * p.a_plane + kh * p.XBS - j;
                         const uint32_t *brow = bptr + ((cl * p.K + kh) * p.J + j) * p.TCO;
                         uint32_t a[TM], b[TN];
 #pragma unroll
@@ -380,6 +316,32 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
 }
 
+// Packed activation rows (Eq. 5): ap[(ci * B*Hp + b*Hp + hp) * XBT + xb] packs the N input pixels of block
+// x = xb - J of padded row hp, i.e. columns (xb - J) N + K - 1 - pad + n of input row hp - pad, zero where the
+// row or a column lies in the padding.  For the comparator S == 0 and N == 1: one int32 code per word.
+template <bool XS>
+__global__ void __launch_bounds__(256) pack_activations_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
+                                                               int pad, int K, int J, int N, int S, int XBT,
+                                                               uint32_t *__restrict__ ap, size_t total) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int xb = (int)(idx % XBT);
+    const size_t rest = idx / XBT;
+    const int rp = (int)(rest % ((size_t)B * Hp));
+    const int ci = (int)(rest / ((size_t)B * Hp));
+    const int b = rp / Hp, hi = rp - b * Hp - pad;
+    uint32_t word = 0;
+    if (hi >= 0 && hi < H) {
+        const int8_t *row = x + (((size_t)b * Ci + ci) * H + hi) * W;
+        const int col0 = (xb - J) * N + K - 1 - pad;
+        for (int n = 0; n < N; ++n) {
+            const int col = col0 + n;
+            if (col >= 0 && col < W) word += (uint32_t)load_code<XS>(row + col) << (S * n);
+        }
+    }
+    ap[idx] = word;
+}
+
 // Reversed, packed kernel rows (Theorem 3: g = W[co][ci][kh][K-1:0], then Eq. 5 per chunk of Kc taps).
 // wp[((ci*K + kh)*J + j)*CoP + co] = sum_{k' < Kc} g[j Kc + k'] 2^(S k').  For the comparator S == 0,
 // Kc == 1: one int32 weight per word.
@@ -433,6 +395,8 @@ struct Conv2dSetup {
     hikonv_layout_t L;
     Conv2dParams kp;
     size_t smem_bytes;
+    size_t wp_bytes;      // packed weights in the workspace (256-byte multiple), packed activations follow
+    size_t ap_words;      // packed activation words
     dim3 grid;
     int threads;
     bool unpacked;
@@ -483,9 +447,17 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
         const int gy = ceil_div(Co, TCO);
         const int max_tmx = kMaxThreads2D / TNX;
         const int maxpos = max_tmx * TM;
-        int NSEG = 1;
-        while (ceil_div(X, NSEG) + J > maxpos) ++NSEG;
-        const int XO = ceil_div(X, NSEG), XB = XO + J;
+        // rows wider than a tile are cut into segments of XO blocks (a multiple of 4, so that every tile
+        // row starts on a 16-byte boundary of the packed activations), each with its own J halo positions
+        int NSEG = 1, XO = X;
+        if (X + J > maxpos) {
+            XO = (maxpos - J) / 4 * 4;
+            if (XO < 4) continue;
+            NSEG = ceil_div(X, XO);
+            XO = (ceil_div(X, NSEG) + 3) / 4 * 4;
+            NSEG = ceil_div(X, XO);
+        }
+        const int XB = XO + J;
         const int tr_hi = std::max(1, std::min(maxpos / XB, total_rows));
         const int tr_lo = force_tr > 0 ? std::min(force_tr, tr_hi) : 1;
         const int tr_end = force_tr > 0 ? tr_lo : tr_hi;
@@ -504,7 +476,7 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
             const int span = (TR + Ho - 2) / Ho + 1;
             const double NR = TR + (K - 1) * span;
             const double work = (double)K * J * (TM * TN + 8) * threads;
-            const double stage = NR * XB * (4.0 * N + 10.0) + (double)K * J * TCO;
+            const double stage = 0.5 * NR * XB + 0.5 * K * J * TCO;   // a few instructions per 16-byte piece
             time *= 1.0 + stage / work;
             const double useful = (double)total_rows * X * Co;     // output blocks x channels
             const double cost = time * sms / useful;
@@ -564,8 +536,10 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     s->threads = tc.TMX * tc.TNX;
     const int span = (kp.TR + Ho - 2) / Ho + 1;              // images a tile can touch
     kp.NRmax = kp.TR + (K - 1) * span;
-    kp.lead = L.J;                                           // room for the xb - j reads at the front
-    kp.a_plane = kp.NRmax * kp.XB + kp.lead;
+    kp.XBS = (kp.XB + 3) / 4 * 4;
+    kp.XBT = (kp.NSEG - 1) * kp.XO + kp.XBS;
+    kp.lead = (L.J + 3) / 4 * 4;                             // room for the xb - j reads in front of the first row
+    kp.a_plane = kp.NRmax * kp.XBS + kp.lead;
     // channels per stage and stages between two carry-save moves (at most M (ci, kh) pairs)
     int CK = std::min(8, Ci);
     kp.flush_chunks = 1 << 30;
@@ -577,14 +551,14 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         kp.flush_chunks = fc;
     }
     kp.CK = CK;
-    kp.b_off = (CK * kp.a_plane + 3) / 4 * 4;
+    kp.a_words = CK * kp.a_plane;
+    kp.b_off = 2 * kp.a_words;
     kp.b_words = CK * K * L.J * kp.TCO;
-    kp.raw_off = kp.b_off + 2 * kp.b_words;
-    kp.RPW = (std::min(W, kp.XB * N) + 6) / 4 + 1;
-    kp.x_bytes = B * Ci * H * W;
-    size_t words = (size_t)kp.raw_off + (size_t)CK * kp.NRmax * kp.RPW + (size_t)kp.NRmax;
-    size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
+    const size_t words = (size_t)kp.b_off + 2 * (size_t)kp.b_words;
+    const size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
     s->smem_bytes = std::max(words, xch_words) * 4 + 16;
+    s->wp_bytes = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
+    s->ap_words = (size_t)Ci * B * kp.Hp * kp.XBT;
     if (s->smem_bytes > 200 * 1024) return HIKONV_ERR_UNSUPPORTED;
     const long long row_tiles = ((long long)kp.total_rows + kp.TR - 1) / kp.TR;
     const long long gx = row_tiles * kp.NSEG;
@@ -620,10 +594,17 @@ static int launch_conv2d(const Conv2dSetup &s, bool xs, cudaStream_t st) {
 
 using namespace hikonv;
 
-extern "C" size_t hikonv_conv2d_workspace_bytes(int Ci, int Co, int K) {
-    if (Ci < 1 || Co < 1 || K < 1) return 0;
-    // at most K words per (ci, kh) row (one tap per word in the comparator), Co rounded up to 4
-    return align_up((size_t)Ci * K * K * ((Co + 3) / 4 * 4) * sizeof(uint32_t), 256);
+extern "C" size_t hikonv_conv2d_workspace_bytes(int B, int Ci, int H, int W, int Co, int K, int pad) {
+    if (B < 1 || Ci < 1 || H < 1 || W < 1 || Co < 1 || K < 1 || pad < 0) return 0;
+    const long long Ho = (long long)H + 2 * pad - K + 1, Wo = (long long)W + 2 * pad - K + 1;
+    if (Ho < 1 || Wo < 1) return 0;
+    // packed kernel rows: at most K words per (ci, kh) row (one tap per word in the comparator), Co rounded up to 4
+    const size_t weights = align_up((size_t)Ci * K * K * ((Co + 3) / 4 * 4) * sizeof(uint32_t), 256);
+    // packed activation rows: at most one word per output pixel plus K halo words per row (the comparator's
+    // layout), rounded up to 16-byte pieces, with one more piece per row segment (segments hold >= 32 blocks)
+    const size_t row_words = (size_t)(Wo + K + 3) / 4 * 4 + 16 + (size_t)(Wo + K) / 8;
+    const size_t acts = (size_t)Ci * B * (size_t)(Ho + K - 1) * row_words * sizeof(uint32_t);
+    return weights + align_up(acts, 256);
 }
 
 extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K, int stride,
@@ -636,16 +617,31 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
                         tune, &s);
     if (rc != HIKONV_OK) return rc;
     if (!requant && ((uintptr_t)d_out % 4) != 0) return HIKONV_ERR_INVALID_ARG;
-    if (!d_workspace || ((uintptr_t)d_workspace % 256) != 0 || workspace_bytes < hikonv_conv2d_workspace_bytes(Ci, Co, K))
+    const size_t need = s.wp_bytes + s.ap_words * sizeof(uint32_t);
+    if (!d_workspace || ((uintptr_t)d_workspace % 256) != 0 || workspace_bytes < need ||
+        workspace_bytes < hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad))
         return HIKONV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    uint32_t *d_wp = (uint32_t *)d_workspace;
+    uint32_t *d_ap = (uint32_t *)((char *)d_workspace + s.wp_bytes);
     s.kp.x = d_x;
-    s.kp.async_ok = ((uintptr_t)d_x % 4 == 0) ? 1 : 0;
-    s.kp.wp = (const uint32_t *)d_workspace;
+    s.kp.wp = d_wp;
+    s.kp.ap = d_ap;
     s.kp.out = d_out;
-    const int total = Ci * K * s.L.J * s.kp.CoP;
-    pack_weights_kernel<<<ceil_div(total, 256), 256, 0, st>>>(d_w, Co, Ci, K, s.L.J, s.L.Kc, s.L.S, w_signed ? 1 : 0, s.kp.CoP,
-                                                             (uint32_t *)d_workspace, total);
+    // a2: reversed kernel rows packed per (ci, kh, chunk); a3: activation rows packed per block
+    const int total_w = Ci * K * s.L.J * s.kp.CoP;
+    pack_weights_kernel<<<ceil_div(total_w, 256), 256, 0, st>>>(d_w, Co, Ci, K, s.L.J, s.L.Kc, s.L.S, w_signed ? 1 : 0, s.kp.CoP,
+                                                               d_wp, total_w);
+    rc = launch_status();
+    if (rc != HIKONV_OK) return rc;
+    const size_t blocks_a = (s.ap_words + 255) / 256;
+    if (blocks_a > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
+    if (x_signed)
+        pack_activations_kernel<true><<<(unsigned)blocks_a, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.N, s.L.S,
+                                                                         s.kp.XBT, d_ap, s.ap_words);
+    else
+        pack_activations_kernel<false><<<(unsigned)blocks_a, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.N, s.L.S,
+                                                                          s.kp.XBT, d_ap, s.ap_words);
     rc = launch_status();
     if (rc != HIKONV_OK) return rc;
     return launch_conv2d(s, x_signed != 0, st);
@@ -679,13 +675,13 @@ extern "C" int hikonv_conv2d_static_scratch(const int8_t *d_x, int B, int Ci, in
                                             int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out,
                                             int requant, int shift, int lo, int hi, int algo, const hikonv_tuning_t *tune,
                                             void *stream) {
-    if (Ci < 1 || Co < 1 || K < 1) return HIKONV_ERR_INVALID_ARG;
-    const size_t need = hikonv_conv2d_workspace_bytes(Ci, Co, K);
+    const size_t need = hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad);
+    if (need == 0) return HIKONV_ERR_INVALID_ARG;
     if (need > (size_t)HIKONV_STATIC_SCRATCH_BYTES) return HIKONV_ERR_TOO_LARGE;
     void *scratch = nullptr;
     const int rc = static_scratch_address(&scratch);
     if (rc != HIKONV_OK) return rc;
-    // the packing kernel writes every word the layer kernel reads, so stale contents are harmless
+    // the packing kernels write every word the layer kernel reads, so stale contents are harmless
     return hikonv_conv2d(d_x, B, Ci, H, W, d_w, Co, K, stride, pad, p, q, x_signed, w_signed, d_out, requant, shift, lo, hi,
                          scratch, (size_t)HIKONV_STATIC_SCRATCH_BYTES, algo, tune, stream);
 }
@@ -696,7 +692,7 @@ extern "C" size_t hikonv_conv2d_host_workspace_bytes(int B, int Ci, int H, int W
     if (Ho < 1 || Wo < 1) return 0;
     const size_t out_bytes = (size_t)B * Co * Ho * Wo * (requant ? 1 : 4);
     return align_up((size_t)B * Ci * H * W, 256) + align_up((size_t)Co * Ci * K * K, 256) + align_up(out_bytes, 256) +
-           hikonv_conv2d_workspace_bytes(Ci, Co, K);
+           hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad);
 }
 
 extern "C" int hikonv_conv2d_host(const int8_t *h_x, int B, int Ci, int H, int W, const int8_t *h_w, int Co, int K, int stride,
@@ -718,7 +714,7 @@ extern "C" int hikonv_conv2d_host(const int8_t *h_x, int B, int Ci, int H, int W
     HIKONV_CUDA_TRY(cudaMemcpyAsync(d_x, h_x, x_bytes, cudaMemcpyHostToDevice, st));
     HIKONV_CUDA_TRY(cudaMemcpyAsync(d_w, h_w, w_bytes, cudaMemcpyHostToDevice, st));
     const int rc = hikonv_conv2d(d_x, B, Ci, H, W, d_w, Co, K, stride, pad, p, q, x_signed, w_signed, d_out, requant, shift, lo,
-                                 hi, d_ws, hikonv_conv2d_workspace_bytes(Ci, Co, K), algo, tune, st);
+                                 hi, d_ws, hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad), algo, tune, st);
     if (rc != HIKONV_OK) return rc;
     HIKONV_CUDA_TRY(cudaMemcpyAsync(h_out, d_out, out_bytes, cudaMemcpyDeviceToHost, st));
     return HIKONV_OK;

@@ -19,18 +19,32 @@ class CompactCnn:
     def __init__(self, layers: List[dict], head_w, device="cuda"):
         self.device = torch.device(device)
         self.layers = []
-        ws_bytes = 0
         for L in layers:
             w = torch.from_numpy(inputs.to_storage(L["w"])).to(self.device)
             self.layers.append({**{k: v for k, v in L.items() if k != "w"}, "d_w": w})
-            Co, Ci, K, _ = w.shape
-            ws_bytes = max(ws_bytes, hk.conv2d_workspace_bytes(Ci, Co, K))
         self.head_w = torch.from_numpy(inputs.to_storage(head_w)).to(self.device)
+        self.workspace = None
+        self._ws_shape = None
+
+    def _ensure_workspace(self, shape):
+        """One workspace large enough for every layer of a batch of this input shape."""
+        if self._ws_shape == tuple(shape):
+            return
+        B, _, H, W = shape
+        need = 0
+        for L in self.layers:
+            Co, Ci, K, _ = L["d_w"].shape
+            need = max(need, hk.conv2d_workspace_bytes(B, Ci, H, W, Co, K, L["pad"]))
+            H, W = H + 2 * L["pad"] - K + 1, W + 2 * L["pad"] - K + 1
+            if L["pool"]:
+                H, W = H // 2, W // 2
         Co, Ci, K, _ = self.head_w.shape
-        ws_bytes = max(ws_bytes, hk.conv2d_workspace_bytes(Ci, Co, K))
-        self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=self.device)
+        need = max(need, hk.conv2d_workspace_bytes(B, Ci, H, W, Co, K, 0))
+        self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        self._ws_shape = tuple(shape)
 
     def forward(self, d_x: torch.Tensor, algo: int = hk.ALGO_PACKED32, keep_activations: bool = False, stream=None):
+        self._ensure_workspace(d_x.shape)
         acts = []
         a = d_x
         for L in self.layers:

@@ -162,7 +162,9 @@ def test_device_entry_points_validate_before_touching_cuda():
     assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 0, 0, 0, 0, None, 0, 0, None, None) == hk.ERR_WORKSPACE
     assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 1, 40, 0, 15, 256, 1 << 20, 0, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_maxpool2x2_i8(None, 1, 1, 4, 4, 0, None, None) == hk.ERR_INVALID_ARG
-    assert hk.conv2d_workspace_bytes(64, 64, 3) >= 64 * 3 * 64 * 4
+    # room for the packed kernel rows and for one packed word per input pixel in the comparator's layout
+    assert hk.conv2d_workspace_bytes(2, 64, 8, 8, 64, 3, 1) >= 64 * 3 * 3 * 64 * 4 + 64 * 2 * 10 * 11 * 4
+    assert hk.conv2d_workspace_bytes(2, 64, 8, 8, 64, 3, 4) > 0 and hk.conv2d_workspace_bytes(2, 64, 2, 2, 64, 7, 0) == 0
     assert hk.conv1d_host_workspace_bytes(1000, 3) >= 1000 + 3 + 4 * 1002
 
 

@@ -4,7 +4,7 @@
 (they own only the input and output tensors, or may not allocate once their service has started).
 It must give exactly what ``hikonv_conv2d`` gives with a caller-provided workspace, on consecutive
 calls that reuse the built-in buffer with different contents, and it must refuse layers whose
-packed weights do not fit that buffer.  This file sorts last on purpose, so a run that stops at the
+packed rows do not fit that buffer.  This file sorts last on purpose, so a run that stops at the
 first failure has already exercised every other test.
 """
 import numpy as np
@@ -42,8 +42,8 @@ def test_static_scratch_matches_workspace_path_on_consecutive_calls():
 
 
 def test_static_scratch_rejects_layers_beyond_its_capacity():
-    # 512 x 512 x 3 x 3 needs 512*3*3*512*4 bytes = 9.4 MB of packed rows: more than the built-in 4 MiB
-    assert hk.conv2d_workspace_bytes(512, 512, 3) > hk.STATIC_SCRATCH_BYTES
+    # 512 x 512 x 3 x 3 needs 512*3*3*512*4 bytes = 9.4 MB of packed kernel rows alone: more than the built-in 4 MiB
+    assert hk.conv2d_workspace_bytes(1, 512, 4, 4, 512, 3, 1) > hk.STATIC_SCRATCH_BYTES
     d_x = torch.zeros((1, 512, 4, 4), dtype=torch.int8, device="cuda")
     d_w = torch.zeros((512, 512, 3, 3), dtype=torch.int8, device="cuda")
     out = torch.empty((1, 512, 4, 4), dtype=torch.int32, device="cuda")
