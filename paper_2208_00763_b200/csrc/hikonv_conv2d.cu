@@ -87,10 +87,13 @@ __device__ __forceinline__ void mac(typename AccType<UNPACKED>::type &acc, uint3
 
 // N: pixels per packed word; SC: slot width when known at compile time (0: read from the parameters);
 // TM x TN: per-thread tile (positions x channels); UNPACKED: comparator (N == 1, one tap per word,
-// 32-bit multiply-add, int32 accumulators); SP: signed product; XS: signed activations;
+// 32-bit multiply-add, int32 accumulators); SP: signed product;
 // KT, JT: kernel size and chunks per kernel row when known at compile time (0, 0: read from the
-// parameters; the (kh, j) loops are then not unrolled).
-template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, bool XS, int KT, int JT>
+// parameters; the (kh, j) loops are then not unrolled);
+// PITCH: words per activation row in shared memory when known at compile time (then every operand load
+// of the unrolled loops has an immediate offset), 0: read from the parameters.
+constexpr int kBPitch = 64;        // words per packed kernel row in shared memory (TCO <= 64)
+template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, int KT, int JT, int PITCH>
 __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dParams p) {
     typedef typename AccType<UNPACKED>::type acc_t;
     extern __shared__ __align__(16) uint32_t smem[];
@@ -158,7 +161,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     };
 
     const int KJ = p.K * p.J;
-    const int xq = p.XBS / 4;                                        // 16-byte pieces per activation row
+    const int xq = (p.XB + 3) / 4;                                   // 16-byte pieces per activation row
     const size_t ap_plane = (size_t)p.B * p.Hp * p.XBT;              // words per channel of Ap
     const uint32_t *ap_tile = p.ap + (size_t)Rp0 * p.XBT + seg * p.XO;   // first word this tile reads (16-byte aligned)
 
@@ -179,7 +182,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         for (int idx = tid; idx < rows * tco4; idx += nthreads) {
             const int kr = idx / tco4, c4 = idx - kr * tco4;
             const int co = co0 + c4 * 4;
-            uint32_t *dst = Bdst + (kr * tco4 + c4) * 4;
+            uint32_t *dst = Bdst + kr * kBPitch + c4 * 4;
             if (co < p.CoP) cp_async_16(dst, p.wp + (size_t)(ci0 * KJ + kr) * p.CoP + co);
             else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
         }
@@ -197,22 +200,22 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         const int astage = stage * p.a_words;
         const uint32_t *bptr = Bs + stage * p.b_words + tn * TN;
         // ---- multiply-accumulate over (ci, kh, j)
-        if constexpr (KT > 0) {
+        if constexpr (KT > 0 && PITCH > 0) {
+            const uint32_t *ap[TM];
+#pragma unroll
+            for (int i = 0; i < TM; ++i) ap[i] = aptr[i] + astage;
+            const uint32_t *bp = bptr;
             for (int cl = 0; cl < ckn; ++cl) {
-                const int abase = astage + cl * p.a_plane;
-                const int bbase = cl * (KT * JT) * p.TCO;
 #pragma unroll
                 for (int kh = 0; kh < KT; ++kh) {
 #pragma unroll
                     for (int j = 0; j < JT; ++j) {
-                        const int aoff = abase + kh * p.XBS - j;
-                        const uint32_t *brow = bptr + bbase + (kh * JT + j) * p.TCO;
                         uint32_t a[TM], b[TN];
 #pragma unroll
-                        for (int i = 0; i < TM; ++i) a[i] = aptr[i][aoff];
+                        for (int i = 0; i < TM; ++i) a[i] = ap[i][kh * PITCH - j];
 #pragma unroll
                         for (int t = 0; t < TN; t += 4) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(brow + t);
+                            const uint4 v = *reinterpret_cast<const uint4 *>(bp + (kh * JT + j) * kBPitch + t);
                             b[t] = v.x; b[t + 1] = v.y; b[t + 2] = v.z; b[t + 3] = v.w;
                         }
 #pragma unroll
@@ -221,13 +224,16 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                             for (int t = 0; t < TN; ++t) mac<UNPACKED, SP>(acc[i][t], a[i], b[t]);
                     }
                 }
+#pragma unroll
+                for (int i = 0; i < TM; ++i) ap[i] += p.a_plane;
+                bp += KT * JT * kBPitch;
             }
         } else {
             for (int cl = 0; cl < ckn; ++cl) {
                 for (int kh = 0; kh < p.K; ++kh) {
                     for (int j = 0; j < p.J; ++j) {
                         const int aoff = astage + cl * p.a_plane + kh * p.XBS - j;
-                        const uint32_t *brow = bptr + ((cl * p.K + kh) * p.J + j) * p.TCO;
+                        const uint32_t *brow = bptr + ((cl * p.K + kh) * p.J + j) * kBPitch;
                         uint32_t a[TM], b[TN];
 #pragma unroll
                         for (int i = 0; i < TM; ++i) a[i] = aptr[i][aoff];
@@ -408,20 +414,32 @@ static int sm_count() {
     return sms;
 }
 
-template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT>
-static int launch_variant(const Conv2dSetup &s, bool sp, bool xs, cudaStream_t st) {
-#define HK_LAUNCH(SPV, XSV)                                                                                      \
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, int PITCH>
+static int launch_pitch(const Conv2dSetup &s, bool sp, cudaStream_t st) {
+#define HK_LAUNCH(SPV)                                                                                           \
     do {                                                                                                         \
-        auto kern = conv2d_kernel<N, SC, TM, TN, UNPACKED, SPV, XSV, KT, JT>;                                    \
+        auto kern = conv2d_kernel<N, SC, TM, TN, UNPACKED, SPV, KT, JT, PITCH>;                                  \
         if (s.smem_bytes > 48 * 1024)                                                                            \
             HIKONV_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem_bytes)); \
         kern<<<s.grid, s.threads, s.smem_bytes, st>>>(s.kp);                                                     \
     } while (0)
-    if (!sp) HK_LAUNCH(false, false);
-    else if (xs) HK_LAUNCH(true, true);
-    else HK_LAUNCH(true, false);
+    if (!sp) HK_LAUNCH(false);
+    else HK_LAUNCH(true);
 #undef HK_LAUNCH
     return launch_status();
+}
+
+// KT > 0: the kernel with unrolled (kh, j) loops and a compile-time row pitch; KT == 0: everything at run time.
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT>
+static int launch_variant(const Conv2dSetup &s, bool sp, cudaStream_t st) {
+    if (KT == 0) return launch_pitch<N, SC, TM, TN, UNPACKED, 0, 0, 0>(s, sp, st);
+    switch (s.kp.XBS) {
+        case 8: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 8>(s, sp, st);
+        case 16: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 16>(s, sp, st);
+        case 32: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 32>(s, sp, st);
+        case 64: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 64>(s, sp, st);
+        default: return HIKONV_ERR_UNSUPPORTED;
+    }
 }
 
 constexpr int kTM = 4, kTN = 4;          // per-thread tile of the packed kernels
@@ -449,9 +467,10 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
         const int maxpos = max_tmx * TM;
         // rows wider than a tile are cut into segments of XO blocks (a multiple of 4, so that every tile
         // row starts on a 16-byte boundary of the packed activations), each with its own J halo positions
+        const int rowmax = std::min(maxpos, 64);                  // a staged row holds at most 64 words
         int NSEG = 1, XO = X;
-        if (X + J > maxpos) {
-            XO = (maxpos - J) / 4 * 4;
+        if (X + J > rowmax) {
+            XO = (rowmax - J) / 4 * 4;
             if (XO < 4) continue;
             NSEG = ceil_div(X, XO);
             XO = (ceil_div(X, NSEG) + 3) / 4 * 4;
@@ -536,8 +555,9 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     s->threads = tc.TMX * tc.TNX;
     const int span = (kp.TR + Ho - 2) / Ho + 1;              // images a tile can touch
     kp.NRmax = kp.TR + (K - 1) * span;
-    kp.XBS = (kp.XB + 3) / 4 * 4;
-    kp.XBT = (kp.NSEG - 1) * kp.XO + kp.XBS;
+    // words per activation row in shared memory: 8, 16, 32 or 64 (the unrolled kernels have them as constants)
+    kp.XBS = kp.XB <= 8 ? 8 : kp.XB <= 16 ? 16 : kp.XB <= 32 ? 32 : 64;
+    kp.XBT = (kp.NSEG - 1) * kp.XO + (kp.XB + 3) / 4 * 4;
     kp.lead = (L.J + 3) / 4 * 4;                             // room for the xb - j reads in front of the first row
     kp.a_plane = kp.NRmax * kp.XBS + kp.lead;
     // channels per stage and stages between two carry-save moves (at most M (ci, kh) pairs)
@@ -553,7 +573,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.CK = CK;
     kp.a_words = CK * kp.a_plane;
     kp.b_off = 2 * kp.a_words;
-    kp.b_words = CK * K * L.J * kp.TCO;
+    kp.b_words = CK * K * L.J * kBPitch;
     const size_t words = (size_t)kp.b_off + 2 * (size_t)kp.b_words;
     const size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
     s->smem_bytes = std::max(words, xch_words) * 4 + 16;
@@ -568,24 +588,24 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     return HIKONV_OK;
 }
 
-static int launch_conv2d(const Conv2dSetup &s, bool xs, cudaStream_t st) {
+static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
     const bool sp = s.L.signed_prod != 0;
     const int K = s.kp.K, J = s.L.J;
     if (s.unpacked) {
-        if (K == 3) return launch_variant<1, 0, kTMU, kTNU, true, 3, 3>(s, sp, xs, st);
-        if (K == 1) return launch_variant<1, 0, kTMU, kTNU, true, 1, 1>(s, sp, xs, st);
-        return launch_variant<1, 0, kTMU, kTNU, true, 0, 0>(s, sp, xs, st);
+        if (K == 3) return launch_variant<1, 0, kTMU, kTNU, true, 3, 3>(s, sp, st);
+        if (K == 1) return launch_variant<1, 0, kTMU, kTNU, true, 1, 1>(s, sp, st);
+        return launch_variant<1, 0, kTMU, kTNU, true, 0, 0>(s, sp, st);
     }
     // the layouts of 3x3 and 1x1 layers with the slot width and loop bounds as compile-time constants
-    if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1>(s, sp, xs, st);
-    if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, xs, st);
-    if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, xs, st);
-    if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, xs, st);
+    if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1>(s, sp, st);
+    if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, st);
+    if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
+    if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     switch (s.L.N) {
-        case 1: return launch_variant<1, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
-        case 2: return launch_variant<2, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
-        case 3: return launch_variant<3, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
-        case 4: return launch_variant<4, 0, kTM, kTN, false, 0, 0>(s, sp, xs, st);
+        case 1: return launch_variant<1, 0, kTM, kTN, false, 0, 0>(s, sp, st);
+        case 2: return launch_variant<2, 0, kTM, kTN, false, 0, 0>(s, sp, st);
+        case 3: return launch_variant<3, 0, kTM, kTN, false, 0, 0>(s, sp, st);
+        case 4: return launch_variant<4, 0, kTM, kTN, false, 0, 0>(s, sp, st);
         default: return HIKONV_ERR_UNSUPPORTED;
     }
 }
@@ -644,7 +664,7 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
                                                                           s.kp.XBT, d_ap, s.ap_words);
     rc = launch_status();
     if (rc != HIKONV_OK) return rc;
-    return launch_conv2d(s, x_signed != 0, st);
+    return launch_conv2d(s, st);
 }
 
 // ---- scratch that needs no allocation: a fixed buffer inside the library image, one copy per GPU
