@@ -486,7 +486,12 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
             if (threads > kMaxThreads2D) continue;
             TMX = threads / TNX;
             const long long tiles = (long long)ceil_div(total_rows, TR) * NSEG * gy;
-            const int per_sm = std::max(1, std::min(2048 / threads, 65536 / (threads * 128)));
+            // shared memory of the two double-buffered tiles (8 channels per stage at most)
+            const int pitch = XB <= 8 ? 8 : XB <= 16 ? 16 : XB <= 32 ? 32 : 64;
+            const int span_s = (TR + Ho - 2) / Ho + 1;
+            const size_t smem = 2 * 4 * ((size_t)8 * ((TR + (K - 1) * span_s) * pitch + 8) + (size_t)8 * K * J * kBPitch);
+            if (smem > 100 * 1024) continue;
+            const int per_sm = std::max(1, std::min(std::min(2048 / threads, 65536 / (threads * 128)), (int)(220 * 1024 / smem)));
             const long long slots = (long long)per_sm * sms;
             const long long full_waves = tiles / slots;
             const long long rest = tiles - full_waves * slots;
