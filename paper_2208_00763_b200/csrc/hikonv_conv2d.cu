@@ -143,18 +143,27 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
     int nmoves = 0, chunks_since_move = 0;
 
-    // move the upper bits of every slot to E and restart the slots at their bias
+    // move the upper bits of every slot to E and restart the slots at their bias (on 32-bit halves, so
+    // that it is two funnel/plain shifts, four logic operations and one add with carry per accumulator)
     auto carry_save = [&]() {
         if constexpr (!UNPACKED) {
-            const uint64_t mask_high = p.mask_high, mask_low = p.mask_low, bias = p.bias;
-            const int h = p.hbits;
+            const uint32_t mh_lo = (uint32_t)p.mask_high, mh_hi = (uint32_t)(p.mask_high >> 32);
+            const uint32_t ml_lo = (uint32_t)p.mask_low, ml_hi = (uint32_t)(p.mask_low >> 32);
+            const uint32_t b_lo = (uint32_t)p.bias, b_hi = (uint32_t)(p.bias >> 32);
+            const int h = p.hbits;                                   // 1 .. 31 whenever a move happens
 #pragma unroll
             for (int i = 0; i < TM; ++i)
 #pragma unroll
                 for (int t = 0; t < TN; ++t) {
-                    const uint64_t Q = (uint64_t)acc[i][t];
-                    E[i][t] += (Q >> h) & mask_high;
-                    acc[i][t] = (acc_t)((Q & mask_low) | bias);
+                    uint32_t qlo = (uint32_t)acc[i][t], qhi = (uint32_t)((uint64_t)acc[i][t] >> 32);
+                    uint32_t elo = (uint32_t)E[i][t], ehi = (uint32_t)((uint64_t)E[i][t] >> 32);
+                    const uint32_t hlo = __funnelshift_r(qlo, qhi, h) & mh_lo;
+                    const uint32_t hhi = (qhi >> h) & mh_hi;
+                    asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(elo), "+r"(ehi) : "r"(hlo), "r"(hhi));
+                    qlo = (qlo & ml_lo) | b_lo;
+                    qhi = (qhi & ml_hi) | b_hi;
+                    E[i][t] = (acc_t)(((uint64_t)ehi << 32) | elo);
+                    acc[i][t] = (acc_t)(((uint64_t)qhi << 32) | qlo);
                 }
             ++nmoves;
         }
@@ -162,28 +171,55 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 
     const int KJ = p.K * p.J;
     const int xq = (p.XB + 3) / 4;                                   // 16-byte pieces per activation row
-    const size_t ap_plane = (size_t)p.B * p.Hp * p.XBT;              // words per channel of Ap
+    const int ap_plane = p.B * p.Hp * p.XBT;                         // words per channel of Ap
     const uint32_t *ap_tile = p.ap + (size_t)Rp0 * p.XBT + seg * p.XO;   // first word this tile reads (16-byte aligned)
+
+    // The 16-byte pieces of an activation stage this thread copies: the same ones every stage, so their
+    // offsets are worked out once (channel in the top byte of the destination offset, -1: none).
+    constexpr int kPieces = 4;
+    int piece_src[kPieces], piece_dst[kPieces];
+    {
+        const int per_ch = NR * xq;
+#pragma unroll
+        for (int k = 0; k < kPieces; ++k) {
+            const int q = tid + k * nthreads;
+            piece_src[k] = 0;
+            piece_dst[k] = -1;
+            if (q < p.CK * per_ch) {
+                const int cl = q / per_ch, r = q - cl * per_ch;
+                const int rl = r / xq, qd = r - rl * xq;
+                piece_src[k] = cl * ap_plane + rl * p.XBT + 4 * qd;
+                piece_dst[k] = (cl << 24) | (cl * p.a_plane + p.lead + rl * p.XBS + 4 * qd);
+            }
+        }
+    }
+    const bool pieces_in_regs = p.CK * NR * xq <= kPieces * nthreads;
+    const int tco4 = p.TCO / 4, tco4_log2 = 31 - __clz(tco4);        // TCO / 4 is a power of two
 
     // Asynchronous fetch of one stage: NR packed rows of ckn channels and the packed kernel rows of the
     // same channels for TCO output channels, all in 16-byte pieces.
     auto fetch = [&](int ci0, int ckn, uint32_t *Adst, uint32_t *Bdst) {
-        const int per_ch = NR * xq;
-        for (int cl = 0; cl < ckn; ++cl) {
-            const uint32_t *src = ap_tile + (size_t)(ci0 + cl) * ap_plane;
-            uint32_t *dst = Adst + cl * p.a_plane + p.lead;
-            for (int idx = tid; idx < per_ch; idx += nthreads) {
-                const int rl = idx / xq, qd = idx - rl * xq;
-                cp_async_16(dst + rl * p.XBS + 4 * qd, src + (size_t)rl * p.XBT + 4 * qd);
+        const uint32_t *asrc = ap_tile + (size_t)ci0 * ap_plane;
+        if (pieces_in_regs) {
+#pragma unroll
+            for (int k = 0; k < kPieces; ++k)
+                if (piece_dst[k] >= 0 && (piece_dst[k] >> 24) < ckn) cp_async_16(Adst + (piece_dst[k] & 0xFFFFFF), asrc + piece_src[k]);
+        } else {
+            const int per_ch = NR * xq;
+            for (int cl = 0; cl < ckn; ++cl) {
+                const uint32_t *src = asrc + (size_t)cl * ap_plane;
+                uint32_t *dst = Adst + cl * p.a_plane + p.lead;
+                for (int idx = tid; idx < per_ch; idx += nthreads) {
+                    const int rl = idx / xq, qd = idx - rl * xq;
+                    cp_async_16(dst + rl * p.XBS + 4 * qd, src + (size_t)rl * p.XBT + 4 * qd);
+                }
             }
         }
-        const int tco4 = p.TCO / 4;
-        const int rows = ckn * KJ;
-        for (int idx = tid; idx < rows * tco4; idx += nthreads) {
-            const int kr = idx / tco4, c4 = idx - kr * tco4;
-            const int co = co0 + c4 * 4;
+        const uint32_t *bsrc = p.wp + (size_t)ci0 * KJ * p.CoP + co0;
+        for (int idx = tid; idx < (ckn * KJ) << tco4_log2; idx += nthreads) {
+            const int kr = idx >> tco4_log2, c4 = idx & (tco4 - 1);
             uint32_t *dst = Bdst + kr * kBPitch + c4 * 4;
-            if (co < p.CoP) cp_async_16(dst, p.wp + (size_t)(ci0 * KJ + kr) * p.CoP + co);
+            if (co0 + c4 * 4 < p.CoP) cp_async_16(dst, bsrc + kr * p.CoP + c4 * 4);
             else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
         }
         cp_async_commit();
@@ -584,6 +620,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     s->smem_bytes = std::max(words, xch_words) * 4 + 16;
     s->wp_bytes = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
     s->ap_words = (size_t)Ci * B * kp.Hp * kp.XBT;
+    if (s->ap_words >= 0x7FFFFFFFull || (size_t)Ci * K * L.J * kp.CoP >= 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
     if (s->smem_bytes > 200 * 1024) return HIKONV_ERR_UNSUPPORTED;
     const long long row_tiles = ((long long)kp.total_rows + kp.TR - 1) / kp.TR;
     const long long gx = row_tiles * kp.NSEG;
