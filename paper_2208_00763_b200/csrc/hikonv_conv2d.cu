@@ -53,7 +53,8 @@ struct Conv2dParams {
     int NRmax, a_plane, lead;  // staged rows per channel; words per channel in shared memory; words before the first row
     int a_words;               // words per activation tile (CK * a_plane)
     int b_off;                 // word offset of the first weight tile in shared memory
-    int b_words;               // words per weight tile (CK * K * J * TCO)
+    int b_words;               // words per weight tile (CK * K * J rows of 64 words)
+    int e_off;                 // word offset of the second accumulators in shared memory (after the tiles and the exchange area)
     int requant, shift, lo, hi;
     int total_rows;            // B * Ho
     int flush_chunks;          // channel stages accumulated between two carry-save moves (CK * K * flush_chunks <= M)
@@ -130,16 +131,17 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
 
     acc_t acc[TM][TN];
-    acc_t E[UNPACKED ? 1 : TM][UNPACKED ? 1 : TN];     // second packed accumulator (upper slot bits)
+    // second packed accumulator (upper slot bits): in shared memory, one 8-byte entry per accumulator and
+    // thread, [accumulator][thread] so that a warp touches consecutive entries; only read-modify-written
+    // every M products, it would otherwise hold half of the thread's registers
+    uint2 *Es = reinterpret_cast<uint2 *>(smem + p.e_off) + tid;
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int t = 0; t < TN; ++t) acc[i][t] = UNPACKED ? (acc_t)0 : (acc_t)p.bias;
     if constexpr (!UNPACKED) {
 #pragma unroll
-        for (int i = 0; i < TM; ++i)
-#pragma unroll
-            for (int t = 0; t < TN; ++t) E[i][t] = 0;
+        for (int k = 0; k < TM * TN; ++k) Es[k * kMaxThreads2D] = make_uint2(0u, 0u);
     }
     int nmoves = 0, chunks_since_move = 0;
 
@@ -156,13 +158,14 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
                 for (int t = 0; t < TN; ++t) {
                     uint32_t qlo = (uint32_t)acc[i][t], qhi = (uint32_t)((uint64_t)acc[i][t] >> 32);
-                    uint32_t elo = (uint32_t)E[i][t], ehi = (uint32_t)((uint64_t)E[i][t] >> 32);
+                    uint2 e = Es[(i * TN + t) * kMaxThreads2D];
+                    uint32_t elo = e.x, ehi = e.y;
                     const uint32_t hlo = __funnelshift_r(qlo, qhi, h) & mh_lo;
                     const uint32_t hhi = (qhi >> h) & mh_hi;
                     asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(elo), "+r"(ehi) : "r"(hlo), "r"(hhi));
                     qlo = (qlo & ml_lo) | b_lo;
                     qhi = (qhi & ml_hi) | b_hi;
-                    E[i][t] = (acc_t)(((uint64_t)ehi << 32) | elo);
+                    Es[(i * TN + t) * kMaxThreads2D] = make_uint2(elo, ehi);
                     acc[i][t] = (acc_t)(((uint64_t)qhi << 32) | qlo);
                 }
             ++nmoves;
@@ -298,6 +301,10 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         const uint32_t ev = (uint32_t)(Ev >> (S * m)) & msk;
         return (ev << p.hbits) + qv - nb * (uint32_t)p.slot_bias[m];
     };
+    auto load_e = [&](int i, int t) -> uint64_t {
+        const uint2 e = Es[(i * TN + t) * kMaxThreads2D];
+        return ((uint64_t)e.y << 32) | e.x;
+    };
     // the upper slots of a thread's last position belong to the next thread's first position (Theorem 2)
     if constexpr (!UNPACKED) {
         __syncthreads();
@@ -307,7 +314,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
             for (int t = 0; t < TN; ++t)
                 xch[(tm * N + m) * p.TCO + tn * TN + t] =
-                    (N + m < p.nslots) ? slot_value((uint64_t)acc[TM - 1][t], (uint64_t)E[TM - 1][t], N + m) : 0u;
+                    (N + m < p.nslots) ? slot_value((uint64_t)acc[TM - 1][t], load_e(TM - 1, t), N + m) : 0u;
         __syncthreads();
     }
 
@@ -324,11 +331,12 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         for (int i = 0; i < TM; ++i) {
             uint32_t Y[N];
             if constexpr (!UNPACKED) {
+                const uint64_t ev = load_e(i, t);
 #pragma unroll
-                for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], (uint64_t)E[i][t], m) + upper[m];
+                for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], ev, m) + upper[m];
 #pragma unroll
                 for (int m = 0; m < N; ++m)
-                    upper[m] = (N + m < p.nslots) ? slot_value((uint64_t)acc[i][t], (uint64_t)E[i][t], N + m) : 0u;
+                    upper[m] = (N + m < p.nslots) ? slot_value((uint64_t)acc[i][t], ev, N + m) : 0u;
             } else {
                 Y[0] = (uint32_t)acc[i][t];
             }
@@ -526,8 +534,8 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
             const int pitch = XB <= 8 ? 8 : XB <= 16 ? 16 : XB <= 32 ? 32 : 64;
             const int span_s = (TR + Ho - 2) / Ho + 1;
             const size_t smem = 2 * 4 * ((size_t)8 * ((TR + (K - 1) * span_s) * pitch + 8) + (size_t)8 * K * J * kBPitch);
-            if (smem > 100 * 1024) continue;
-            const int per_sm = std::max(1, std::min(std::min(2048 / threads, 65536 / (threads * 128)), (int)(220 * 1024 / smem)));
+            if (smem > 72 * 1024) continue;                            // plus 32 KB of second accumulators per CTA
+            const int per_sm = std::max(1, std::min(std::min(2048 / threads, 65536 / (threads * 128)), (int)(220 * 1024 / (smem + 32 * 1024))));
             const long long slots = (long long)per_sm * sms;
             const long long full_waves = tiles / slots;
             const long long rest = tiles - full_waves * slots;
@@ -617,7 +625,9 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.b_words = CK * K * L.J * kBPitch;
     const size_t words = (size_t)kp.b_off + 2 * (size_t)kp.b_words;
     const size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
-    s->smem_bytes = std::max(words, xch_words) * 4 + 16;
+    kp.e_off = (int)((std::max(words, xch_words) + 3) / 4 * 4);
+    const size_t e_words = s->unpacked ? 0 : (size_t)TM * TN * kMaxThreads2D * 2;
+    s->smem_bytes = ((size_t)kp.e_off + e_words) * 4 + 16;
     s->wp_bytes = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
     s->ap_words = (size_t)Ci * B * kp.Hp * kp.XBT;
     if (s->ap_words >= 0x7FFFFFFFull || (size_t)Ci * K * L.J * kp.CoP >= 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
