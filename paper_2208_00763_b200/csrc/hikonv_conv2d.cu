@@ -93,7 +93,6 @@ __device__ __forceinline__ void mac(typename AccType<UNPACKED>::type &acc, uint3
 // parameters; the (kh, j) loops are then not unrolled);
 // PITCH: words per activation row in shared memory when known at compile time (then every operand load
 // of the unrolled loops has an immediate offset), 0: read from the parameters.
-constexpr int kBPitch = 64;        // words per packed kernel row in shared memory (TCO <= 64)
 template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, int KT, int JT, int PITCH>
 __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dParams p) {
     typedef typename AccType<UNPACKED>::type acc_t;
@@ -533,7 +532,8 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
             // shared memory of the two double-buffered tiles (8 channels per stage at most)
             const int pitch = XB <= 8 ? 8 : XB <= 16 ? 16 : XB <= 32 ? 32 : 64;
             const int span_s = (TR + Ho - 2) / Ho + 1;
-            const size_t smem = 2 * 4 * ((size_t)8 * ((TR + (K - 1) * span_s) * pitch + 8) + (size_t)8 * K * J * kBPitch);
+            const int ckc = stage_channel_cap(K, J);
+            const size_t smem = 2 * 4 * ((size_t)ckc * ((TR + (K - 1) * span_s) * pitch + 8) + (size_t)ckc * K * J * kBPitch);
             if (smem > 72 * 1024) continue;                            // plus 32 KB of second accumulators per CTA
             const int per_sm = std::max(1, std::min(std::min(2048 / threads, 65536 / (threads * 128)), (int)(220 * 1024 / (smem + 32 * 1024))));
             const long long slots = (long long)per_sm * sms;
@@ -610,12 +610,13 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.lead = (L.J + 3) / 4 * 4;                             // room for the xb - j reads in front of the first row
     kp.a_plane = kp.NRmax * kp.XBS + kp.lead;
     // channels per stage and stages between two carry-save moves (at most M (ci, kh) pairs)
-    int CK = std::min(8, Ci);
+    const int ck_cap = stage_channel_cap(K, L.J);
+    int CK = std::min(ck_cap, Ci);
     kp.flush_chunks = 1 << 30;
     if (!s->unpacked && L.M < Ci * K) {
         if (L.M < K) return HIKONV_ERR_NO_FIT;               // not even one channel's kernel rows between two moves
         int fc = 1;
-        const int eff = pick_chunking(L.M / K, Ci, &CK, &fc);
+        const int eff = pick_chunking(L.M / K, Ci, &CK, &fc, ck_cap);
         if (ceil_div(Ci, eff) > (1 << L.carry_bits)) return HIKONV_ERR_NO_FIT;
         kp.flush_chunks = fc;
     }

@@ -41,19 +41,27 @@ SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int f_sign
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Words per packed kernel row in the 2-D kernels' shared memory, and the cap on channels per stage that
+// keeps one staged weight tile within 32 KB.
+constexpr int kBPitch = 64;
+inline int stage_channel_cap(int K, int J) {
+    const int c = 8192 / (K * J * kBPitch);
+    return c < 1 ? 1 : (c > 8 ? 8 : c);
+}
+
 // 2-D kernels stage CK input channels at a time and move the upper slot bits to the second
 // accumulator every `fc` stages.  Given the number of channels CF that may be accumulated between two
-// such moves, picks CK <= 8 and fc with CK * fc <= CF as large as possible (stages of fewer than
+// such moves, picks CK <= ck_cap and fc with CK * fc <= CF as large as possible (stages of fewer than
 // three channels are avoided when something close is available).  Returns CK * fc.
-inline int pick_chunking(int CF, int Ci, int *CK, int *fc) {
+inline int pick_chunking(int CF, int Ci, int *CK, int *fc, int ck_cap = 8) {
     if (CF >= Ci) {
-        *CK = Ci < 8 ? Ci : 8;
+        *CK = Ci < ck_cap ? Ci : ck_cap;
         *fc = 1 << 30;
         return Ci;
     }
     int best = 0;
     double best_score = -1.0;
-    for (int ck = (CF < 8 ? CF : 8); ck >= 1; --ck) {
+    for (int ck = (CF < ck_cap ? CF : ck_cap); ck >= 1; --ck) {
         const int f = CF / ck, eff = ck * f;
         const double score = ck >= 3 ? eff : 0.7 * eff;
         if (score > best_score) {

@@ -153,7 +153,7 @@ static bool check_candidate(int p, int q, int fs, int gs, int K, int N, int S, b
                 const int Ci = (int)(carry_save_total / K);
                 if (a < K) continue;
                 int ck, fc;
-                const int eff = pick_chunking((int)(a / K), Ci, &ck, &fc);
+                const int eff = pick_chunking((int)(a / K), Ci, &ck, &fc, stage_channel_cap(K, J));
                 if (ceil_div(Ci, eff) > (1LL << h)) continue;
                 a = (long long)eff * K;
             }
