@@ -243,6 +243,9 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
             for (int i = 0; i < TM; ++i) ap[i] = aptr[i] + astage;
             const uint32_t *bp = bptr;
+            // two channels per iteration: the operand loads of the next step then rotate through register
+            // names instead of being copied at the loop edge
+#pragma unroll 2
             for (int cl = 0; cl < ckn; ++cl) {
 #pragma unroll
                 for (int kh = 0; kh < KT; ++kh) {

@@ -2,6 +2,8 @@
 // the CUDA kernels run with.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "hikonv_internal.h"
 
@@ -181,8 +183,8 @@ static bool check_candidate(int p, int q, int fs, int gs, int K, int N, int S, b
     return true;
 }
 
-int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, int row_outputs,
-                const hikonv_tuning_t *tune, hikonv_layout_t *out) {
+static int search_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, int row_outputs,
+                         const hikonv_tuning_t *tune, hikonv_layout_t *out) {
     if (validate_codes(p, q) != HIKONV_OK || K < 1 || K > kMaxK || !out || (dims != 1 && dims != 2))
         return HIKONV_ERR_INVALID_ARG;
     fs = fs ? 1 : 0;
@@ -244,6 +246,48 @@ int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, 
     }
     *out = best;
     return HIKONV_OK;
+}
+
+// The search above costs about a hundred microseconds of host time, as much as a layer takes on the
+// device, and its result depends on its arguments alone: keep the most recent results.
+namespace {
+struct LayoutKey {
+    int v[11];
+    bool operator==(const LayoutKey &o) const { return std::memcmp(v, o.v, sizeof(v)) == 0; }
+};
+struct LayoutEntry {
+    LayoutKey key;
+    int status;
+    hikonv_layout_t layout;
+};
+constexpr size_t kLayoutCacheEntries = 128;
+std::mutex g_layout_mutex;
+std::vector<LayoutEntry> g_layout_cache;
+size_t g_layout_next = 0;
+}  // namespace
+
+int make_layout(int p, int q, int fs, int gs, int K, int dims, int total_terms, int row_outputs,
+                const hikonv_tuning_t *tune, hikonv_layout_t *out) {
+    if (!out) return HIKONV_ERR_INVALID_ARG;
+    LayoutKey key = {{p, q, fs ? 1 : 0, gs ? 1 : 0, K, dims, total_terms, row_outputs, tune ? tune->N : 0,
+                      tune ? tune->S : 0, tune ? tune->M : 0}};
+    {
+        std::lock_guard<std::mutex> lock(g_layout_mutex);
+        for (const LayoutEntry &e : g_layout_cache)
+            if (e.key == key) {
+                *out = e.layout;
+                return e.status;
+            }
+    }
+    LayoutEntry e;
+    e.key = key;
+    std::memset(&e.layout, 0, sizeof(e.layout));
+    e.status = search_layout(p, q, fs, gs, K, dims, total_terms, row_outputs, tune, &e.layout);
+    *out = e.layout;
+    std::lock_guard<std::mutex> lock(g_layout_mutex);
+    if (g_layout_cache.size() < kLayoutCacheEntries) g_layout_cache.push_back(e);
+    else g_layout_cache[g_layout_next++ % kLayoutCacheEntries] = e;
+    return e.status;
 }
 
 // Term counts per product slot for a layout: T[m] = number of code products that land in slot m
