@@ -30,7 +30,11 @@ if ROOT not in sys.path:
 METRIC = "effective low-bit conv MAC/s"
 UNIT = "MAC/s"
 HBM_FALLBACK_GBS = 6650.0            # earlier pool measurement, used only when MEASURED_PEAKS.json is absent
-IMAD_PER_CLK_PER_SM = 64             # 32-bit integer multiply-add lanes per SM per clock (confirmed by microbenchmark)
+# Integer multiply-add lanes per SM per clock, measured with shared-memory-fed operands: the 32-bit
+# multiply-add of the comparator issues on 64 lanes, the 32x32->64 multiply with 64-bit accumulate of
+# the packed kernels on 32.
+IMAD32_PER_CLK_PER_SM = 64
+IMAD_WIDE_PER_CLK_PER_SM = 32
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of each kernel,
 # with the SHA-256 of the kernel source at capture time (a changed source voids the figure).
@@ -202,7 +206,9 @@ def run_ours(args):
     hk.lib()
     hbm_peak_gbs, sm_max_mhz, peak_kind = measured_peaks()
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    imad_peak = sms * IMAD_PER_CLK_PER_SM * sm_max_mhz * 1e6        # multiply-adds per second
+    # multiply-adds per second by kind of multiply
+    imad_peak = {"packed": sms * IMAD_WIDE_PER_CLK_PER_SM * sm_max_mhz * 1e6,
+                 "unpacked": sms * IMAD32_PER_CLK_PER_SM * sm_max_mhz * 1e6}
 
     def barrier():
         if world > 1:
@@ -426,9 +432,12 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
         "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
     }
     if muls is not None:
-        line["roofline"] = {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": imad_peak / 1e12,
-                            "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / imad_peak, "traffic": None,
-                            "kernel": "conv2d_kernel", "peak_kind": "derived: SMs x 64 lanes/clk x max SM clock"}
+        peak = imad_peak[args.algo]
+        line["roofline"] = {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": peak / 1e12,
+                            "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / peak, "traffic": None,
+                            "kernel": "conv2d_kernel",
+                            "peak_kind": "derived: SMs x %d lanes/clk x max SM clock; the step also holds the two packing kernels"
+                                         % (IMAD_WIDE_PER_CLK_PER_SM if args.algo == "packed" else IMAD32_PER_CLK_PER_SM)}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -506,8 +515,8 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
             muls = hk.conv2d_multiplies(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
                                         shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], algo)
             rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT,
-                        "roofline": {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": imad_peak / 1e12,
-                                     "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / imad_peak, "traffic": None}}
+                        "roofline": {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": imad_peak[key] / 1e12,
+                                     "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / imad_peak[key], "traffic": None}}
         rec["layout"] = hk.layout(shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], shape["K"], 2, shape["Ci"] * shape["K"])
         rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
         out[name] = rec

@@ -21,6 +21,8 @@ __host__ __device__ constexpr int gcd_c(int a, int b) { return b == 0 ? a : gcd_
 // blocks per lane: L = R N is a multiple of 4 and at least kMinRun
 constexpr int kMinRun = 24;
 __host__ __device__ constexpr int blocks_per_lane(int N) {
+    // N = 5 and 10 would get runs of 40 outputs, whose registers cost a resident CTA per SM: 20 instead
+    if (N == 5 || N == 10) return 20 / N;
     const int step = 4 / gcd_c(N, 4);
     int r = step;
     while (r * N < kMinRun) r += step;

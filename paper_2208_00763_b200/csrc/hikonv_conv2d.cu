@@ -30,6 +30,7 @@
 #include <algorithm>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "hikonv_cuda.cuh"
 
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     uint32_t *Bs = smem + p.b_off;                         // two tiles [CK*K*J][TCO]
 
     const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int tn = tid % p.TNX, tm = tid / p.TNX;
+    const int tn = tid % p.TNX;
     const int seg = blockIdx.x % p.NSEG;
     const int R0 = (blockIdx.x / p.NSEG) * p.TR;
     const int co0 = blockIdx.y * p.TCO;
@@ -114,11 +115,17 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     const int TP = TRe * p.XB;                              // positions of this tile
     const int S = SC > 0 ? SC : p.S;
 
+    // A warp owns 32 / TNX * TM consecutive positions, dealt round-robin to its 32 / TNX position lanes:
+    // the lanes of one operand load then read consecutive words (no bank conflicts), and the block in
+    // front of a lane's position sits in the lane before it.
+    const int lane = tid & 31, warp = tid >> 5;
+    const int lanes_m = 32 / p.TNX, lm = lane / p.TNX;
+    const int wpos0 = warp * lanes_m * TM;
     // this thread's positions: shared-memory address of the packed word for (ci = 0, kh = 0, j = 0)
     const uint32_t *aptr[TM];
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
-        const int pos = tm * TM + i;
+        const int pos = wpos0 + i * lanes_m + lm;
         int off = p.lead;                                    // idle position: reads valid memory, result dropped
         if (pos < TP) {
             const int r = pos / p.XB, xb = pos - r * p.XB;
@@ -296,76 +303,107 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
 
     // ---- extract the slots: slot m holds 2^h E_m + Q_m - (moves + 1) bias_m (uint32 arithmetic wraps by design)
-    const uint32_t nb = (uint32_t)nmoves + 1u;
+    uint32_t slot_sub[2 * N], slot_msk[2 * N];                        // per slot: (moves + 1) bias_m and the field mask
+#pragma unroll
+    for (int m = 0; m < 2 * N; ++m) {
+        slot_sub[m] = ((uint32_t)nmoves + 1u) * (uint32_t)p.slot_bias[m];
+        slot_msk[m] = (m == p.nslots - 1) ? p.top_mask : p.slot_mask;
+    }
     auto slot_value = [&](uint64_t Q, uint64_t Ev, int m) -> uint32_t {
-        const uint32_t msk = (m == p.nslots - 1) ? p.top_mask : p.slot_mask;
-        const uint32_t qv = (uint32_t)(Q >> (S * m)) & msk;
-        const uint32_t ev = (uint32_t)(Ev >> (S * m)) & msk;
-        return (ev << p.hbits) + qv - nb * (uint32_t)p.slot_bias[m];
+        const uint32_t qv = (uint32_t)(Q >> (S * m)) & slot_msk[m];
+        const uint32_t ev = (uint32_t)(Ev >> (S * m)) & slot_msk[m];
+        return (ev << p.hbits) + qv - slot_sub[m];
     };
     auto load_e = [&](int i, int t) -> uint64_t {
         const uint2 e = Es[(i * TN + t) * kMaxThreads2D];
         return ((uint64_t)e.y << 32) | e.x;
     };
-    // the upper slots of a thread's last position belong to the next thread's first position (Theorem 2)
+    // The upper slots of a position belong to the next position (Theorem 2), which the next lane holds:
+    // they travel by a rotating shuffle, in which the last lane hands over those of its previous
+    // position; a warp's first position takes them from the warp before through shared memory.
     if constexpr (!UNPACKED) {
         __syncthreads();
-        uint32_t *xch = smem;                                        // [TMX][N][TCO]
+        uint32_t *xch = smem;                                        // [warp][N][TCO]
+        if (lm == lanes_m - 1) {
 #pragma unroll
-        for (int m = 0; m < N; ++m)
+            for (int m = 0; m < N; ++m)
 #pragma unroll
-            for (int t = 0; t < TN; ++t)
-                xch[(tm * N + m) * p.TCO + tn * TN + t] =
-                    (N + m < p.nslots) ? slot_value((uint64_t)acc[TM - 1][t], load_e(TM - 1, t), N + m) : 0u;
+                for (int t = 0; t < TN; ++t)
+                    xch[(warp * N + m) * p.TCO + tn * TN + t] =
+                        (N + m < p.nslots) ? slot_value((uint64_t)acc[TM - 1][t], load_e(TM - 1, t), N + m) : 0u;
+        }
         __syncthreads();
     }
 
-    // ---- overlap-add, optional requantisation (arithmetic shift, clamp), store
+    // where each position's pixels go (channel 0): element offset and number of pixels to store (0: none)
+    size_t pix_off[TM];
+    int pix_n[TM];
 #pragma unroll
-    for (int t = 0; t < TN; ++t) {
-        const int co = co0 + tn * TN + t;
-        uint32_t upper[N];                                           // upper slots of the previous position
-        if constexpr (!UNPACKED) {
-#pragma unroll
-            for (int m = 0; m < N; ++m) upper[m] = (tm > 0) ? smem[((tm - 1) * N + m) * p.TCO + tn * TN + t] : 0u;
-        }
-#pragma unroll
-        for (int i = 0; i < TM; ++i) {
-            uint32_t Y[N];
-            if constexpr (!UNPACKED) {
-                const uint64_t ev = load_e(i, t);
-#pragma unroll
-                for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], ev, m) + upper[m];
-#pragma unroll
-                for (int m = 0; m < N; ++m)
-                    upper[m] = (N + m < p.nslots) ? slot_value((uint64_t)acc[i][t], ev, N + m) : 0u;
-            } else {
-                Y[0] = (uint32_t)acc[i][t];
-            }
-            const int pos = tm * TM + i;
-            if (pos >= TP || co >= p.Co) continue;
+    for (int i = 0; i < TM; ++i) {
+        const int pos = wpos0 + i * lanes_m + lm;
+        pix_off[i] = 0;
+        pix_n[i] = 0;
+        if (pos < TP) {
             const int r = pos / p.XB, xbl = pos - r * p.XB;
-            if (xbl < p.J) continue;                                 // halo positions produce no pixels
-            const int xg = seg * p.XO + xbl - p.J;                   // output block in the row
-            if (xg >= p.X) continue;
-            const int R = R0 + r;
-            const int b = R / p.Ho, h = R - b * p.Ho;
-            const size_t row_off = (((size_t)b * p.Co + co) * p.Ho + h) * p.Wo;
-#pragma unroll
-            for (int m = 0; m < N; ++m) {
-                const int w = xg * N + m;
-                if (w >= p.Wo) continue;
-                int32_t v = (int32_t)Y[m];
-                if (p.requant) {
-                    v >>= p.shift;
-                    v = max(p.lo, min(p.hi, v));
-                    ((int8_t *)p.out)[row_off + w] = (int8_t)v;
-                } else {
-                    ((int32_t *)p.out)[row_off + w] = v;
-                }
+            const int xg = seg * p.XO + xbl - p.J;                   // output block in the row; halo positions give no pixels
+            if (xbl >= p.J && xg < p.X) {
+                const int R = R0 + r;
+                const int b = R / p.Ho, h = R - b * p.Ho;
+                pix_off[i] = (((size_t)b * p.Co) * p.Ho + h) * p.Wo + (size_t)xg * N;
+                pix_n[i] = min(N, p.Wo - xg * N);
             }
         }
     }
+    const size_t chan_stride = (size_t)p.Ho * p.Wo;
+
+    // ---- overlap-add, optional requantisation (arithmetic shift, clamp), store
+    auto finish = [&](auto requant_tag) {
+        constexpr bool REQ = decltype(requant_tag)::value;
+#pragma unroll
+        for (int t = 0; t < TN; ++t) {
+            const int co = co0 + tn * TN + t;
+            const size_t chan_off = (size_t)co * chan_stride;
+            uint32_t up_prev[N];                                     // upper slots of this lane's previous position
+#pragma unroll
+            for (int m = 0; m < N; ++m) up_prev[m] = 0u;
+#pragma unroll
+            for (int i = 0; i < TM; ++i) {
+                uint32_t Y[N];
+                if constexpr (!UNPACKED) {
+                    const uint64_t ev = load_e(i, t);
+#pragma unroll
+                    for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], ev, m);
+#pragma unroll
+                    for (int m = 0; m < N; ++m) {
+                        if (N + m < p.nslots) {                      // uniform over the launch
+                            const uint32_t up = slot_value((uint64_t)acc[i][t], ev, N + m);
+                            uint32_t in = __shfl_sync(0xFFFFFFFFu, lm == lanes_m - 1 ? up_prev[m] : up, (lane - p.TNX) & 31);
+                            if (i == 0 && lm == 0) in = warp > 0 ? smem[((warp - 1) * N + m) * p.TCO + tn * TN + t] : 0u;
+                            Y[m] += in;
+                            up_prev[m] = up;
+                        }
+                    }
+                } else {
+                    Y[0] = (uint32_t)acc[i][t];
+                }
+                if (co >= p.Co) continue;
+                const size_t o = pix_off[i] + chan_off;
+#pragma unroll
+                for (int m = 0; m < N; ++m) {
+                    if (m >= pix_n[i]) continue;
+                    int32_t v = (int32_t)Y[m];
+                    if constexpr (REQ) {
+                        v = max(p.lo, min(p.hi, v >> p.shift));
+                        ((int8_t *)p.out)[o + m] = (int8_t)v;
+                    } else {
+                        ((int32_t *)p.out)[o + m] = v;
+                    }
+                }
+            }
+        }
+    };
+    if (p.requant) finish(std::true_type());
+    else finish(std::false_type());
 }
 
 // Packed activation rows (Eq. 5): ap[(ci * B*Hp + b*Hp + hp) * XBT + xb] packs the N input pixels of block
