@@ -409,27 +409,32 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 // Packed activation rows (Eq. 5): ap[(ci * B*Hp + b*Hp + hp) * XBT + xb] packs the N input pixels of block
 // x = xb - J of padded row hp, i.e. columns (xb - J) N + K - 1 - pad + n of input row hp - pad, zero where the
 // row or a column lies in the padding.  For the comparator S == 0 and N == 1: one int32 code per word.
-template <bool XS>
+// One thread packs four consecutive words of a row (one 16-byte store); a CTA stays within one
+// (ci, b) plane, whose rows are contiguous in both the input and the packed layout.
+template <bool XS, int N>
 __global__ void __launch_bounds__(256) pack_activations_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
-                                                               int pad, int K, int J, int N, int S, int XBT,
-                                                               uint32_t *__restrict__ ap, size_t total) {
-    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= total) return;
-    const int xb = (int)(idx % XBT);
-    const size_t rest = idx / XBT;
-    const int rp = (int)(rest % ((size_t)B * Hp));
-    const int ci = (int)(rest / ((size_t)B * Hp));
-    const int b = rp / Hp, hi = rp - b * Hp - pad;
-    uint32_t word = 0;
+                                                               int pad, int K, int J, int S, int XBT, int blocks_per_plane,
+                                                               uint32_t *__restrict__ ap) {
+    const int plane = blockIdx.x / blocks_per_plane;                 // ci * B + b
+    const int piece = (blockIdx.x - plane * blocks_per_plane) * 256 + threadIdx.x;
+    const int xq = XBT / 4;                                          // 16-byte pieces per packed row
+    if (piece >= Hp * xq) return;
+    const int ci = plane / B, b = plane - ci * B;
+    const int hp = piece / xq, q = piece - hp * xq;
+    const int hi = hp - pad;
+    uint32_t word[4] = {0u, 0u, 0u, 0u};
     if (hi >= 0 && hi < H) {
         const int8_t *row = x + (((size_t)b * Ci + ci) * H + hi) * W;
-        const int col0 = (xb - J) * N + K - 1 - pad;
-        for (int n = 0; n < N; ++n) {
-            const int col = col0 + n;
-            if (col >= 0 && col < W) word += (uint32_t)load_code<XS>(row + col) << (S * n);
-        }
+        const int col0 = (4 * q - J) * N + K - 1 - pad;              // input column of slot 0 of the first word
+#pragma unroll
+        for (int w = 0; w < 4; ++w)
+#pragma unroll
+            for (int n = 0; n < N; ++n) {
+                const int col = col0 + w * N + n;
+                if (col >= 0 && col < W) word[w] += (uint32_t)load_code<XS>(row + col) << (S * n);
+            }
     }
-    ap[idx] = word;
+    *reinterpret_cast<uint4 *>(ap + ((size_t)plane * Hp + hp) * XBT + 4 * q) = make_uint4(word[0], word[1], word[2], word[3]);
 }
 
 // Reversed, packed kernel rows (Theorem 3: g = W[co][ci][kh][K-1:0], then Eq. 5 per chunk of Kc taps).
@@ -458,6 +463,28 @@ __global__ void __launch_bounds__(256) pack_weights_kernel(const int8_t *__restr
         }
     }
     wp[idx] = word;
+}
+
+// Eight input columns of two rows per thread (two 8-byte loads, per-byte maxima, one 4-byte store);
+// needs W % 8 == 0 and 8-byte aligned tensors.
+template <bool SIGNED>
+__global__ void __launch_bounds__(256) maxpool2x2_vec_kernel(const int8_t *__restrict__ in, long long items, int H, int W,
+                                                             int8_t *__restrict__ out) {
+    const int Ho = H / 2, W8 = W / 8;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < items; idx += (long long)gridDim.x * blockDim.x) {
+        const int w8 = (int)(idx % W8);
+        const long long rest = idx / W8;
+        const int ho = (int)(rest % Ho);
+        const long long c = rest / Ho;
+        const int8_t *src = in + (c * H + 2 * ho) * (long long)W + 8 * w8;
+        const uint2 r0 = __ldg(reinterpret_cast<const uint2 *>(src));
+        const uint2 r1 = __ldg(reinterpret_cast<const uint2 *>(src + W));
+        uint32_t v0 = SIGNED ? __vmaxs4(r0.x, r1.x) : __vmaxu4(r0.x, r1.x);
+        uint32_t v1 = SIGNED ? __vmaxs4(r0.y, r1.y) : __vmaxu4(r0.y, r1.y);
+        v0 = SIGNED ? __vmaxs4(v0, v0 >> 8) : __vmaxu4(v0, v0 >> 8);             // bytes 0 and 2 hold the pair maxima
+        v1 = SIGNED ? __vmaxs4(v1, v1 >> 8) : __vmaxu4(v1, v1 >> 8);
+        *reinterpret_cast<uint32_t *>(out + (c * Ho + ho) * (long long)(W / 2) + 4 * w8) = __byte_perm(v0, v1, 0x6420);
+    }
 }
 
 __global__ void __launch_bounds__(256) maxpool2x2_kernel(const int8_t *__restrict__ in, int BC, int H, int W, int is_signed,
@@ -748,14 +775,25 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
                                                                d_wp, total_w);
     rc = launch_status();
     if (rc != HIKONV_OK) return rc;
-    const size_t blocks_a = (s.ap_words + 255) / 256;
-    if (blocks_a > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
-    if (x_signed)
-        pack_activations_kernel<true><<<(unsigned)blocks_a, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.N, s.L.S,
-                                                                         s.kp.XBT, d_ap, s.ap_words);
-    else
-        pack_activations_kernel<false><<<(unsigned)blocks_a, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.N, s.L.S,
-                                                                          s.kp.XBT, d_ap, s.ap_words);
+    {
+        const int bpp = ceil_div(s.kp.Hp * (s.kp.XBT / 4), 256);
+        if ((size_t)Ci * B * bpp > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
+        const unsigned grid = (unsigned)((size_t)Ci * B * bpp);
+#define HK_PACK(XSIGN, NN)                                                                                                   \
+    pack_activations_kernel<XSIGN, NN><<<grid, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.S, s.kp.XBT, bpp, d_ap)
+        switch (s.L.N * 2 + (x_signed ? 1 : 0)) {
+            case 2: HK_PACK(false, 1); break;
+            case 3: HK_PACK(true, 1); break;
+            case 4: HK_PACK(false, 2); break;
+            case 5: HK_PACK(true, 2); break;
+            case 6: HK_PACK(false, 3); break;
+            case 7: HK_PACK(true, 3); break;
+            case 8: HK_PACK(false, 4); break;
+            case 9: HK_PACK(true, 4); break;
+            default: return HIKONV_ERR_UNSUPPORTED;
+        }
+#undef HK_PACK
+    }
     rc = launch_status();
     if (rc != HIKONV_OK) return rc;
     return launch_conv2d(s, st);
@@ -839,8 +877,15 @@ extern "C" int hikonv_maxpool2x2_i8(const int8_t *d_in, int B, int C, int H, int
     const long long total = (long long)B * C * (H / 2) * (W / 2);
     if (total == 0) return HIKONV_OK;
     if ((double)B * C >= 2147483647.0) return HIKONV_ERR_UNSUPPORTED;
-    long long blocks = (total + 255) / 256;
     const long long cap = (long long)sm_count() * 32;
+    if (W % 8 == 0 && ((uintptr_t)d_in % 8) == 0 && ((uintptr_t)d_out % 4) == 0) {
+        const long long items = total / 4;
+        const unsigned grid = (unsigned)std::min((items + 255) / 256, cap);
+        if (is_signed) maxpool2x2_vec_kernel<true><<<grid, 256, 0, (cudaStream_t)stream>>>(d_in, items, H, W, d_out);
+        else maxpool2x2_vec_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>(d_in, items, H, W, d_out);
+        return launch_status();
+    }
+    long long blocks = (total + 255) / 256;
     if (blocks > cap) blocks = cap;
     maxpool2x2_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(d_in, B * C, H, W, is_signed ? 1 : 0, d_out);
     return launch_status();
