@@ -144,7 +144,7 @@ def cpu_baseline(sample_len: int):
     data = oracle_inputs(sample_len)
     oracle_sweep(data[:2])
     macs, secs, passes = 0.0, 0.0, 0
-    while secs < 10.0 and passes < 50:
+    while secs < 10.0 and passes < 400:
         m, s = oracle_sweep(data)
         macs += m
         secs += s
@@ -155,9 +155,9 @@ def cpu_baseline(sample_len: int):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return 0
+    from paper_2208_00763_b200 import ranks
+    if ranks.rank_info()[1] != 0:
+        return 0                      # the oracle runs once, on rank 0's host cores
     from oracle import direct
     sample_len = 1 << 22
     data = oracle_inputs(sample_len)
@@ -189,20 +189,16 @@ def run_reference(args):
 def run_ours(args):
     import numpy as np
     import torch
-    import torch.distributed as dist
 
     from paper_2208_00763_b200 import binding as hk
-    from paper_2208_00763_b200 import inputs, network
+    from paper_2208_00763_b200 import inputs, network, ranks
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = ranks.rank_info()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    ranks.init("nccl", dev)
     hk.lib()
     hbm_peak_gbs, sm_max_mhz, peak_kind = measured_peaks()
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -211,20 +207,15 @@ def run_ours(args):
                  "unpacked": sms * IMAD32_PER_CLK_PER_SM * sm_max_mhz * 1e6}
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
     def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return ranks.max_over_ranks(ms, dev)
 
     # ---- the sweep: every rank runs the whole sweep on its own data (weak scaling, no exchange)
     if args.workload != "c2":
-        return run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks,
+        return run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks,
                               imad_peak)
     length = args.length
     cases = inputs.c2_cases(length)
@@ -237,7 +228,7 @@ def run_ours(args):
     host_f, host_g = [], []
     for case in cases:
         f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"],
-                                  case["seed"] + 100000 * rank)
+                                  ranks.rank_seed(case["seed"], rank))
         host_f.append(torch.from_numpy(inputs.to_storage(f)))
         host_g.append(torch.from_numpy(inputs.to_storage(g)))
     d_f = [t.to(dev) for t in host_f]
@@ -276,7 +267,7 @@ def run_ours(args):
     total_ms = max_over_ranks(timed_graph(lambda: sweep(hk.ALGO_PACKED32), args.steps, args.warmup))
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step = total_ms / args.steps
-    value = world * macs_per_step / (ms_per_step * 1e-3)
+    value = ranks.whole_job_rate(macs_per_step, args.steps, total_ms, world)
     launches_per_step = len(cases)
 
     # roofline of the dominant kernel (conv1d_packed): 1 input byte + 4 output bytes per output
@@ -347,12 +338,11 @@ def run_ours(args):
 
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.shutdown()
     return 0
 
 
-def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks, imad_peak):
+def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks, imad_peak):
     """Main line for --workload c3/c4/c5: a step is one layer (or one network pass) on this rank's batch,
     timed with one event pair per step and an L2 flush (256 MB memset) before each step."""
     algo = hk.ALGO_PACKED32 if args.algo == "packed" else hk.ALGO_UNPACKED_IMAD
@@ -362,7 +352,7 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
         shape = dict(inputs.C3_SHAPE if args.workload == "c3" else inputs.C4_SHAPE)
         if args.batch:
             shape["B"] = args.batch
-        shape["seed"] = shape["seed"] + 1000 * rank
+        shape["seed"] = ranks.rank_seed(shape["seed"], rank)
         x, w = inputs.layer_case(shape)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         d_w = torch.from_numpy(inputs.to_storage(w)).to(dev)
@@ -386,7 +376,7 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
         h2d = d_x.numel() + d_w.numel()
         d2h = o.numel() * o.element_size()
     else:
-        x, layers, head_w = inputs.c5_network(seed=5 + 1000 * rank, batch=args.batch or 64)
+        x, layers, head_w = inputs.c5_network(seed=ranks.rank_seed(5, rank), batch=args.batch or 64)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         net = network.CompactCnn(layers, head_w, device=dev)
         macs, muls = 0.0, None
@@ -425,7 +415,8 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
     clocks = sampler.stop() if rank == 0 else None
     ms = total / args.steps
     line = {
-        "metric": METRIC, "value": world * macs / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": ranks.whole_job_rate(macs, args.steps, total, world), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int64" if args.algo == "packed" else "int32", "data": "synthetic",
         "config": {"workload": name, "algo": args.algo, "l2": "flushed before every step (256 MB memset outside the timed events)"},
@@ -440,8 +431,7 @@ def run_layer_main(args, torch, np, dist, hk, inputs, network, dev, world, rank,
                                          % (IMAD_WIDE_PER_CLK_PER_SM if args.algo == "packed" else IMAD32_PER_CLK_PER_SM)}
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.shutdown()
     return 0
 
 
