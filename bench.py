@@ -36,10 +36,13 @@ HBM_FALLBACK_GBS = 6650.0            # earlier pool measurement, used only when 
 IMAD32_PER_CLK_PER_SM = 64
 IMAD_WIDE_PER_CLK_PER_SM = 32
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of each kernel,
-# with the SHA-256 of the kernel source at capture time (a changed source voids the figure).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of the kernel (two
+# launches of the p=q=4, K=3 signed case at 2^24: 16.80 MB read both times, 8.72 and 10.50 MB written
+# before the counters stopped; the rest of the 67 MB output was still in the 126 MB L2), with the
+# SHA-256 of the kernel source at capture time (a changed source voids the figure).
 NCU_TRAFFIC = {
-    # "conv1d_packed": {"sha256": "...", "bytes_per_output": ...},
+    "conv1d_packed_tc": {"sha256": "0d566a8170af2d0606f8887523e085ba80561dce764aabc32ca358adee0df766",
+                         "bytes_per_output": (16.803e6 + 9.613e6) / 16777218.0},
 }
 
 
@@ -275,12 +278,14 @@ def run_ours(args):
     bytes_per_launch = 5.0 * outputs_per_step / launches_per_step
     achieved_gbs = bytes_per_launch / avg_launch_s / 1e9
     traffic = None
-    rec = NCU_TRAFFIC.get("conv1d_packed")
-    if rec and rec.get("sha256") == _source_hash("hikonv_conv1d.cu"):
+    rec = NCU_TRAFFIC.get("conv1d_packed_tc")
+    if rec and rec.get("sha256") == _source_hash("hikonv_conv1d_tc.cu"):
         traffic = rec["bytes_per_output"] * outputs_per_step / launches_per_step
     roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": hbm_peak_gbs, "unit": "GB/s",
                 "frac": achieved_gbs / hbm_peak_gbs, "traffic": traffic, "peak_kind": "of " + peak_kind,
-                "kernel": "conv1d_packed_kernel", "bytes_per_output": 5}
+                "kernel": "conv1d_packed_tc_kernel", "bytes_per_output": 5,
+                "traffic_note": "DRAM bytes of one launch under ncu; below the algorithmic bytes because most of a launch's "
+                                "output is still in L2 when its counters stop"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),

@@ -15,8 +15,9 @@
 // kernel streams both with 16-byte asynchronous copies into double-buffered shared memory.
 //
 // A CTA computes TR consecutive output rows (one row segment each) times TCO output channels; it
-// is a register-tiled integer "GEMM" over packed words: each thread owns TM consecutive positions
-// times TN channels, the k dimension runs over (ci, kh, j).
+// is a register-tiled integer "GEMM" over packed words: each thread owns TM positions times TN
+// channels (a warp's consecutive positions are dealt round-robin to its lanes), the k dimension runs
+// over (ci, kh, j).
 //
 // Split.  Every slot starts at a bias that makes its running sum non-negative, so slots never borrow
 // from each other (this replaces the sign-borrow increment of Eq. 29).  After at most M accumulated
