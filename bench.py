@@ -141,6 +141,11 @@ def oracle_sweep(data):
     return macs, time.perf_counter() - t0
 
 
+def inputs_mod():
+    from paper_2208_00763_b200 import inputs
+    return inputs
+
+
 def cpu_baseline(sample_len: int):
     """The oracle as it stands on the host cores: the 48 sweep cases at `sample_len`, repeated for about 10 s."""
     from oracle import direct
@@ -152,7 +157,37 @@ def cpu_baseline(sample_len: int):
         macs += m
         secs += s
         passes += 1
-    return {"value": macs / secs, "unit": UNIT, "cores": direct.num_threads(), "kind": "oracle",
+    layers = {}
+    for name, shape, batch in (("c3", inputs_mod().C3_SHAPE, 2), ("c4", inputs_mod().C4_SHAPE, 2)):
+        x, w = inputs_mod().layer_case(shape, batch=batch)
+        t0 = time.perf_counter()
+        direct.conv2d_nchw(x, w, shape["pad"])
+        dt = time.perf_counter() - t0
+        Ho = shape["H"] + 2 * shape["pad"] - shape["K"] + 1
+        lm = float(batch) * shape["Co"] * Ho * Ho * shape["Ci"] * shape["K"] ** 2
+        layers[name] = {"value": lm / dt, "unit": UNIT, "sample": "%d of %d images, %.2f s" % (batch, shape["B"], dt)}
+    # the paper's own CPU experiment on this host: its packed loop (Algorithm 2) beside the plain loops,
+    # one thread, K = 3, where the kernel fits one 32-bit word
+    from oracle import algorithm2
+    alg2 = {}
+    rng_len = 1 << 22
+    threads_before = direct.num_threads()
+    direct.set_num_threads(1)
+    for bits in (1, 2, 4):
+        for signed in (False, True):
+            if algorithm2.layout(bits, bits, 3, signed) is None:
+                continue
+            f, g = inputs_mod().conv1d_case(rng_len, 3, bits, bits, signed, signed, 7000 + 10 * bits + int(signed))
+            t0 = time.perf_counter()
+            direct.conv1d_full(f, g)
+            t1 = time.perf_counter()
+            algorithm2.conv1d_full(f, g, bits, bits, signed, 1)
+            t2 = time.perf_counter()
+            alg2["p%d_%s" % (bits, "s" if signed else "u")] = {"plain_ms": 1e3 * (t1 - t0), "packed_ms": 1e3 * (t2 - t1),
+                                                             "speedup": (t1 - t0) / (t2 - t1)}
+    direct.set_num_threads(threads_before)
+    return {"value": macs / secs, "unit": UNIT, "cores": direct.num_threads(), "kind": "oracle", "layers": layers,
+            "algorithm2_one_thread": alg2,
             "sample": "%d pass(es) over the 48 sweep cases at signal length %d (benchmark length 2^24), int64 direct "
                       "convolution, OpenMP over outputs, %.1f s of CPU time" % (passes, sample_len, secs)}
 
@@ -334,6 +369,7 @@ def run_ours(args):
             extra["c2_unpacked"] = {"value": macs_per_step / (un_ms * 1e-3), "unit": UNIT, "ms_per_step": un_ms,
                                     "hbm_frac": 5.0 * outputs_per_step / (un_ms * 1e-3) / 1e9 / hbm_peak_gbs}
             del d_y
+            extra["c1"] = small_case(torch, hk, inputs, dev)
             extra["c2_by_bits"] = per_bitwidth_table(torch, hk, cases, d_f, d_g, length)
             del d_f, d_g
             torch.cuda.empty_cache()
@@ -438,6 +474,36 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         print(json.dumps(line), flush=True)
     ranks.shutdown()
     return 0
+
+
+def small_case(torch, hk, inputs, dev):
+    """C1 (4096 codes, K = 3, unsigned 4-bit): microseconds per launch inside a graph of 100 launches.  At this
+    size the launch itself is the cost; the case is there for parity, not for throughput."""
+    f, g = inputs.c1()
+    d_f = torch.from_numpy(inputs.to_storage(f)).to(dev)
+    d_g = torch.from_numpy(inputs.to_storage(g)).to(dev)
+    y = torch.empty(f.size + g.size - 1, dtype=torch.int32, device=dev)
+    row = {}
+    for name, algo in (("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD)):
+        def fn():
+            for _ in range(100):
+                hk.conv1d(d_f, d_g, 4, 4, False, False, algo=algo, out=y)
+        fn()
+        torch.cuda.synchronize()
+        g_ = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_):
+            fn()
+        g_.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(5):
+            g_.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        row[name] = e0.elapsed_time(e1) * 1e3 / 500
+    row["macs"] = float(y.numel()) * g.size
+    return row
 
 
 def per_bitwidth_table(torch, hk, cases, d_f, d_g, length):
