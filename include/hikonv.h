@@ -84,7 +84,9 @@ typedef struct {
     int N;          /* force activations per word                                   */
     int S;          /* force slot width                                             */
     int M;          /* force the number of accumulated products between two splits  */
-    int tile;       /* kernel-specific tile selector (0 = automatic)                */
+    int tile;       /* kernel-specific tile selector (0 = automatic); conv2d: > 0 output
+                       rows per CTA, < 0 carry-save moves at stage ends instead of at
+                       fixed places inside channel groups; conv1d: > 0 the general kernel */
 } hikonv_tuning_t;
 
 /*

@@ -60,6 +60,7 @@ struct Conv2dParams {
     int requant, shift, lo, hi;
     int total_rows;            // B * Ho
     int flush_chunks;          // channel stages accumulated between two carry-save moves (CK * K * flush_chunks <= M)
+    int move_every;            // > 0: every accumulator row moves once per this many channels, at a fixed place of an unrolled group (CK a multiple of it)
     int hbits, nslots;         // carry-save: low bits kept per slot; number of slots N + Kc - 1
     uint64_t bias, mask_low, mask_high;
     uint32_t slot_mask, top_mask;
@@ -95,7 +96,10 @@ __device__ __forceinline__ void mac(typename AccType<UNPACKED>::type &acc, uint3
 // parameters; the (kh, j) loops are then not unrolled);
 // PITCH: words per activation row in shared memory when known at compile time (then every operand load
 // of the unrolled loops has an immediate offset), 0: read from the parameters.
-template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, int KT, int JT, int PITCH>
+// U > 0: the channel loop runs in unrolled groups of U channels in which accumulator row i does its
+// carry-save move after channel (i U) / TM of the group, so that the moves of different rows sit between
+// the multiplies of the others instead of forming one burst per stage (channels past Ci carry zero weights).
+template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, int KT, int JT, int PITCH, int U>
 __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dParams p) {
     typedef typename AccType<UNPACKED>::type acc_t;
     extern __shared__ __align__(16) uint32_t smem[];
@@ -154,29 +158,31 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 
     // move the upper bits of every slot to E and restart the slots at their bias (on 32-bit halves, so
     // that it is two funnel/plain shifts, four logic operations and one add with carry per accumulator)
-    auto carry_save = [&]() {
+    auto carry_save_row = [&](int i) {
         if constexpr (!UNPACKED) {
             const uint32_t mh_lo = (uint32_t)p.mask_high, mh_hi = (uint32_t)(p.mask_high >> 32);
             const uint32_t ml_lo = (uint32_t)p.mask_low, ml_hi = (uint32_t)(p.mask_low >> 32);
             const uint32_t b_lo = (uint32_t)p.bias, b_hi = (uint32_t)(p.bias >> 32);
             const int h = p.hbits;                                   // 1 .. 31 whenever a move happens
 #pragma unroll
-            for (int i = 0; i < TM; ++i)
-#pragma unroll
-                for (int t = 0; t < TN; ++t) {
-                    uint32_t qlo = (uint32_t)acc[i][t], qhi = (uint32_t)((uint64_t)acc[i][t] >> 32);
-                    uint2 e = Es[(i * TN + t) * kMaxThreads2D];
-                    uint32_t elo = e.x, ehi = e.y;
-                    const uint32_t hlo = __funnelshift_r(qlo, qhi, h) & mh_lo;
-                    const uint32_t hhi = (qhi >> h) & mh_hi;
-                    asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(elo), "+r"(ehi) : "r"(hlo), "r"(hhi));
-                    qlo = (qlo & ml_lo) | b_lo;
-                    qhi = (qhi & ml_hi) | b_hi;
-                    Es[(i * TN + t) * kMaxThreads2D] = make_uint2(elo, ehi);
-                    acc[i][t] = (acc_t)(((uint64_t)qhi << 32) | qlo);
-                }
-            ++nmoves;
+            for (int t = 0; t < TN; ++t) {
+                uint32_t qlo = (uint32_t)acc[i][t], qhi = (uint32_t)((uint64_t)acc[i][t] >> 32);
+                uint2 e = Es[(i * TN + t) * kMaxThreads2D];
+                uint32_t elo = e.x, ehi = e.y;
+                const uint32_t hlo = __funnelshift_r(qlo, qhi, h) & mh_lo;
+                const uint32_t hhi = (qhi >> h) & mh_hi;
+                asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(elo), "+r"(ehi) : "r"(hlo), "r"(hhi));
+                qlo = (qlo & ml_lo) | b_lo;
+                qhi = (qhi & ml_hi) | b_hi;
+                Es[(i * TN + t) * kMaxThreads2D] = make_uint2(elo, ehi);
+                acc[i][t] = (acc_t)(((uint64_t)qhi << 32) | qlo);
+            }
         }
+    };
+    auto carry_save = [&]() {
+#pragma unroll
+        for (int i = 0; i < TM; ++i) carry_save_row(i);
+        ++nmoves;
     };
 
     const int KJ = p.K * p.J;
@@ -226,10 +232,11 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             }
         }
         const uint32_t *bsrc = p.wp + (size_t)ci0 * KJ * p.CoP + co0;
-        for (int idx = tid; idx < (ckn * KJ) << tco4_log2; idx += nthreads) {
+        const int rows_b = (U > 0 ? p.CK : ckn) * KJ;                // grouped mode multiplies all CK channels of a stage
+        for (int idx = tid; idx < rows_b << tco4_log2; idx += nthreads) {
             const int kr = idx >> tco4_log2, c4 = idx & (tco4 - 1);
             uint32_t *dst = Bdst + kr * kBPitch + c4 * 4;
-            if (co0 + c4 * 4 < p.CoP) cp_async_16(dst, bsrc + kr * p.CoP + c4 * 4);
+            if (co0 + c4 * 4 < p.CoP && kr < ckn * KJ) cp_async_16(dst, bsrc + kr * p.CoP + c4 * 4);
             else *reinterpret_cast<uint4 *>(dst) = make_uint4(0, 0, 0, 0);
         }
         cp_async_commit();
@@ -251,6 +258,38 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
             for (int i = 0; i < TM; ++i) ap[i] = aptr[i] + astage;
             const uint32_t *bp = bptr;
+            if constexpr (U > 0 && !UNPACKED) {
+                for (int c0 = 0; c0 < p.CK; c0 += U) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+#pragma unroll
+                        for (int kh = 0; kh < KT; ++kh) {
+#pragma unroll
+                            for (int j = 0; j < JT; ++j) {
+                                uint32_t a[TM], b[TN];
+#pragma unroll
+                                for (int i = 0; i < TM; ++i) a[i] = ap[i][kh * PITCH - j];
+#pragma unroll
+                                for (int t = 0; t < TN; t += 4) {
+                                    const uint4 v = *reinterpret_cast<const uint4 *>(bp + (kh * JT + j) * kBPitch + t);
+                                    b[t] = v.x; b[t + 1] = v.y; b[t + 2] = v.z; b[t + 3] = v.w;
+                                }
+#pragma unroll
+                                for (int i = 0; i < TM; ++i)
+#pragma unroll
+                                    for (int t = 0; t < TN; ++t) mac<UNPACKED, SP>(acc[i][t], a[i], b[t]);
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < TM; ++i) ap[i] += p.a_plane;
+                        bp += KT * JT * kBPitch;
+#pragma unroll
+                        for (int i = 0; i < TM; ++i)
+                            if ((i * U) / TM == u) carry_save_row(i);
+                    }
+                    ++nmoves;
+                }
+            } else {
             // two channels per iteration: the operand loads of the next step then rotate through register
             // names instead of being copied at the loop edge
 #pragma unroll 2
@@ -276,6 +315,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
                 for (int i = 0; i < TM; ++i) ap[i] += p.a_plane;
                 bp += KT * JT * kBPitch;
+            }
             }
         } else {
             for (int cl = 0; cl < ckn; ++cl) {
@@ -526,11 +566,11 @@ static int sm_count() {
     return sms;
 }
 
-template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, int PITCH>
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, int PITCH, int U>
 static int launch_pitch(const Conv2dSetup &s, bool sp, cudaStream_t st) {
 #define HK_LAUNCH(SPV)                                                                                           \
     do {                                                                                                         \
-        auto kern = conv2d_kernel<N, SC, TM, TN, UNPACKED, SPV, KT, JT, PITCH>;                                  \
+        auto kern = conv2d_kernel<N, SC, TM, TN, UNPACKED, SPV, KT, JT, PITCH, U>;                               \
         if (s.smem_bytes > 48 * 1024)                                                                            \
             HIKONV_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem_bytes)); \
         kern<<<s.grid, s.threads, s.smem_bytes, st>>>(s.kp);                                                     \
@@ -542,16 +582,27 @@ static int launch_pitch(const Conv2dSetup &s, bool sp, cudaStream_t st) {
 }
 
 // KT > 0: the kernel with unrolled (kh, j) loops and a compile-time row pitch; KT == 0: everything at run time.
-template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT>
-static int launch_variant(const Conv2dSetup &s, bool sp, cudaStream_t st) {
-    if (KT == 0) return launch_pitch<N, SC, TM, TN, UNPACKED, 0, 0, 0>(s, sp, st);
+// U: channels per unrolled group with placed carry-save moves (0: moves at stage ends).
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, int U>
+static int launch_variant_u(const Conv2dSetup &s, bool sp, cudaStream_t st) {
+    if (KT == 0) return launch_pitch<N, SC, TM, TN, UNPACKED, 0, 0, 0, 0>(s, sp, st);
     switch (s.kp.XBS) {
-        case 8: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 8>(s, sp, st);
-        case 16: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 16>(s, sp, st);
-        case 32: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 32>(s, sp, st);
-        case 64: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 64>(s, sp, st);
+        case 8: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 8, U>(s, sp, st);
+        case 16: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 16, U>(s, sp, st);
+        case 32: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 32, U>(s, sp, st);
+        case 64: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 64, U>(s, sp, st);
         default: return HIKONV_ERR_UNSUPPORTED;
     }
+}
+
+// GROUPED: also instantiate the kernel with placed moves (groups of 3 channels).
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, bool GROUPED = false>
+static int launch_variant(const Conv2dSetup &s, bool sp, cudaStream_t st) {
+    if constexpr (GROUPED) {
+        if (s.kp.move_every == 3) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 3>(s, sp, st);
+    }
+    if (s.kp.move_every != 0) return HIKONV_ERR_UNSUPPORTED;
+    return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 0>(s, sp, st);
 }
 
 constexpr int kTM = 4, kTN = 4;          // per-thread tile of the packed kernels
@@ -682,12 +733,26 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     const int ck_cap = stage_channel_cap(K, L.J);
     int CK = std::min(ck_cap, Ci);
     kp.flush_chunks = 1 << 30;
+    kp.move_every = 0;
     if (!s->unpacked && L.M < Ci * K) {
         if (L.M < K) return HIKONV_ERR_NO_FIT;               // not even one channel's kernel rows between two moves
-        int fc = 1;
-        const int eff = pick_chunking(L.M / K, Ci, &CK, &fc, ck_cap);
-        if (ceil_div(Ci, eff) > (1 << L.carry_bits)) return HIKONV_ERR_NO_FIT;
-        kp.flush_chunks = fc;
+        // the 3x3 kernel with N = 3, S = 13 has a variant whose moves are placed inside unrolled groups of
+        // 3 channels, for layers that have to move that often (stages then hold two groups instead of one);
+        // it needs room for one move per group in the second accumulator.  With six or more channels between
+        // moves the stage-end form measured faster.
+        const int CF = L.M / K;
+        int U = 0;
+        if (L.N == 3 && L.S == 13 && K == 3 && L.J == 1 && !(tune && tune->tile < 0)) U = (CF >= 3 && CF < 6) ? 3 : 0;
+        if (U > 0 && (ceil_div(Ci, U) > (1 << L.carry_bits) || ck_cap < U)) U = 0;
+        if (U > 0) {
+            kp.move_every = U;
+            CK = ck_cap / U * U;
+        } else {
+            int fc = 1;
+            const int eff = pick_chunking(CF, Ci, &CK, &fc, ck_cap);
+            if (ceil_div(Ci, eff) > (1 << L.carry_bits)) return HIKONV_ERR_NO_FIT;
+            kp.flush_chunks = fc;
+        }
     }
     kp.CK = CK;
     kp.a_words = CK * kp.a_plane;
@@ -719,7 +784,7 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
         return launch_variant<1, 0, kTMU, kTNU, true, 0, 0>(s, sp, st);
     }
     // the layouts of 3x3 and 1x1 layers with the slot width and loop bounds as compile-time constants
-    if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1>(s, sp, st);
+    if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1, true>(s, sp, st);
     if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
