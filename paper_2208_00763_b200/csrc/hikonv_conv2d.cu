@@ -259,6 +259,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             for (int i = 0; i < TM; ++i) ap[i] = aptr[i] + astage;
             const uint32_t *bp = bptr;
             if constexpr (U > 0 && !UNPACKED) {
+#pragma unroll 2
                 for (int c0 = 0; c0 < p.CK; c0 += U) {
 #pragma unroll
                     for (int u = 0; u < U; ++u) {
