@@ -76,6 +76,16 @@ struct AccType<true> {
     typedef int32_t type;
 };
 
+// n / d for 0 <= n < 2^22 and d > 0 with inv_d = 1.0f / d: the float quotient is off by at most one.
+// (The per-thread index arithmetic of a tile would otherwise be some thirty integer divisions.)
+__device__ __forceinline__ int small_div(int n, int d, float inv_d) {
+    int q = (int)((float)n * inv_d);
+    const int r = n - q * d;
+    if (r < 0) --q;
+    else if (r >= d) ++q;
+    return q;
+}
+
 // One multiply-accumulate of the k loop: the packed 32x32->64 product of Eq. 9 added to the 64-bit
 // accumulator, or (comparator) one 32-bit product added to an int32 sum.
 template <bool UNPACKED, bool SP>
@@ -107,7 +117,9 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     uint32_t *Bs = smem + p.b_off;                         // two tiles [CK*K*J][TCO]
 
     const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int tn = tid % p.TNX;
+    const int tnx_log2 = 31 - __clz(p.TNX);                 // TNX is a power of two
+    const int tn = tid & (p.TNX - 1);
+    const float inv_xb = 1.0f / (float)p.XB, inv_ho = 1.0f / (float)p.Ho;
     const int seg = blockIdx.x % p.NSEG;
     const int R0 = (blockIdx.x / p.NSEG) * p.TR;
     const int co0 = blockIdx.y * p.TCO;
@@ -124,7 +136,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     // the lanes of one operand load then read consecutive words (no bank conflicts), and the block in
     // front of a lane's position sits in the lane before it.
     const int lane = tid & 31, warp = tid >> 5;
-    const int lanes_m = 32 / p.TNX, lm = lane / p.TNX;
+    const int lanes_m = 32 >> tnx_log2, lm = lane >> tnx_log2;
     const int wpos0 = warp * lanes_m * TM;
     // this thread's positions: shared-memory address of the packed word for (ci = 0, kh = 0, j = 0)
     const uint32_t *aptr[TM];
@@ -133,10 +145,9 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         const int pos = wpos0 + i * lanes_m + lm;
         int off = p.lead;                                    // idle position: reads valid memory, result dropped
         if (pos < TP) {
-            const int r = pos / p.XB, xb = pos - r * p.XB;
-            const int R = R0 + r;
-            const int b = R / p.Ho;
-            off = p.lead + ((b * p.Hp + (R - b * p.Ho)) - Rp0) * p.XBS + xb;
+            const int r = small_div(pos, p.XB, inv_xb), xb = pos - r * p.XB;
+            const int db = small_div(h0 + r, p.Ho, inv_ho);          // images past the tile's first one
+            off = p.lead + (db * p.Hp + (h0 + r - db * p.Ho) - h0) * p.XBS + xb;
         }
         aptr[i] = As + off;
     }
@@ -196,14 +207,15 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     int piece_src[kPieces], piece_dst[kPieces];
     {
         const int per_ch = NR * xq;
+        const float inv_per_ch = 1.0f / (float)per_ch, inv_xq = 1.0f / (float)xq;
 #pragma unroll
         for (int k = 0; k < kPieces; ++k) {
             const int q = tid + k * nthreads;
             piece_src[k] = 0;
             piece_dst[k] = -1;
             if (q < p.CK * per_ch) {
-                const int cl = q / per_ch, r = q - cl * per_ch;
-                const int rl = r / xq, qd = r - rl * xq;
+                const int cl = small_div(q, per_ch, inv_per_ch), r = q - cl * per_ch;
+                const int rl = small_div(r, xq, inv_xq), qd = r - rl * xq;
                 piece_src[k] = cl * ap_plane + rl * p.XBT + 4 * qd;
                 piece_dst[k] = (cl << 24) | (cl * p.a_plane + p.lead + rl * p.XBS + 4 * qd);
             }
@@ -386,11 +398,11 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         pix_off[i] = 0;
         pix_n[i] = 0;
         if (pos < TP) {
-            const int r = pos / p.XB, xbl = pos - r * p.XB;
+            const int r = small_div(pos, p.XB, inv_xb), xbl = pos - r * p.XB;
             const int xg = seg * p.XO + xbl - p.J;                   // output block in the row; halo positions give no pixels
             if (xbl >= p.J && xg < p.X) {
-                const int R = R0 + r;
-                const int b = R / p.Ho, h = R - b * p.Ho;
+                const int db = small_div(h0 + r, p.Ho, inv_ho);
+                const int b = b0 + db, h = h0 + r - db * p.Ho;
                 pix_off[i] = (((size_t)b * p.Co) * p.Ho + h) * p.Wo + (size_t)xg * N;
                 pix_n[i] = min(N, p.Wo - xg * N);
             }
@@ -428,17 +440,16 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 } else {
                     Y[0] = (uint32_t)acc[i][t];
                 }
-                if (co >= p.Co) continue;
                 const size_t o = pix_off[i] + chan_off;
+                const int n_store = co < p.Co ? pix_n[i] : 0;
 #pragma unroll
                 for (int m = 0; m < N; ++m) {
-                    if (m >= pix_n[i]) continue;
                     int32_t v = (int32_t)Y[m];
                     if constexpr (REQ) {
                         v = max(p.lo, min(p.hi, v >> p.shift));
-                        ((int8_t *)p.out)[o + m] = (int8_t)v;
+                        if (m < n_store) ((int8_t *)p.out)[o + m] = (int8_t)v;
                     } else {
-                        ((int32_t *)p.out)[o + m] = v;
+                        if (m < n_store) ((int32_t *)p.out)[o + m] = v;
                     }
                 }
             }
@@ -685,6 +696,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     if (requant && (shift < 0 || shift > 31 || lo < -128 || hi > 255 || lo > hi)) return HIKONV_ERR_INVALID_ARG;
     const int Ho = H + 2 * pad - K + 1, Wo = W + 2 * pad - K + 1;
     if (Ho < 1 || Wo < 1) return HIKONV_ERR_INVALID_ARG;
+    if (Ho >= (1 << 21)) return HIKONV_ERR_UNSUPPORTED;          // the kernel's row arithmetic uses a float reciprocal
     if ((double)B * Ci * H * W >= 2147483647.0 || (double)B * Ho >= 2147483647.0) return HIKONV_ERR_UNSUPPORTED;
     // the exact sums must fit int32
     const double max_code = (double)(1 << p) * (double)(1 << q);
