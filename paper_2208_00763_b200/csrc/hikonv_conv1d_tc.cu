@@ -95,7 +95,7 @@ __device__ __forceinline__ void store_run(int32_t *y, long long n_out, long long
 // SC > 0 fixes the slot width at compile time (shifts and masks become immediates); SC == 0 reads it
 // from the parameters.
 template <int N, int J, int SC, bool SP, bool FS>
-__global__ void __launch_bounds__(kThreadsTc) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
+__global__ void __launch_bounds__(kThreadsTc, 4) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
     constexpr int R = blocks_per_lane(N);
     constexpr int L = R * N;
     constexpr int HW = (J * N + 3) / 4;          // words in front of the run
