@@ -9,6 +9,9 @@
 // registers), splits N outputs per block and writes its L outputs with 16-byte stores.  Tiles that
 // touch the ends of the signal, and unaligned buffers, take a guarded byte-wise path in the same kernel.
 // The comparator uses the same loads and stores with one 32-bit multiply-add per product.
+#include <mutex>
+#include <unordered_map>
+
 #include "hikonv_cuda.cuh"
 #include "hikonv_conv1d_tc.h"
 
@@ -95,7 +98,7 @@ __device__ __forceinline__ void store_run(int32_t *y, long long n_out, long long
 // SC > 0 fixes the slot width at compile time (shifts and masks become immediates); SC == 0 reads it
 // from the parameters.
 template <int N, int J, int SC, bool SP, bool FS>
-__global__ void __launch_bounds__(kThreadsTc, 4) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
+__global__ void __launch_bounds__(kThreadsTc, (N >= 9 ? 3 : 4)) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
     constexpr int R = blocks_per_lane(N);
     constexpr int L = R * N;
     constexpr int HW = (J * N + 3) / 4;          // words in front of the run
@@ -237,14 +240,23 @@ __global__ void __launch_bounds__(kThreadsTc) conv1d_unpacked_tc_kernel(const Co
 
 // Persistent launch: as many CTAs as fit on the device at once (occupancy query, cached per kernel),
 // fewer when the problem is small; each warp then walks tiles with a grid-wide stride.
+// CTAs of `kernel` that fit one SM, asked once per kernel (all instantiations share one function-pointer
+// type, so the answer is kept per pointer, not per template instance of the launcher).
+static int resident_ctas(const void *kernel) {
+    static std::mutex mutex;
+    static std::unordered_map<const void *, int> known;
+    std::lock_guard<std::mutex> lock(mutex);
+    auto it = known.find(kernel);
+    if (it != known.end()) return it->second;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kThreadsTc, 0) != cudaSuccess || occ < 1) occ = 1;
+    known[kernel] = occ;
+    return occ;
+}
+
 template <typename Kernel>
 static int launch_persistent(Kernel kernel, const Conv1dTcParams &p, cudaStream_t st) {
-    static int resident = 0;                       // CTAs per SM for this kernel instantiation
-    if (resident == 0) {
-        int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kThreadsTc, 0) != cudaSuccess || occ < 1) occ = 1;
-        resident = occ;
-    }
+    const int resident = resident_ctas(reinterpret_cast<const void *>(kernel));
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long long want = (p.n_tiles + kWarpsTc - 1) / kWarpsTc;
