@@ -370,7 +370,13 @@ def run_ours(args):
                                     "hbm_frac": 5.0 * outputs_per_step / (un_ms * 1e-3) / 1e9 / hbm_peak_gbs}
             del d_y
             extra["c1"] = small_case(torch, hk, inputs, dev)
-            extra["c2_by_bits"] = per_bitwidth_table(torch, hk, cases, d_f, d_g, length)
+            d_fd = {}
+            for i, c in enumerate(cases):
+                if c["p"] in (1, 2, 4):      # the widths that divide a byte have a dense-input entry point
+                    vals = inputs.from_storage(host_f[i].numpy(), c["f_signed"])
+                    d_fd[i] = torch.from_numpy(inputs.to_dense(vals, c["p"])).to(dev)
+            extra["c2_by_bits"] = per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd)
+            del d_fd
             del d_f, d_g
             torch.cuda.empty_cache()
             extra.update(layer_workloads(torch, np, hk, inputs, network, dev, imad_peak))
@@ -506,20 +512,29 @@ def small_case(torch, hk, inputs, dev):
     return row
 
 
-def per_bitwidth_table(torch, hk, cases, d_f, d_g, length):
-    """Microseconds per launch for every sweep case, packed and comparator.  Each timed graph holds 12 launches
-    that rotate over the three inputs of the same bitwidth and signedness and over three output buffers
-    (240 MB per cycle), so no launch finds its data in L2."""
+def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
+    """Microseconds per launch for every sweep case, packed and comparator, and for the 1-, 2- and 4-bit cases
+    the packed kernel on dense input (8 / p codes per byte; `dense_hbm_bytes_per_output` = 4 + p / 8).  Each
+    timed graph holds 12 launches that rotate over the three inputs of the same bitwidth and signedness and
+    over three output buffers (240 MB per cycle), so no launch finds its data in L2."""
     table = {}
     ys = [torch.empty(length + 6, dtype=torch.int32, device=d_f[0].device) for _ in range(3)]
     for i, c in enumerate(cases):
         same = [j for j, o in enumerate(cases) if o["p"] == c["p"] and o["f_signed"] == c["f_signed"]]
         row = {}
-        for name, algo in (("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD)):
+        kinds = [("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD)]
+        if i in d_fd:
+            kinds.append(("dense_us", None))
+            row["dense_hbm_bytes_per_output"] = 4.0 + c["p"] / 8.0
+        for name, algo in kinds:
             def fn():
                 for r in range(12):
-                    hk.conv1d(d_f[same[r % len(same)]], d_g[i], c["p"], c["q"], c["f_signed"], c["g_signed"], algo=algo,
-                              out=ys[r % 3][: length + c["K"] - 1])
+                    src = same[r % len(same)]
+                    out = ys[r % 3][: length + c["K"] - 1]
+                    if algo is None:
+                        hk.conv1d_dense(d_fd[src], length, d_g[i], c["p"], c["q"], c["f_signed"], c["g_signed"], out=out)
+                    else:
+                        hk.conv1d(d_f[src], d_g[i], c["p"], c["q"], c["f_signed"], c["g_signed"], algo=algo, out=out)
             fn()
             torch.cuda.synchronize()
             g = torch.cuda.CUDAGraph()

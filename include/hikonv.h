@@ -135,6 +135,21 @@ int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p
                   int f_signed, int g_signed, int32_t *d_y, int algo, const hikonv_tuning_t *tune,
                   void *stream);
 
+/*
+ * hikonv_conv1d_dense - hikonv_conv1d (packed algorithm) on a signal stored without its unused bits
+ * (Section V-B, "Single convolver architecture": weights and features kept compressed in memory and
+ * unpacked into the multiplier's slices as they are read).
+ * d_f_dense: len codes of p bits, p in {1, 2, 4}, 8 / p codes per byte: code e occupies bits
+ * [(e p) % 8, (e p) % 8 + p) of byte (e p) / 8 (two's complement when f_signed); the unused bits of the
+ * last byte are ignored.  ceil(len p / 8) bytes, device, caller-owned; any alignment is accepted, 4-byte
+ * alignment takes the fast path.  d_g, d_y, q, K, tune, stream as for hikonv_conv1d.
+ * Built for the layouts of K in {3, 5, 7} with q == p and g_signed == f_signed; any other combination
+ * returns HIKONV_ERR_UNSUPPORTED (nothing is launched).
+ */
+int hikonv_conv1d_dense(const uint8_t *d_f_dense, size_t len, const int8_t *d_g, int K, int p, int q,
+                        int f_signed, int g_signed, int32_t *d_y, const hikonv_tuning_t *tune,
+                        void *stream);
+
 /* Device scratch needed by hikonv_conv1d_host: room for f, g and y on the device. */
 size_t hikonv_conv1d_host_workspace_bytes(size_t len, int K);
 

@@ -47,6 +47,7 @@ _SIGNATURES = {
     "hikonv_layout": (_i, [_i] * 7 + [ctypes.POINTER(TuningT), ctypes.POINTER(LayoutT)]),
     "hikonv_pack": (_i, [_vp, _sz, _i, _i, _i, _i, _i, _vp, _vp]),
     "hikonv_conv1d": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _i, ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv1d_dense": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv1d_host_workspace_bytes": (_sz, [_sz, _i]),
     "hikonv_conv1d_host": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _i, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz, _i,
@@ -146,6 +147,21 @@ def conv1d(d_f: torch.Tensor, d_g: torch.Tensor, p: int, q: int, f_signed: bool,
         out = torch.empty(n + K - 1, dtype=torch.int32, device=d_f.device)
     _check(lib().hikonv_conv1d(_dev_i8(d_f, "d_f"), n, _dev_i8(d_g, "d_g"), K, p, q, int(f_signed), int(g_signed),
                                out.data_ptr(), algo, _tune(tune), _stream(stream)), "hikonv_conv1d")
+    return out
+
+
+def conv1d_dense(d_f_dense: torch.Tensor, n: int, d_g: torch.Tensor, p: int, q: int, f_signed: bool, g_signed: bool,
+                 tune=None, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """`d_f_dense`: uint8 tensor holding `n` codes of p bits, 8 / p per byte."""
+    K = d_g.numel()
+    if d_f_dense.dtype != torch.uint8 or not d_f_dense.is_cuda or not d_f_dense.is_contiguous():
+        raise ValueError("d_f_dense must be a contiguous CUDA uint8 tensor")
+    if d_f_dense.numel() * 8 < n * p:
+        raise ValueError("d_f_dense holds fewer than n codes")
+    if out is None:
+        out = torch.empty(n + K - 1, dtype=torch.int32, device=d_f_dense.device)
+    _check(lib().hikonv_conv1d_dense(d_f_dense.data_ptr(), n, _dev_i8(d_g, "d_g"), K, p, q, int(f_signed), int(g_signed),
+                                     out.data_ptr(), _tune(tune), _stream(stream)), "hikonv_conv1d_dense")
     return out
 
 

@@ -347,6 +347,33 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     return launch_packed(L.N, kp, L.signed_prod != 0, f_signed != 0, (unsigned)grid, st);
 }
 
+extern "C" int hikonv_conv1d_dense(const uint8_t *d_f_dense, size_t len, const int8_t *d_g, int K, int p, int q, int f_signed,
+                                   int g_signed, int32_t *d_y, const hikonv_tuning_t *tune, void *stream) {
+    int rc = check_conv1d_args(d_f_dense, len, d_g, K, p, q, d_y, HIKONV_ALGO_PACKED32);
+    if (rc != HIKONV_OK) return rc;
+    if (p != 1 && p != 2 && p != 4) return HIKONV_ERR_UNSUPPORTED;      // codes must not straddle bytes
+    hikonv_layout_t L;
+    rc = make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L);
+    if (rc != HIKONV_OK) return rc;
+    if (!conv1d_packed_dense_available(p, L.N, L.J, L.S, L.signed_prod != 0, f_signed != 0)) return HIKONV_ERR_UNSUPPORTED;
+    const SplitConsts sc = make_split_consts(L, p, q, f_signed, g_signed, K, 1);
+    Conv1dTcParams tp;
+    std::memset(&tp, 0, sizeof(tp));
+    const long long n_out = (long long)len + K - 1;
+    tp.f = reinterpret_cast<const int8_t *>(d_f_dense); tp.g = d_g; tp.y = d_y; tp.len = (long long)len; tp.n_out = n_out; tp.K = K;
+    tp.g_signed = g_signed ? 1 : 0;
+    tp.aligned = (((uintptr_t)d_y % 16 == 0) && ((uintptr_t)d_f_dense % 4 == 0)) ? 1 : 0;
+    tp.dense_words = (long long)(((unsigned long long)len * (unsigned)p + 7) / 8 / 4);
+    const int per_tile = conv1d_tc_outputs_per_tile(L.N);
+    tp.n_tiles = (n_out + per_tile - 1) / per_tile;
+    tp.S = L.S; tp.Kc = L.Kc; tp.hi_shift = L.S * L.N; tp.mask = sc.slot_mask; tp.bias = sc.bias;
+    for (int m = 0; m < kMaxN1D; ++m) {
+        tp.seg_shift[m] = m < L.N ? L.S * m : 0;
+        tp.carry_bias[m] = m < L.N ? sc.carry_bias[m] : 0;
+    }
+    return launch_conv1d_packed_dense(tp, p, L.N, L.J, L.signed_prod != 0, f_signed != 0, (cudaStream_t)stream);
+}
+
 extern "C" size_t hikonv_conv1d_host_workspace_bytes(size_t len, int K) {
     if (K < 1) return 0;
     return align_up(len, 256) + align_up((size_t)K, 256) + align_up((len + (size_t)K - 1) * sizeof(int32_t), 256);

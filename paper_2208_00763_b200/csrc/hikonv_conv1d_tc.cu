@@ -64,6 +64,46 @@ __device__ __forceinline__ void load_words(const int8_t *f, long long len, long 
     }
 }
 
+// Dense input: P bits per code (1, 2 or 4), code e at bit (e P) % 8 of byte (e P) / 8.  Field `k` (a
+// compile-time index) of a word array that starts at the lane's first code: one bit-field extract.
+template <bool SIGNED, int P>
+__device__ __forceinline__ uint32_t extract_dense(const uint32_t *v, int k) {
+    constexpr int EPW = 32 / P;
+    uint32_t r;
+    if (SIGNED) asm("bfe.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(v[k / EPW]), "r"((k % EPW) * P), "r"(P));
+    else asm("bfe.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(v[k / EPW]), "r"((k % EPW) * P), "r"(P));
+    return r;
+}
+
+// Loads the NE codes that start at code e_first into v[0 .. NV), code k at bit (k % EPW) P of v[k / EPW].
+// Fast path: NV + 1 aligned words and a funnel shift each (the run of a lane starts at any bit of a word);
+// guarded path: one byte load per code, zero outside [0, len) (Eq. 2).
+template <int NV, int NE, int P>
+__device__ __forceinline__ void load_dense(const int8_t *f, long long len, long long e_first, bool fast, uint32_t (&v)[NV]) {
+    constexpr int EPW = 32 / P;
+    if (fast) {
+        const long long w0 = e_first / EPW;
+        const int boff = (int)(e_first - w0 * EPW) * P;
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(f) + w0;
+        uint32_t w[NV + 1];
+#pragma unroll
+        for (int i = 0; i < NV + 1; ++i) w[i] = __ldg(src + i);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) v[i] = __funnelshift_r(w[i], w[i + 1], boff);
+    } else {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) v[i] = 0;
+#pragma unroll
+        for (int k = 0; k < NE; ++k) {
+            const long long e = e_first + k;
+            if (e >= 0 && e < len) {
+                const uint32_t byte = (uint8_t)__ldg(f + (e * P) / 8);
+                v[k / EPW] |= ((byte >> (int)((e * P) % 8)) & ((1u << P) - 1u)) << ((k % EPW) * P);
+            }
+        }
+    }
+}
+
 // Row pitch (in words) of a lane's run in the warp's staging buffer: L padded so that the 16-byte
 // stores of eight neighbouring lanes fall into different banks.
 __host__ __device__ constexpr int stage_pitch(int L) { return (L % 8 == 0) ? L + 4 : L; }
@@ -97,12 +137,15 @@ __device__ __forceinline__ void store_run(int32_t *y, long long n_out, long long
 
 // SC > 0 fixes the slot width at compile time (shifts and masks become immediates); SC == 0 reads it
 // from the parameters.
-template <int N, int J, int SC, bool SP, bool FS>
-__global__ void __launch_bounds__(kThreadsTc, (N >= 9 ? 3 : 4)) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
+// P == 0: one code per byte; P = 1, 2, 4: dense input with P bits per code.
+template <int N, int J, int SC, bool SP, bool FS, int P = 0>
+__global__ void __launch_bounds__(kThreadsTc, ((N >= 9 && P == 0) ? 3 : 4)) conv1d_packed_tc_kernel(const Conv1dTcParams p) {
     constexpr int R = blocks_per_lane(N);
     constexpr int L = R * N;
-    constexpr int HW = (J * N + 3) / 4;          // words in front of the run
-    constexpr int NWORDS = HW + L / 4;
+    constexpr int HW = (J * N + 3) / 4;          // words in front of the run (one code per byte)
+    constexpr int NE = L + J * N;                // codes a lane needs
+    constexpr int NWORDS = P == 0 ? HW + L / 4 : (NE * (P == 0 ? 8 : P) + 31) / 32;
+    constexpr int FRONT = P == 0 ? 4 * HW : J * N;   // codes held in front of the run
     __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
 
     const int S = SC > 0 ? SC : p.S;
@@ -130,12 +173,24 @@ __global__ void __launch_bounds__(kThreadsTc, (N >= 9 ? 3 : 4)) conv1d_packed_tc
     const int lane = threadIdx.x & 31;
     const long long stride = (long long)gridDim.x * kWarpsTc;
     long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5);
+    // a tile takes the fast path when all its loads and stores are aligned and inside the buffers
+    auto tile_is_fast = [&](long long tile0) -> bool {
+        if (!p.aligned || tile0 < FRONT || tile0 + 32 * L > p.len) return false;
+        if (P == 0) return true;
+        // dense: the last lane reads NWORDS + 1 words from the word that holds its first code
+        const long long last_first = tile0 + 31 * L - J * N;
+        return last_first / (32 / (P == 0 ? 8 : P)) + NWORDS + 1 <= p.dense_words;
+    };
+    auto load_tile = [&](long long tile0, bool fast, uint32_t (&dst)[NWORDS]) {
+        if constexpr (P == 0) load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast, dst);
+        else load_dense<NWORDS, NE, (P == 0 ? 8 : P)>(p.f, p.len, tile0 + lane * L - J * N, fast, dst);
+    };
     uint32_t wn[NWORDS];
     bool fast_n = false;
     if (t < p.n_tiles) {
         const long long tile0 = t * (32 * L);
-        fast_n = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
-        load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast_n, wn);
+        fast_n = tile_is_fast(tile0);
+        load_tile(tile0, fast_n, wn);
     }
     while (t < p.n_tiles) {
         const long long tile0 = t * (32 * L);
@@ -146,19 +201,21 @@ __global__ void __launch_bounds__(kThreadsTc, (N >= 9 ? 3 : 4)) conv1d_packed_tc
         t += stride;
         if (t < p.n_tiles) {                       // next tile's codes are in flight while this one is computed
             const long long next0 = t * (32 * L);
-            fast_n = p.aligned && next0 >= 4 * HW && next0 + 32 * L <= p.len;
-            load_words<NWORDS, HW>(p.f, p.len, next0 + lane * L, fast_n, wn);
+            fast_n = tile_is_fast(next0);
+            load_tile(next0, fast_n, wn);
         }
 
-        // A_x for x = -J .. R-1 (index x + J); element n of block x sits at byte 4 HW + x N + n of w
+        // A_x for x = -J .. R-1 (index x + J); element n of block x is code FRONT + x N + n of w
         uint32_t A[R + J];
 #pragma unroll
         for (int x = -J; x < R; ++x) {
             uint32_t a = 0;
 #pragma unroll
             for (int n = 0; n < N; ++n) {
-                const int pos = 4 * HW + x * N + n;
-                const uint32_t c = extract_code<FS>(w[pos / 4], pos % 4);
+                const int pos = FRONT + x * N + n;
+                uint32_t c;
+                if constexpr (P == 0) c = extract_code<FS>(w[pos / 4], pos % 4);
+                else c = extract_dense<FS, (P == 0 ? 8 : P)>(w, pos);
                 a = (n == 0) ? c : a + c * slot_pow[n];
             }
             A[x + J] = a;
@@ -306,6 +363,31 @@ int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool sp, bool
     HK_NJ(2, 3) HK_NJ(3, 3)
     HK_NJ(2, 4)
 #undef HK_NJ
+    return HIKONV_ERR_UNSUPPORTED;
+}
+
+// Dense input: the layouts of the 1-, 2- and 4-bit cases of the sweep (K = 3, 5, 7; both operands unsigned or
+// both signed), slot width at compile time.
+#define HK_DENSE_LAYOUTS(X) X(1, 11, 1, 3) X(1, 8, 1, 4) X(2, 6, 1, 6) X(2, 5, 1, 6) X(2, 5, 1, 7) X(2, 5, 2, 7) \
+                            X(4, 3, 1, 10) X(4, 3, 2, 11) X(4, 3, 3, 11)
+
+bool conv1d_packed_dense_available(int P, int N, int J, int S, bool sp, bool fs) {
+    if (sp != fs) return false;
+#define HK_X(pp, n, j, sc) if (P == pp && N == n && J == j && S == sc) return true;
+    HK_DENSE_LAYOUTS(HK_X)
+#undef HK_X
+    return false;
+}
+
+int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, bool sp, bool fs, cudaStream_t st) {
+    if (sp != fs) return HIKONV_ERR_UNSUPPORTED;
+#define HK_X(pp, n, j, sc)                                                                                       \
+    if (P == pp && N == n && J == j && p.S == sc) {                                                              \
+        if (fs) return launch_persistent(conv1d_packed_tc_kernel<n, j, sc, true, true, pp>, p, st);             \
+        return launch_persistent(conv1d_packed_tc_kernel<n, j, sc, false, false, pp>, p, st);                   \
+    }
+    HK_DENSE_LAYOUTS(HK_X)
+#undef HK_X
     return HIKONV_ERR_UNSUPPORTED;
 }
 

@@ -18,6 +18,7 @@ struct Conv1dTcParams {
     int hi_shift;            // S * N
     int g_signed;
     int aligned;             // f is 4-byte aligned and y is 16-byte aligned
+    long long dense_words;   // dense input only: whole 32-bit words in the input buffer
     uint32_t mask;
     uint64_t bias;
     int seg_shift[kMaxN1D];
@@ -27,6 +28,9 @@ struct Conv1dTcParams {
 int conv1d_tc_outputs_per_tile(int N);
 bool conv1d_packed_tc_available(int N, int J);
 int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool signed_prod, bool f_signed, cudaStream_t st);
+// Dense input (P = 1, 2 or 4 bits per code, 8 / P codes per byte): the layouts that are instantiated.
+bool conv1d_packed_dense_available(int P, int N, int J, int S, bool signed_prod, bool f_signed);
+int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, bool signed_prod, bool f_signed, cudaStream_t st);
 bool conv1d_unpacked_tc_available(int K);
 int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool f_signed, cudaStream_t st);
 

@@ -37,6 +37,19 @@ def to_storage(values: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(v.astype(np.int64) & 0xFF).astype(np.uint8).view(np.int8)
 
 
+def to_dense(values: np.ndarray, bits: int) -> np.ndarray:
+    """Code values -> dense storage: 8 / bits codes per byte, code e at bit (e * bits) % 8 of byte
+    (e * bits) // 8, two's complement for negative codes.  bits must divide 8."""
+    if bits not in (1, 2, 4, 8):
+        raise ValueError("bits must divide 8")
+    v = np.asarray(values).astype(np.int64).ravel() & ((1 << bits) - 1)
+    per = 8 // bits
+    pad = (-v.size) % per
+    v = np.concatenate([v, np.zeros(pad, dtype=np.int64)]).reshape(-1, per)
+    shifts = (np.arange(per) * bits).astype(np.int64)
+    return np.ascontiguousarray((v << shifts).sum(axis=1).astype(np.uint8))
+
+
 def from_storage(stored: np.ndarray, signed: bool) -> np.ndarray:
     """int8 storage bytes -> code values as int64."""
     s = np.asarray(stored)
