@@ -607,11 +607,12 @@ static int launch_variant_u(const Conv2dSetup &s, bool sp, cudaStream_t st) {
     }
 }
 
-// GROUPED: also instantiate the kernel with placed moves (groups of 3 channels).
+// GROUPED: also instantiate the kernels with placed moves (groups of 3 and 4 channels).
 template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, bool GROUPED = false>
 static int launch_variant(const Conv2dSetup &s, bool sp, cudaStream_t st) {
     if constexpr (GROUPED) {
         if (s.kp.move_every == 3) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 3>(s, sp, st);
+        if (s.kp.move_every == 4) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 4>(s, sp, st);
     }
     if (s.kp.move_every != 0) return HIKONV_ERR_UNSUPPORTED;
     return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 0>(s, sp, st);
@@ -749,13 +750,13 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.move_every = 0;
     if (!s->unpacked && L.M < Ci * K) {
         if (L.M < K) return HIKONV_ERR_NO_FIT;               // not even one channel's kernel rows between two moves
-        // the 3x3 kernel with N = 3, S = 13 has a variant whose moves are placed inside unrolled groups of
-        // 3 channels, for layers that have to move that often (stages then hold two groups instead of one);
+        // the 3x3 kernel with N = 3, S = 13 has variants whose moves are placed inside unrolled groups of
+        // 3 or 4 channels, for layers that have to move that often (stages then hold two groups instead of one);
         // it needs room for one move per group in the second accumulator.  With six or more channels between
         // moves the stage-end form measured faster.
         const int CF = L.M / K;
         int U = 0;
-        if (L.N == 3 && L.S == 13 && K == 3 && L.J == 1 && !(tune && tune->tile < 0)) U = (CF >= 3 && CF < 6) ? 3 : 0;
+        if (L.N == 3 && L.S == 13 && K == 3 && L.J == 1 && !(tune && tune->tile < 0)) U = CF >= 6 ? 0 : CF >= 4 ? 4 : CF == 3 ? 3 : 0;
         if (U > 0 && (ceil_div(Ci, U) > (1 << L.carry_bits) || ck_cap < U)) U = 0;
         if (U > 0) {
             kp.move_every = U;

@@ -73,11 +73,11 @@ def test_forced_words_per_block(n):
             _layer(x, w, 1, 4, 4, True, True, hk.ALGO_PACKED32, tune={"N": 4})
 
 
-@pytest.mark.parametrize("ci", [4, 7, 20, 64, 130])
+@pytest.mark.parametrize("ci", [4, 7, 20, 64, 130, 256])
 def test_carry_save_schedules(ci):
     # 3x3 layers at N = 3, S = 13 move slot bits to the second accumulator at stage ends (s4 x s4, and any layer
-    # with tile < 0) or at fixed places inside groups of 3 channels (u4 x s4); channel counts that are not
-    # multiples of the group leave zero-weight channels in the last group
+    # with tile < 0) or at fixed places inside groups of 3 or 4 channels (u4 x s4, by depth); channel counts that
+    # are not multiples of the group leave zero-weight channels in the last group
     for (xs, ws) in ((True, True), (False, True)):
         x, w = inputs.conv2d_case(2, ci, 6, 17, 12, 3, 4, 4, xs, ws, seed=300 + ci)
         ref = direct.conv2d_nchw(x, w, 1)
