@@ -42,10 +42,10 @@ SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int f_sign
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // Words per packed kernel row in the 2-D kernels' shared memory, and the cap on channels per stage that
-// keeps one staged weight tile within 32 KB.
+// keeps one staged weight tile within 24 KB (two of them and the activation tiles share 72 KB).
 constexpr int kBPitch = 64;
 inline int stage_channel_cap(int K, int J) {
-    const int c = 8192 / (K * J * kBPitch);
+    const int c = 6144 / (K * J * kBPitch);
     return c < 1 ? 1 : (c > 8 ? 8 : c);
 }
 
