@@ -58,3 +58,28 @@ def test_conv2d_random_configuration(seed):
     g = got.cpu().numpy()
     g = g.astype(np.int64) if lo < 0 else g.view(np.uint8).astype(np.int64)
     assert np.array_equal(g, direct.requant(ref, shift, lo, hi)), what + " requant"
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_conv2d_deep_and_wide_layers(seed):
+    # many input channels (several carry-save moves, every schedule) and rows wider than one tile segment
+    rng = np.random.default_rng(5000 + seed)
+    p, q = int(rng.choice([1, 2, 3, 4, 4, 4, 5, 8])), int(rng.choice([1, 2, 4, 4, 4, 6, 8]))
+    xs, ws = bool(rng.integers(0, 2)), bool(rng.integers(0, 2))
+    K = int(rng.choice([1, 3, 3, 3, 5]))
+    pad = K // 2
+    Ci, Co = int(rng.integers(40, 300)), int(rng.integers(1, 140))
+    if seed % 2:
+        B, H, W = 1, int(rng.integers(1, 5)), int(rng.integers(150, 400))
+    else:
+        B, H, W = int(rng.integers(1, 5)), int(rng.integers(1, 9)), int(rng.integers(1, 30))
+    x, w = inputs.conv2d_case(B, Ci, H, W, Co, K, p, q, xs, ws, seed=seed)
+    ref = direct.conv2d_nchw(x, w, pad)
+    what = "B=%d Ci=%d H=%d W=%d Co=%d K=%d p=%d q=%d xs=%d ws=%d" % (B, Ci, H, W, Co, K, p, q, xs, ws)
+    for algo in (hk.ALGO_PACKED32, hk.ALGO_UNPACKED_IMAD):
+        try:
+            got = hk.conv2d(dev(x), dev(w), pad, p, q, xs, ws, algo=algo)
+        except hk.HikonvError as e:
+            assert algo == hk.ALGO_PACKED32 and e.status in (hk.ERR_NO_FIT, hk.ERR_UNSUPPORTED), what
+            continue
+        assert_exact(got, ref, what + " algo=%d" % algo)
