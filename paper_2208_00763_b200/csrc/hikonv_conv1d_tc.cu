@@ -124,7 +124,7 @@ __device__ __forceinline__ void store_run(int32_t *y, long long n_out, long long
         for (int k = 0; k < L / 4; ++k) {
             const int idx = 4 * (lane + 32 * k);              // first output of this 16-byte piece within the tile
             const int src_lane = idx / L, src_off = idx % L;  // L is a multiple of 4: a piece never straddles two runs
-            dst[lane + 32 * k] = *reinterpret_cast<const int4 *>(stage + src_lane * P + src_off);
+            __stcs(dst + lane + 32 * k, *reinterpret_cast<const int4 *>(stage + src_lane * P + src_off));   // written once, never re-read
         }
         __syncwarp();
     } else {
