@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         aptr[i] = As + off;
     }
 
+    constexpr bool NOE = U < 0;          // the whole (ci, kh) sum fits the slots: no second accumulator at all
     acc_t acc[TM][TN];
     // second packed accumulator (upper slot bits): in shared memory, one 8-byte entry per accumulator and
     // thread, [accumulator][thread] so that a warp touches consecutive entries; only read-modify-written
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int t = 0; t < TN; ++t) acc[i][t] = UNPACKED ? (acc_t)0 : (acc_t)p.bias;
-    if constexpr (!UNPACKED) {
+    if constexpr (!UNPACKED && !NOE) {
 #pragma unroll
         for (int k = 0; k < TM * TN; ++k) Es[k * kMaxThreads2D] = make_uint2(0u, 0u);
     }
@@ -353,7 +354,9 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             }
         }
         // at most M (ci, kh) pairs between two moves; none is needed after the last stage
-        if (!UNPACKED && ++chunks_since_move == p.flush_chunks && ci0 + p.CK < p.Ci) { carry_save(); chunks_since_move = 0; }
+        if constexpr (!UNPACKED && !NOE) {
+            if (++chunks_since_move == p.flush_chunks && ci0 + p.CK < p.Ci) { carry_save(); chunks_since_move = 0; }
+        }
     }
 
     // ---- extract the slots: slot m holds 2^h E_m + Q_m - (moves + 1) bias_m (uint32 arithmetic wraps by design)
@@ -365,10 +368,12 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
     auto slot_value = [&](uint64_t Q, uint64_t Ev, int m) -> uint32_t {
         const uint32_t qv = (uint32_t)(Q >> (S * m)) & slot_msk[m];
+        if constexpr (NOE) return qv - slot_sub[m];
         const uint32_t ev = (uint32_t)(Ev >> (S * m)) & slot_msk[m];
         return (ev << p.hbits) + qv - slot_sub[m];
     };
     auto load_e = [&](int i, int t) -> uint64_t {
+        if constexpr (NOE) return 0;
         const uint2 e = Es[(i * TN + t) * kMaxThreads2D];
         return ((uint64_t)e.y << 32) | e.x;
     };
@@ -608,8 +613,10 @@ static int launch_variant_u(const Conv2dSetup &s, bool sp, cudaStream_t st) {
 }
 
 // GROUPED: also instantiate the kernels with placed moves (groups of 3 and 4 channels).
-template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, bool GROUPED = false>
+template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, bool GROUPED = false, bool SHALLOW = false>
 static int launch_variant(const Conv2dSetup &s, bool sp, cudaStream_t st) {
+    // SHALLOW: instantiated for layers whose whole (ci, kh) sum fits the slots (no second accumulator)
+    if constexpr (SHALLOW) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, -1>(s, sp, st);
     if constexpr (GROUPED) {
         if (s.kp.move_every == 3) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 3>(s, sp, st);
         if (s.kp.move_every == 4) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 4>(s, sp, st);
@@ -800,6 +807,9 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
     // the layouts of 3x3 and 1x1 layers with the slot width and loop bounds as compile-time constants
     if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1, true>(s, sp, st);
     if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, st);
+    // 8-bit activations x 4-bit weights with few input channels (a network's first layer): no moves at all
+    if (s.L.N == 2 && s.L.S == 17 && K == 3 && J == 2 && s.L.M >= s.kp.Ci * K && s.kp.move_every == 0)
+        return launch_variant<2, 17, kTM, kTN, false, 3, 2, false, true>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     switch (s.L.N) {
