@@ -9,7 +9,7 @@
  * (Algorithm 2 / Eq. 29) and optionally requantised.
  *
  * Conventions for every entry point
- *   - Codes are stored one per byte (int8_t).  A signed p-bit code is its int8 value; an
+ *   - Codes are stored one per byte (int8_t; hikonv_conv1d_dense alone reads a denser format).  A signed p-bit code is its int8 value; an
  *     unsigned p-bit code is the byte read as uint8 (so unsigned 8-bit codes use all 256
  *     byte values).  Codes are ASSUMED to lie in their p-bit range; a code outside it
  *     silently breaks the guard bits.
