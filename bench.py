@@ -416,7 +416,7 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         def step():
             hk.conv2d(d_x, d_w, shape["pad"], shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], requant=rq,
                       algo=algo, workspace=ws, out=o)
-        launches_per_step = 3
+        launches_per_step = 2           # one packing launch, one layer launch
         name = "%s: 2-D layer %dx%dx%dx%d -> %d channels, %dx%d, pad %d, p=%d q=%d" % (
             args.workload, shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["K"], shape["pad"],
             shape["p"], shape["q"])
@@ -437,7 +437,7 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
 
         def step():
             net.forward(d_x, algo=algo)
-        launches_per_step = 3 * 9 + 4
+        launches_per_step = 2 * 9 + 4   # nine layers of two launches, four pools
         name = "c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head" % x.shape[0]
         h2d = d_x.numel()
         d2h = x.shape[0] * 36 * H * W * 4

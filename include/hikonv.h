@@ -172,7 +172,7 @@ int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, 
  *   requant != 0: d_out is int8, clamp(sum >> shift, lo, hi) with an arithmetic (floor) shift,
  *                 0 <= shift <= 31, -128 <= lo <= hi <= 255 (values above 127 are stored as the
  *                 byte of the unsigned code).
- * Three kernels run on `stream`: the reversed kernel rows (g = W[co][ci][kh][K-1:0], Theorem 3) and the
+ * Two kernels run on `stream`: the reversed kernel rows (g = W[co][ci][kh][K-1:0], Theorem 3) and the
  * activation rows are packed (Eq. 5) into d_workspace, then the layer kernel streams the packed words.
  * d_workspace: hikonv_conv2d_workspace_bytes(...) bytes of device memory, 256-byte aligned; the call
  * overwrites it and needs nothing from it afterwards.  The unpacked comparator uses the same workspace for

@@ -10,8 +10,8 @@
 // kernel row (g = W[co][ci][kh][K-1:0], Theorem 3).  Slot m < N of Q holds partial sums of pixel
 // xN + m, slot m >= N those of pixel (x+1)N + (m-N): the overlap-add of Theorem 2.
 //
-// Activations are packed once per layer by pack_activations_kernel into Ap[ci][b*Hp + hp][xb] (zero padding
-// rows and halo words materialised), weights by pack_weights_kernel into Bw[(ci,kh,j)][co]; the layer
+// Activations are packed once per layer by pack_operands_kernel into Ap[ci][b*Hp + hp][xb] (zero padding
+// rows and halo words materialised), weights by the same launch into Bw[(ci,kh,j)][co]; the layer
 // kernel streams both with 16-byte asynchronous copies into double-buffered shared memory.
 //
 // A CTA computes TR consecutive output rows (one row segment each) times TCO output channels; it
@@ -464,15 +464,52 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     else finish(std::false_type());
 }
 
+// Reversed, packed kernel rows (Theorem 3: g = W[co][ci][kh][K-1:0], then Eq. 5 per chunk of Kc taps).
+// wp[((ci*K + kh)*J + j)*CoP + co] = sum_{k' < Kc} g[j Kc + k'] 2^(S k').  For the comparator S == 0,
+// Kc == 1: one int32 weight per word.
+struct WeightPackParams {
+    const int8_t *w;
+    uint32_t *wp;
+    int Co, Ci, K, J, Kc, S, w_signed, CoP, total;
+};
+
+__device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int idx) {
+    if (idx >= q.total) return;
+    const int co = idx % q.CoP;
+    int rest = idx / q.CoP;
+    const int j = rest % q.J;
+    rest /= q.J;
+    const int kh = rest % q.K;
+    const int ci = rest / q.K;
+    uint32_t word = 0;
+    if (co < q.Co) {
+        const int8_t *row = q.w + (((size_t)co * q.Ci + ci) * q.K + kh) * q.K;
+        for (int k = 0; k < q.Kc; ++k) {
+            const int g_idx = j * q.Kc + k;              // index into the reversed row
+            if (g_idx < q.K) {
+                const int8_t raw = __ldg(row + (q.K - 1 - g_idx));
+                const int32_t v = q.w_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+                word += (uint32_t)v << (q.S * k);
+            }
+        }
+    }
+    q.wp[idx] = word;
+}
+
 // Packed activation rows (Eq. 5): ap[(ci * B*Hp + b*Hp + hp) * XBT + xb] packs the N input pixels of block
 // x = xb - J of padded row hp, i.e. columns (xb - J) N + K - 1 - pad + n of input row hp - pad, zero where the
 // row or a column lies in the padding.  For the comparator S == 0 and N == 1: one int32 code per word.
 // One thread packs four consecutive words of a row (one 16-byte store); a CTA stays within one
-// (ci, b) plane, whose rows are contiguous in both the input and the packed layout.
+// (ci, b) plane, whose rows are contiguous in both the input and the packed layout.  The CTAs past the
+// activation planes pack the kernel rows (one word per thread), so that a layer needs one packing launch.
 template <bool XS, int N>
-__global__ void __launch_bounds__(256) pack_activations_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
-                                                               int pad, int K, int J, int S, int XBT, int blocks_per_plane,
-                                                               uint32_t *__restrict__ ap) {
+__global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
+                                                            int pad, int K, int J, int S, int XBT, int blocks_per_plane,
+                                                            uint32_t *__restrict__ ap, int act_blocks, const WeightPackParams wq) {
+    if ((int)blockIdx.x >= act_blocks) {
+        pack_weight_word(wq, ((int)blockIdx.x - act_blocks) * 256 + (int)threadIdx.x);
+        return;
+    }
     const int plane = blockIdx.x / blocks_per_plane;                 // ci * B + b
     const int piece = (blockIdx.x - plane * blocks_per_plane) * 256 + threadIdx.x;
     const int xq = XBT / 4;                                          // 16-byte pieces per packed row
@@ -493,34 +530,6 @@ __global__ void __launch_bounds__(256) pack_activations_kernel(const int8_t *__r
             }
     }
     *reinterpret_cast<uint4 *>(ap + ((size_t)plane * Hp + hp) * XBT + 4 * q) = make_uint4(word[0], word[1], word[2], word[3]);
-}
-
-// Reversed, packed kernel rows (Theorem 3: g = W[co][ci][kh][K-1:0], then Eq. 5 per chunk of Kc taps).
-// wp[((ci*K + kh)*J + j)*CoP + co] = sum_{k' < Kc} g[j Kc + k'] 2^(S k').  For the comparator S == 0,
-// Kc == 1: one int32 weight per word.
-__global__ void __launch_bounds__(256) pack_weights_kernel(const int8_t *__restrict__ w, int Co, int Ci, int K, int J, int Kc,
-                                                           int S, int w_signed, int CoP, uint32_t *__restrict__ wp, int total) {
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= total) return;
-    const int co = idx % CoP;
-    int rest = idx / CoP;
-    const int j = rest % J;
-    rest /= J;
-    const int kh = rest % K;
-    const int ci = rest / K;
-    uint32_t word = 0;
-    if (co < Co) {
-        const int8_t *row = w + (((size_t)co * Ci + ci) * K + kh) * K;
-        for (int k = 0; k < Kc; ++k) {
-            const int g_idx = j * Kc + k;                // index into the reversed row
-            if (g_idx < K) {
-                const int8_t raw = __ldg(row + (K - 1 - g_idx));
-                const int32_t v = w_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
-                word += (uint32_t)v << (S * k);
-            }
-        }
-    }
-    wp[idx] = word;
 }
 
 // Eight input columns of two rows per thread (two 8-byte loads, per-byte maxima, one 4-byte store);
@@ -859,18 +868,18 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
     s.kp.wp = d_wp;
     s.kp.ap = d_ap;
     s.kp.out = d_out;
-    // a2: reversed kernel rows packed per (ci, kh, chunk); a3: activation rows packed per block
-    const int total_w = Ci * K * s.L.J * s.kp.CoP;
-    pack_weights_kernel<<<ceil_div(total_w, 256), 256, 0, st>>>(d_w, Co, Ci, K, s.L.J, s.L.Kc, s.L.S, w_signed ? 1 : 0, s.kp.CoP,
-                                                               d_wp, total_w);
-    rc = launch_status();
-    if (rc != HIKONV_OK) return rc;
+    // a2: reversed kernel rows packed per (ci, kh, chunk); a3: activation rows packed per block; one launch
     {
+        WeightPackParams wq;
+        wq.w = d_w; wq.wp = d_wp; wq.Co = Co; wq.Ci = Ci; wq.K = K; wq.J = s.L.J; wq.Kc = s.L.Kc; wq.S = s.L.S;
+        wq.w_signed = w_signed ? 1 : 0; wq.CoP = s.kp.CoP; wq.total = Ci * K * s.L.J * s.kp.CoP;
         const int bpp = ceil_div(s.kp.Hp * (s.kp.XBT / 4), 256);
-        if ((size_t)Ci * B * bpp > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
-        const unsigned grid = (unsigned)((size_t)Ci * B * bpp);
-#define HK_PACK(XSIGN, NN)                                                                                                   \
-    pack_activations_kernel<XSIGN, NN><<<grid, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.S, s.kp.XBT, bpp, d_ap)
+        const size_t act_blocks = (size_t)Ci * B * bpp, w_blocks = (size_t)ceil_div(wq.total, 256);
+        if (act_blocks + w_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
+        const unsigned grid = (unsigned)(act_blocks + w_blocks);
+#define HK_PACK(XSIGN, NN)                                                                                                 \
+    pack_operands_kernel<XSIGN, NN><<<grid, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.S, s.kp.XBT, bpp, d_ap, \
+                                                          (int)act_blocks, wq)
         switch (s.L.N * 2 + (x_signed ? 1 : 0)) {
             case 2: HK_PACK(false, 1); break;
             case 3: HK_PACK(true, 1); break;
