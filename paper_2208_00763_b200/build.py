@@ -15,6 +15,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-O3", "-lineinfo", "-std=c++17", "--use_fast_math",
     "-Xcompiler", "-fPIC", "-shared",
+    "--threads", "0",          # the translation units compile side by side
 ]
 
 
