@@ -39,6 +39,8 @@ namespace hikonv {
 
 constexpr int kMaxThreads2D = 256;
 constexpr int kMaxN2DSeg = 8;      // N + Kc - 1 <= 2 N <= 8
+constexpr int kCopyPieces = 4;     // 16-byte activation pieces per thread and stage whose offsets are kept in registers
+constexpr int kEPitch = 17;        // 8-byte entries per thread in the second-accumulator area (16 used)
 
 struct Conv2dParams {
     const int8_t *x;
@@ -152,19 +154,21 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         aptr[i] = As + off;
     }
 
+    static_assert(UNPACKED || TM * TN <= kEPitch, "second-accumulator pitch too small for the thread tile");
     constexpr bool NOE = U < 0;          // the whole (ci, kh) sum fits the slots: no second accumulator at all
     acc_t acc[TM][TN];
-    // second packed accumulator (upper slot bits): in shared memory, one 8-byte entry per accumulator and
-    // thread, [accumulator][thread] so that a warp touches consecutive entries; only read-modify-written
-    // every M products, it would otherwise hold half of the thread's registers
-    uint2 *Es = reinterpret_cast<uint2 *>(smem + p.e_off) + tid;
+    // second packed accumulator (upper slot bits): in shared memory, TM * TN 8-byte entries per thread with
+    // a pitch of kEPitch entries per thread (odd, so that the lanes of a warp fall into different banks
+    // and every access has an immediate offset); only read-modify-written every M products, it would
+    // otherwise hold half of the thread's registers
+    uint2 *Es = reinterpret_cast<uint2 *>(smem + p.e_off) + tid * kEPitch;
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int t = 0; t < TN; ++t) acc[i][t] = UNPACKED ? (acc_t)0 : (acc_t)p.bias;
     if constexpr (!UNPACKED && !NOE) {
 #pragma unroll
-        for (int k = 0; k < TM * TN; ++k) Es[k * kMaxThreads2D] = make_uint2(0u, 0u);
+        for (int k = 0; k < TM * TN; ++k) Es[k] = make_uint2(0u, 0u);
     }
     int nmoves = 0, chunks_since_move = 0;
 
@@ -179,14 +183,14 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
             for (int t = 0; t < TN; ++t) {
                 uint32_t qlo = (uint32_t)acc[i][t], qhi = (uint32_t)((uint64_t)acc[i][t] >> 32);
-                uint2 e = Es[(i * TN + t) * kMaxThreads2D];
+                uint2 e = Es[i * TN + t];
                 uint32_t elo = e.x, ehi = e.y;
                 const uint32_t hlo = __funnelshift_r(qlo, qhi, h) & mh_lo;
                 const uint32_t hhi = (qhi >> h) & mh_hi;
                 asm("add.cc.u32 %0, %0, %2;\n\taddc.u32 %1, %1, %3;" : "+r"(elo), "+r"(ehi) : "r"(hlo), "r"(hhi));
                 qlo = (qlo & ml_lo) | b_lo;
                 qhi = (qhi & ml_hi) | b_hi;
-                Es[(i * TN + t) * kMaxThreads2D] = make_uint2(elo, ehi);
+                Es[i * TN + t] = make_uint2(elo, ehi);
                 acc[i][t] = (acc_t)(((uint64_t)qhi << 32) | qlo);
             }
         }
@@ -204,7 +208,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 
     // The 16-byte pieces of an activation stage this thread copies: the same ones every stage, so their
     // offsets are worked out once (channel in the top byte of the destination offset, -1: none).
-    constexpr int kPieces = 4;
+    constexpr int kPieces = kCopyPieces;
     int piece_src[kPieces], piece_dst[kPieces];
     {
         const int per_ch = NR * xq;
@@ -235,11 +239,12 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 if (piece_dst[k] >= 0 && (piece_dst[k] >> 24) < ckn) cp_async_16(Adst + (piece_dst[k] & 0xFFFFFF), asrc + piece_src[k]);
         } else {
             const int per_ch = NR * xq;
+            const float inv_xq = 1.0f / (float)xq;
             for (int cl = 0; cl < ckn; ++cl) {
                 const uint32_t *src = asrc + (size_t)cl * ap_plane;
                 uint32_t *dst = Adst + cl * p.a_plane + p.lead;
                 for (int idx = tid; idx < per_ch; idx += nthreads) {
-                    const int rl = idx / xq, qd = idx - rl * xq;
+                    const int rl = small_div(idx, xq, inv_xq), qd = idx - rl * xq;
                     cp_async_16(dst + rl * p.XBS + 4 * qd, src + (size_t)rl * p.XBT + 4 * qd);
                 }
             }
@@ -374,7 +379,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     };
     auto load_e = [&](int i, int t) -> uint64_t {
         if constexpr (NOE) return 0;
-        const uint2 e = Es[(i * TN + t) * kMaxThreads2D];
+        const uint2 e = Es[i * TN + t];
         return ((uint64_t)e.y << 32) | e.x;
     };
     // The upper slots of a position belong to the next position (Theorem 2), which the next lane holds:
@@ -683,7 +688,8 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
             const int span_s = (TR + Ho - 2) / Ho + 1;
             const int ckc = stage_channel_cap(K, J);
             const size_t smem = 2 * 4 * ((size_t)ckc * ((TR + (K - 1) * span_s) * pitch + 8) + (size_t)ckc * K * J * kBPitch);
-            if (smem > 72 * 1024) continue;                            // plus 32 KB of second accumulators per CTA
+            if (smem > 72 * 1024) continue;                            // plus the second accumulators, 136 bytes per thread
+            // (the model keeps charging 32 KB for them: with their true size it preferred tiles that measured slower)
             const int per_sm = std::max(1, std::min(std::min(2048 / threads, 65536 / (threads * 128)), (int)(220 * 1024 / (smem + 32 * 1024))));
             const long long slots = (long long)per_sm * sms;
             const long long full_waves = tiles / slots;
@@ -777,6 +783,10 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         if (U > 0) {
             kp.move_every = U;
             CK = ck_cap / U * U;
+            // a stage's activation pieces should fit the per-thread copy descriptors (kPieces each): small CTAs
+            // stage one group at a time
+            const int pieces_per_channel = kp.NRmax * ((kp.XB + 3) / 4);
+            while (CK > U && CK * pieces_per_channel > kCopyPieces * s->threads) CK -= U;
         } else {
             int fc = 1;
             const int eff = pick_chunking(CF, Ci, &CK, &fc, ck_cap);
@@ -791,7 +801,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     const size_t words = (size_t)kp.b_off + 2 * (size_t)kp.b_words;
     const size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
     kp.e_off = (int)((std::max(words, xch_words) + 3) / 4 * 4);
-    const size_t e_words = s->unpacked ? 0 : (size_t)TM * TN * kMaxThreads2D * 2;
+    const size_t e_words = s->unpacked ? 0 : (size_t)kEPitch * s->threads * 2;
     s->smem_bytes = ((size_t)kp.e_off + e_words) * 4 + 16;
     s->wp_bytes = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
     s->ap_words = (size_t)Ci * B * kp.Hp * kp.XBT;
