@@ -156,6 +156,11 @@ def test_device_entry_points_validate_before_touching_cuda():
     assert lib.hikonv_conv1d(8, 10, 8, 3, 9, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 8, 1, None, None) == hk.ERR_UNSUPPORTED     # 64x64 emulation not built
     assert lib.hikonv_conv1d(8, 10, 8, 0, 4, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
+    # dense input: null pointers, widths that straddle bytes, layouts that are not instantiated
+    assert lib.hikonv_conv1d_dense(None, 10, 8, 3, 4, 4, 0, 0, 8, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_conv1d_dense(8, 10, 8, 3, 3, 3, 0, 0, 8, None, None) == hk.ERR_UNSUPPORTED
+    assert lib.hikonv_conv1d_dense(8, 10, 8, 3, 4, 4, 0, 1, 8, None, None) == hk.ERR_UNSUPPORTED     # mixed signs
+    assert lib.hikonv_conv1d_dense(8, 10, 8, 9, 4, 4, 0, 0, 8, None, None) == hk.ERR_UNSUPPORTED     # K = 9
     assert lib.hikonv_pack(None, 10, 4, 0, 10, 3, 32, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_pack(8, 10, 4, 0, 10, 4, 32, 8, None) == hk.ERR_NO_FIT
     assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 2, 1, 4, 4, 0, 0, 8, 0, 0, 0, 0, 256, 1 << 20, 0, None, None) == hk.ERR_UNSUPPORTED
