@@ -115,6 +115,7 @@ template <int N, int SC, int TM, int TN, bool UNPACKED, bool SP, int KT, int JT,
 __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dParams p) {
     typedef typename AccType<UNPACKED>::type acc_t;
     extern __shared__ __align__(16) uint32_t smem[];
+    grid_dependency_release();
     uint32_t *As = smem;                                   // two tiles [CK][a_plane]
     uint32_t *Bs = smem + p.b_off;                         // two tiles [CK*K*J][TCO]
 
@@ -260,6 +261,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         cp_async_commit();
     };
 
+    grid_dependency_wait();                                          // everything above touched no global memory
     fetch(0, min(p.CK, p.Ci), As, Bs);
     int stage = 0;
     for (int ci0 = 0; ci0 < p.Ci; ci0 += p.CK, stage ^= 1) {
@@ -511,6 +513,8 @@ template <bool XS, int N>
 __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
                                                             int pad, int K, int J, int S, int XBT, int blocks_per_plane,
                                                             uint32_t *__restrict__ ap, int act_blocks, const WeightPackParams wq) {
+    grid_dependency_release();
+    grid_dependency_wait();                                          // the input may come from the kernel before; the workspace may still be read by it
     if ((int)blockIdx.x >= act_blocks) {
         pack_weight_word(wq, ((int)blockIdx.x - act_blocks) * 256 + (int)threadIdx.x);
         return;
@@ -542,6 +546,8 @@ __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__rest
 template <bool SIGNED>
 __global__ void __launch_bounds__(256) maxpool2x2_vec_kernel(const int8_t *__restrict__ in, long long items, int H, int W,
                                                              int8_t *__restrict__ out) {
+    grid_dependency_release();
+    grid_dependency_wait();
     const int Ho = H / 2, W8 = W / 8;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < items; idx += (long long)gridDim.x * blockDim.x) {
         const int w8 = (int)(idx % W8);
@@ -604,7 +610,8 @@ static int launch_pitch(const Conv2dSetup &s, bool sp, cudaStream_t st) {
         auto kern = conv2d_kernel<N, SC, TM, TN, UNPACKED, SPV, KT, JT, PITCH, U>;                               \
         if (s.smem_bytes > 48 * 1024)                                                                            \
             HIKONV_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem_bytes)); \
-        kern<<<s.grid, s.threads, s.smem_bytes, st>>>(s.kp);                                                     \
+        const int launch_rc = launch_dependent(kern, s.grid, dim3(s.threads), s.smem_bytes, st, s.kp);          \
+        if (launch_rc != HIKONV_OK) return launch_rc;                                                            \
     } while (0)
     if (!sp) HK_LAUNCH(false);
     else HK_LAUNCH(true);
@@ -888,8 +895,8 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
         if (act_blocks + w_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
         const unsigned grid = (unsigned)(act_blocks + w_blocks);
 #define HK_PACK(XSIGN, NN)                                                                                                 \
-    pack_operands_kernel<XSIGN, NN><<<grid, 256, 0, st>>>(d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, s.L.S, s.kp.XBT, bpp, d_ap, \
-                                                          (int)act_blocks, wq)
+    rc = launch_dependent(pack_operands_kernel<XSIGN, NN>, dim3(grid), dim3(256), 0, st, d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, \
+                          s.L.S, s.kp.XBT, bpp, d_ap, (int)act_blocks, wq)
         switch (s.L.N * 2 + (x_signed ? 1 : 0)) {
             case 2: HK_PACK(false, 1); break;
             case 3: HK_PACK(true, 1); break;
@@ -990,9 +997,8 @@ extern "C" int hikonv_maxpool2x2_i8(const int8_t *d_in, int B, int C, int H, int
     if (W % 8 == 0 && ((uintptr_t)d_in % 8) == 0 && ((uintptr_t)d_out % 4) == 0) {
         const long long items = total / 4;
         const unsigned grid = (unsigned)std::min((items + 255) / 256, cap);
-        if (is_signed) maxpool2x2_vec_kernel<true><<<grid, 256, 0, (cudaStream_t)stream>>>(d_in, items, H, W, d_out);
-        else maxpool2x2_vec_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>(d_in, items, H, W, d_out);
-        return launch_status();
+        if (is_signed) return launch_dependent(maxpool2x2_vec_kernel<true>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, d_in, items, H, W, d_out);
+        return launch_dependent(maxpool2x2_vec_kernel<false>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, d_in, items, H, W, d_out);
     }
     long long blocks = (total + 255) / 256;
     if (blocks > cap) blocks = cap;

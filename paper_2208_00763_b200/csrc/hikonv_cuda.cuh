@@ -19,6 +19,30 @@ namespace hikonv {
 // After a kernel launch: report a launch failure without clearing an earlier sticky error.
 inline int launch_status() { return cudaPeekAtLastError() == cudaSuccess ? HIKONV_OK : HIKONV_ERR_CUDA; }
 
+// Programmatic dependent launch.  A kernel launched with launch_dependent() may be scheduled while the
+// kernel before it on the stream is still running; it must call grid_dependency_wait() before its first
+// access to global memory (the wait returns once the earlier kernel has finished and its writes are
+// visible).  grid_dependency_release() lets the NEXT kernel of the stream be scheduled early; it takes
+// effect once every CTA of this grid has called it or exited.  Every CTA of every such kernel waits, so
+// completion of a kernel still implies completion of all kernels before it.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <typename... Params, typename... Args>
+inline int launch_dependent(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...) == cudaSuccess ? HIKONV_OK : HIKONV_ERR_CUDA;
+}
+
 // One 32x32->64 multiply-accumulate, acc += a * b (the packed multiply of Eq. 9).
 template <bool SIGNED>
 __device__ __forceinline__ void mad_wide(uint64_t &acc, uint32_t a, uint32_t b) {
