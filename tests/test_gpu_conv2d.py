@@ -178,3 +178,27 @@ def test_compact_cnn_full_size_sampled():
     for b in (0, 63):
         ref_head, _ = direct.cnn_forward(x[b:b + 1], layers, head_w)
         assert np.array_equal(g[b:b + 1], ref_head), "image %d" % b
+
+
+def test_layer_chain_captured_in_a_cuda_graph():
+    # a layer, a requantised layer and a pool captured once and replayed: the kernels are launched with
+    # programmatic dependencies, which a captured graph has to preserve
+    x, w = inputs.conv2d_case(2, 16, 12, 20, 24, 3, 4, 4, True, True, seed=3)
+    d_x, d_w = dev(x), dev(w)
+    ws = torch.empty(hk.conv2d_workspace_bytes(2, 16, 12, 20, 24, 3, 1), dtype=torch.uint8, device="cuda")
+    out = torch.empty((2, 24, 12, 20), dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        hk.conv2d(d_x, d_w, 1, 4, 4, True, True, workspace=ws, out=out)          # first call outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        hk.conv2d(d_x, d_w, 1, 4, 4, True, True, workspace=ws, out=out)
+        o8 = hk.conv2d(d_x, d_w, 1, 4, 4, True, True, requant=(6, -8, 7), workspace=ws)
+        pooled = hk.maxpool2x2_i8(o8, True)
+    out.zero_()
+    graph.replay()
+    graph.replay()
+    ref = direct.conv2d_nchw(x, w, 1)
+    assert_exact(out, ref, "captured layer")
+    assert_exact(pooled, direct.maxpool2x2(direct.requant(ref, 6, -8, 7)), "captured requantised layer and pool")
