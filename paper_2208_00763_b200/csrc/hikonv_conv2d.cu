@@ -541,27 +541,40 @@ __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__rest
     *reinterpret_cast<uint4 *>(ap + ((size_t)plane * Hp + hp) * XBT + 4 * q) = make_uint4(word[0], word[1], word[2], word[3]);
 }
 
-// Eight input columns of two rows per thread (two 8-byte loads, per-byte maxima, one 4-byte store);
-// needs W % 8 == 0 and 8-byte aligned tensors.
+// VEC input bytes of two rows per thread (VEC = 8: two 8-byte loads, one 4-byte store; VEC = 16: two
+// 16-byte loads, one 8-byte store), per-byte maxima; needs W % VEC == 0 and VEC-byte aligned input,
+// VEC/2-byte aligned output.
 template <bool SIGNED>
+__device__ __forceinline__ uint32_t pool_pairs(uint32_t a0, uint32_t a1, uint32_t b0, uint32_t b1) {
+    uint32_t v0 = SIGNED ? __vmaxs4(a0, b0) : __vmaxu4(a0, b0);     // the two rows
+    uint32_t v1 = SIGNED ? __vmaxs4(a1, b1) : __vmaxu4(a1, b1);
+    v0 = SIGNED ? __vmaxs4(v0, v0 >> 8) : __vmaxu4(v0, v0 >> 8);    // bytes 0 and 2 hold the pair maxima
+    v1 = SIGNED ? __vmaxs4(v1, v1 >> 8) : __vmaxu4(v1, v1 >> 8);
+    return __byte_perm(v0, v1, 0x6420);
+}
+
+template <bool SIGNED, int VEC>
 __global__ void __launch_bounds__(256) maxpool2x2_vec_kernel(const int8_t *__restrict__ in, long long items, int H, int W,
                                                              int8_t *__restrict__ out) {
     grid_dependency_release();
     grid_dependency_wait();
-    const int Ho = H / 2, W8 = W / 8;
+    const int Ho = H / 2, WV = W / VEC;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < items; idx += (long long)gridDim.x * blockDim.x) {
-        const int w8 = (int)(idx % W8);
-        const long long rest = idx / W8;
+        const int wv = (int)(idx % WV);
+        const long long rest = idx / WV;
         const int ho = (int)(rest % Ho);
         const long long c = rest / Ho;
-        const int8_t *src = in + (c * H + 2 * ho) * (long long)W + 8 * w8;
-        const uint2 r0 = __ldg(reinterpret_cast<const uint2 *>(src));
-        const uint2 r1 = __ldg(reinterpret_cast<const uint2 *>(src + W));
-        uint32_t v0 = SIGNED ? __vmaxs4(r0.x, r1.x) : __vmaxu4(r0.x, r1.x);
-        uint32_t v1 = SIGNED ? __vmaxs4(r0.y, r1.y) : __vmaxu4(r0.y, r1.y);
-        v0 = SIGNED ? __vmaxs4(v0, v0 >> 8) : __vmaxu4(v0, v0 >> 8);             // bytes 0 and 2 hold the pair maxima
-        v1 = SIGNED ? __vmaxs4(v1, v1 >> 8) : __vmaxu4(v1, v1 >> 8);
-        *reinterpret_cast<uint32_t *>(out + (c * Ho + ho) * (long long)(W / 2) + 4 * w8) = __byte_perm(v0, v1, 0x6420);
+        const int8_t *src = in + (c * H + 2 * ho) * (long long)W + VEC * wv;
+        int8_t *dst = out + (c * Ho + ho) * (long long)(W / 2) + (VEC / 2) * wv;
+        if constexpr (VEC == 16) {
+            const uint4 r0 = __ldg(reinterpret_cast<const uint4 *>(src));
+            const uint4 r1 = __ldg(reinterpret_cast<const uint4 *>(src + W));
+            *reinterpret_cast<uint2 *>(dst) = make_uint2(pool_pairs<SIGNED>(r0.x, r0.y, r1.x, r1.y), pool_pairs<SIGNED>(r0.z, r0.w, r1.z, r1.w));
+        } else {
+            const uint2 r0 = __ldg(reinterpret_cast<const uint2 *>(src));
+            const uint2 r1 = __ldg(reinterpret_cast<const uint2 *>(src + W));
+            *reinterpret_cast<uint32_t *>(dst) = pool_pairs<SIGNED>(r0.x, r0.y, r1.x, r1.y);
+        }
     }
 }
 
@@ -994,11 +1007,18 @@ extern "C" int hikonv_maxpool2x2_i8(const int8_t *d_in, int B, int C, int H, int
     if (total == 0) return HIKONV_OK;
     if ((double)B * C >= 2147483647.0) return HIKONV_ERR_UNSUPPORTED;
     const long long cap = (long long)sm_count() * 32;
+    const cudaStream_t pst = (cudaStream_t)stream;
+    if (W % 16 == 0 && ((uintptr_t)d_in % 16) == 0 && ((uintptr_t)d_out % 8) == 0) {
+        const long long items = total / 8;
+        const unsigned grid = (unsigned)std::min((items + 255) / 256, cap);
+        if (is_signed) return launch_dependent(maxpool2x2_vec_kernel<true, 16>, dim3(grid), dim3(256), 0, pst, d_in, items, H, W, d_out);
+        return launch_dependent(maxpool2x2_vec_kernel<false, 16>, dim3(grid), dim3(256), 0, pst, d_in, items, H, W, d_out);
+    }
     if (W % 8 == 0 && ((uintptr_t)d_in % 8) == 0 && ((uintptr_t)d_out % 4) == 0) {
         const long long items = total / 4;
         const unsigned grid = (unsigned)std::min((items + 255) / 256, cap);
-        if (is_signed) return launch_dependent(maxpool2x2_vec_kernel<true>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, d_in, items, H, W, d_out);
-        return launch_dependent(maxpool2x2_vec_kernel<false>, dim3(grid), dim3(256), 0, (cudaStream_t)stream, d_in, items, H, W, d_out);
+        if (is_signed) return launch_dependent(maxpool2x2_vec_kernel<true, 8>, dim3(grid), dim3(256), 0, pst, d_in, items, H, W, d_out);
+        return launch_dependent(maxpool2x2_vec_kernel<false, 8>, dim3(grid), dim3(256), 0, pst, d_in, items, H, W, d_out);
     }
     long long blocks = (total + 255) / 256;
     if (blocks > cap) blocks = cap;

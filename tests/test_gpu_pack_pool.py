@@ -48,9 +48,17 @@ def test_pack_reproduces_the_printed_multiplicands():
 def test_maxpool():
     rng = np.random.default_rng(2)
     for signed in (False, True):
-        for shape in ((1, 1, 2, 2), (2, 3, 6, 10), (3, 5, 7, 9), (4, 16, 40, 80)):
+        # widths that take the scalar kernel, the 8-byte kernel (W % 8 == 0) and the 16-byte kernel (W % 16 == 0)
+        for shape in ((1, 1, 2, 2), (2, 3, 6, 10), (3, 5, 7, 9), (2, 3, 9, 24), (2, 4, 6, 40), (4, 16, 40, 80), (3, 7, 5, 48)):
             v = inputs.uniform_codes(rng, shape, 8, signed)
             out = hk.maxpool2x2_i8(dev(v), signed)
             torch.cuda.synchronize()
             got = inputs.from_storage(out.cpu().numpy(), signed)
             assert np.array_equal(got, direct.maxpool2x2(v)), (shape, signed)
+        # a view that starts 8 bytes into an allocation: the 16-byte kernel must not be chosen for it
+        v = inputs.uniform_codes(rng, (2, 3, 4, 32), 8, signed)
+        buf = torch.zeros(v.size + 16, dtype=torch.int8, device="cuda")
+        buf[8:8 + v.size] = dev(v).reshape(-1)
+        out = hk.maxpool2x2_i8(buf[8:8 + v.size].view(2, 3, 4, 32), signed)
+        torch.cuda.synchronize()
+        assert np.array_equal(inputs.from_storage(out.cpu().numpy(), signed), direct.maxpool2x2(v))
