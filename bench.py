@@ -527,7 +527,8 @@ def small_case(torch, hk, inputs, dev):
 
 
 def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
-    """Microseconds per launch for every sweep case, packed and comparator, and for the 1-, 2- and 4-bit cases
+    """Microseconds per launch for every sweep case, packed, comparator and the packed method on an emulated
+    64x64 multiplier (`emu64_us`), and for the 1-, 2- and 4-bit cases
     the packed kernel on dense input (8 / p codes per byte; `dense_hbm_bytes_per_output` = 4 + p / 8).  Each
     timed graph holds 12 launches that rotate over the three inputs of the same bitwidth and signedness and
     over three output buffers (240 MB per cycle), so no launch finds its data in L2."""
@@ -536,7 +537,7 @@ def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
     for i, c in enumerate(cases):
         same = [j for j, o in enumerate(cases) if o["p"] == c["p"] and o["f_signed"] == c["f_signed"]]
         row = {}
-        kinds = [("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD)]
+        kinds = [("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD), ("emu64_us", hk.ALGO_PACKED64EMU)]
         if i in d_fd:
             kinds.append(("dense_us", None))
             row["dense_hbm_bytes_per_output"] = 4.0 + c["p"] / 8.0

@@ -12,7 +12,7 @@
  *   - Codes are stored one per byte (int8_t; hikonv_conv1d_dense alone reads a denser format).  A signed p-bit code is its int8 value; an
  *     unsigned p-bit code is the byte read as uint8 (so unsigned 8-bit codes use all 256
  *     byte values).  Codes are ASSUMED to lie in their p-bit range; a code outside it
- *     silently breaks the guard bits.
+ *     silently breaks the guard bits (hikonv_check_range is the debug pass that looks).
  *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  All memory is owned
  *     by the caller; the library allocates nothing and keeps no pointer after a call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device
@@ -39,12 +39,14 @@ typedef enum {
     HIKONV_ERR_NO_FIT = 3,      /* no (N >= 1, S) satisfies the operand, slot and accumulator bounds   */
     HIKONV_ERR_WORKSPACE = 4,   /* workspace pointer null/misaligned or workspace_bytes too small      */
     HIKONV_ERR_CUDA = 5,        /* a CUDA runtime call failed (see cudaGetLastError)                   */
-    HIKONV_ERR_TOO_LARGE = 6    /* the layer needs more scratch than the built-in static buffer holds  */
+    HIKONV_ERR_TOO_LARGE = 6,   /* the layer needs more scratch than the built-in static buffer holds  */
+    HIKONV_ERR_RANGE = 7        /* hikonv_check_range: a stored code lies outside its p-bit range      */
 } hikonv_status;
 
 typedef enum {
     HIKONV_ALGO_PACKED32 = 0,      /* packed operands, 32x32->64 multiply (mad.wide)                    */
-    HIKONV_ALGO_PACKED64EMU = 1,   /* 64x64 multiplier emulated from 32-bit pieces: not built           */
+    HIKONV_ALGO_PACKED64EMU = 1,   /* packed operands of 64 bits, 64x64->128 product built from 32-bit
+                                      multiplies (Section IV-C's wider multiplier); hikonv_conv1d only */
     HIKONV_ALGO_UNPACKED_IMAD = 2  /* comparator: one product per 32-bit multiply-add, int32 accumulate */
 } hikonv_algo;
 
@@ -115,6 +117,17 @@ int hikonv_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int
                   const hikonv_tuning_t *tune, hikonv_layout_t *out);
 
 /*
+ * hikonv_layout_emu64 - the 1-D layout for a 64x64->128 multiplier (HIKONV_ALGO_PACKED64EMU; host only).
+ * The rules of hikonv_layout with dims == 1 and 64 / 128 bits in place of 32 / 64: Eq. 6 with
+ * Gb = ceil(log2 K) as the starting slot width, widened until both packed operands fit 64 bits
+ * (63 for an unsigned operand of a signed multiply), the N + Kc - 1 slots fit 128 bits and every slot
+ * holds the extreme sum it can receive after the overlap-add of Theorem 2.  N is at most 16.
+ * Fields of `out` as in hikonv_layout_t (M = 1, carry_bits = 0).  Only tune->N and tune->S are used.
+ */
+int hikonv_layout_emu64(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune,
+                        hikonv_layout_t *out);
+
+/*
  * hikonv_pack - Eq. 5: words[x] = sum_{n<N} in[x N + n] * 2^(S n), modulo 2^word_bits.
  * d_in: n codes (device, int8 storage, `bits` wide, signed or not).  The tail of the last word is
  * zero-filled.  d_words: ceil(n / N) words of word_bits (32 or 64) bits, device, naturally aligned.
@@ -125,11 +138,25 @@ int hikonv_pack(const int8_t *d_in, size_t n, int bits, int is_signed, int S, in
                 void *d_words, void *stream);
 
 /*
+ * hikonv_check_range - debug pass: do all n stored codes lie in their range?
+ * The slot width of Eq. 6 and the operand bounds of Eq. 7-8 are derived from the code ranges
+ * [0, 2^bits - 1] (unsigned) and [-2^(bits-1), 2^(bits-1) - 1] (signed); the convolution entry points
+ * assume them and do not look.  This call counts the codes of d_in (device, one code per byte, n of them,
+ * any alignment) outside that range.  d_count: one 8-byte-aligned device word owned by the caller; the
+ * call zeroes it, adds the violations, copies it to *h_count (host, may be NULL) and SYNCHRONISES
+ * `stream` before it returns.  Returns HIKONV_OK when every code is in range, HIKONV_ERR_RANGE when at
+ * least one is not (the count is in *h_count and *d_count).  With bits == 8 every byte is a valid code.
+ */
+int hikonv_check_range(const int8_t *d_in, size_t n, int bits, int is_signed, unsigned long long *d_count,
+                       unsigned long long *h_count, void *stream);
+
+/*
  * hikonv_conv1d - full 1-D convolution F_{len,K}(f, g) (Eq. 2-4 via Theorems 1 and 2).
  * d_f: len codes of p bits; d_g: K codes of q bits; d_y: len + K - 1 int32 outputs (device, 4-byte
  * aligned), y[m] = sum_k f[m-k] g[k] with f zero outside [0, len).
- * algo: HIKONV_ALGO_PACKED32 or HIKONV_ALGO_UNPACKED_IMAD.  tune may be NULL.
- * len >= 1, 1 <= K <= 64.
+ * algo: HIKONV_ALGO_PACKED32, HIKONV_ALGO_UNPACKED_IMAD, or HIKONV_ALGO_PACKED64EMU (64-bit packed
+ * words, layout of hikonv_layout_emu64; same results, kept as the wider-multiplier variant).
+ * tune may be NULL.  len >= 1, 1 <= K <= 64.
  */
 int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p, int q,
                   int f_signed, int g_signed, int32_t *d_y, int algo, const hikonv_tuning_t *tune,

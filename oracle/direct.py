@@ -11,6 +11,8 @@ textbook definition:
 * ``cnn_forward``  - a chain of the above (conv, requantize, optional pool) plus
                      a final convolution with int64 output.
 * ``pack_words``   - Eq. 5, ``A = sum_n f[n] * 2**(S*n)`` reduced modulo the word size.
+* ``count_out_of_range`` - how many values lie outside the p-bit code range the paper assumes
+                     (``[0, 2**p - 1]`` or ``[-2**(p-1), 2**(p-1) - 1]``, the ranges behind Eq. 6-8).
 
 The C file is compiled on first use with ``gcc -O2 -fopenmp`` into
 ``oracle/_build/`` (never committed).
@@ -167,3 +169,10 @@ def pack_words(values, S: int, N: int, word_bits: int) -> np.ndarray:
     if word_bits == 32:
         words &= np.uint64(0xFFFFFFFF)
     return words
+
+
+def count_out_of_range(values, bits: int, signed: bool) -> int:
+    """Number of values outside the p-bit code range (Section IV-A: p-bit unsigned or two's-complement inputs)."""
+    v = _i64(values).ravel()
+    lo, hi = (-(1 << (bits - 1)), (1 << (bits - 1)) - 1) if signed else (0, (1 << bits) - 1)
+    return int(np.count_nonzero((v < lo) | (v > hi)))

@@ -14,7 +14,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhikonv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE = range(7)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE, ERR_RANGE = range(8)
 STATIC_SCRATCH_BYTES = 4 << 20
 ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD = 0, 1, 2
 GB_SINGLE, GB_1D, GB_DNN = 0, 1, 2
@@ -45,7 +45,9 @@ _vp, _sz, _i, _d = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_doub
 _SIGNATURES = {
     "hikonv_plan": (_i, [_i] * 7 + [ctypes.POINTER(PlanT)]),
     "hikonv_layout": (_i, [_i] * 7 + [ctypes.POINTER(TuningT), ctypes.POINTER(LayoutT)]),
+    "hikonv_layout_emu64": (_i, [_i] * 5 + [ctypes.POINTER(TuningT), ctypes.POINTER(LayoutT)]),
     "hikonv_pack": (_i, [_vp, _sz, _i, _i, _i, _i, _i, _vp, _vp]),
+    "hikonv_check_range": (_i, [_vp, _sz, _i, _i, _vp, ctypes.POINTER(ctypes.c_ulonglong), _vp]),
     "hikonv_conv1d": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _i, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv1d_dense": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv1d_host_workspace_bytes": (_sz, [_sz, _i]),
@@ -129,6 +131,13 @@ def layout(p, q, f_signed, g_signed, K, dims, total_terms=0, tune=None) -> dict:
     return {n: getattr(out, n) for n, _ in LayoutT._fields_}
 
 
+def layout_emu64(p, q, f_signed, g_signed, K, tune=None) -> dict:
+    out = LayoutT()
+    _check(lib().hikonv_layout_emu64(p, q, int(f_signed), int(g_signed), K, _tune(tune), ctypes.byref(out)),
+           "hikonv_layout_emu64")
+    return {n: getattr(out, n) for n, _ in LayoutT._fields_}
+
+
 # ------------------------------------------------------------------ device entry points
 
 def pack(d_in: torch.Tensor, bits: int, is_signed: bool, S: int, N: int, word_bits: int = 32, stream=None) -> torch.Tensor:
@@ -138,6 +147,18 @@ def pack(d_in: torch.Tensor, bits: int, is_signed: bool, S: int, N: int, word_bi
     _check(lib().hikonv_pack(_dev_i8(d_in, "d_in"), n, bits, int(is_signed), S, N, word_bits, out.data_ptr(), _stream(stream)),
            "hikonv_pack")
     return out
+
+
+def check_range(d_in: torch.Tensor, bits: int, is_signed: bool, stream=None) -> int:
+    """Number of stored codes outside their range (0 = all valid).  Synchronises the stream."""
+    d_count = torch.empty(1, dtype=torch.int64, device=d_in.device)
+    found = ctypes.c_ulonglong(0)
+    rc = lib().hikonv_check_range(_dev_i8(d_in, "d_in"), d_in.numel(), bits, int(is_signed), d_count.data_ptr(),
+                                  ctypes.byref(found), _stream(stream))
+    if rc not in (OK, ERR_RANGE):
+        _check(rc, "hikonv_check_range")
+    assert (rc == ERR_RANGE) == (found.value > 0)
+    return int(found.value)
 
 
 def conv1d(d_f: torch.Tensor, d_g: torch.Tensor, p: int, q: int, f_signed: bool, g_signed: bool,

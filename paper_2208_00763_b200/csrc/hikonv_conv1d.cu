@@ -13,6 +13,7 @@
 #include <cstring>
 
 #include "hikonv_cuda.cuh"
+#include "hikonv_conv1d_emu64.h"
 #include "hikonv_conv1d_tc.h"
 
 namespace hikonv {
@@ -259,8 +260,8 @@ static int check_conv1d_args(const void *f, size_t len, const void *g, int K, in
     if (!f || !g || !y || len < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
     if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
     if (len > (size_t)1 << 40) return HIKONV_ERR_UNSUPPORTED;
-    if (algo == HIKONV_ALGO_PACKED64EMU) return HIKONV_ERR_UNSUPPORTED;
-    if (algo != HIKONV_ALGO_PACKED32 && algo != HIKONV_ALGO_UNPACKED_IMAD) return HIKONV_ERR_INVALID_ARG;
+    if (algo != HIKONV_ALGO_PACKED32 && algo != HIKONV_ALGO_PACKED64EMU && algo != HIKONV_ALGO_UNPACKED_IMAD)
+        return HIKONV_ERR_INVALID_ARG;
     if (((uintptr_t)y) % 4 != 0) return HIKONV_ERR_INVALID_ARG;
     return HIKONV_OK;
 }
@@ -274,6 +275,8 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     int rc = check_conv1d_args(d_f, len, d_g, K, p, q, d_y, algo);
     if (rc != HIKONV_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    if (algo == HIKONV_ALGO_PACKED64EMU)
+        return launch_conv1d_emu64(d_f, len, d_g, K, p, q, f_signed, g_signed, d_y, tune, st);
     const long long n_out = (long long)len + K - 1;
     const int y_aligned16 = ((uintptr_t)d_y % 16 == 0) ? 1 : 0;
 
@@ -403,7 +406,9 @@ extern "C" double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int 
     const double n_out = (double)len + K - 1;
     if (algo == HIKONV_ALGO_UNPACKED_IMAD) return n_out * K;
     hikonv_layout_t L;
-    if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L) != HIKONV_OK) return 0.0;
+    if (algo == HIKONV_ALGO_PACKED64EMU) {
+        if (make_layout_emu64(p, q, f_signed, g_signed, K, tune, &L) != HIKONV_OK) return 0.0;
+    } else if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L) != HIKONV_OK) return 0.0;
     const double blocks = (double)(((long long)n_out + L.N - 1) / L.N);
     return blocks * L.J;
 }

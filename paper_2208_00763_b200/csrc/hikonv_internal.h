@@ -10,6 +10,7 @@ namespace hikonv {
 
 constexpr int kMaxN1D = 12;     // largest N the 1-D kernels are instantiated for
 constexpr int kMaxN2D = 4;      // largest N the 2-D kernels are instantiated for
+constexpr int kMaxNEmu64 = 16;  // largest N the emulated 64x64 1-D kernel is instantiated for
 constexpr int kMaxSegments = 24;
 constexpr int kMaxK = 64;       // longest kernel accepted
 constexpr int kMaxJ = 16;       // most weight chunks per kernel row
@@ -32,11 +33,22 @@ struct CostModel {
     double carry_save_cycles = 10.0; // moving the upper slot bits to the second accumulator, per accumulator
 };
 
+// Constants of the biased split for the 128-bit product of the emulated 64x64 multiplier (1-D only).
+struct SplitConsts128 {
+    uint64_t bias_lo, bias_hi;          // sum_m seg_bias[m] 2^(S m), low and high halves
+    int32_t carry_bias[kMaxSegments];   // slot m of (product + carry of the previous block), m < N
+    uint32_t slot_mask;                 // 2^S - 1
+};
+
 int validate_codes(int p, int q);
 // Exact-range layout search; `packed_overlap` selects the 1-D rule (block carries are added
 // before the split, so a slot holds all K terms).
 int make_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int total_terms,
                 int row_outputs, const hikonv_tuning_t *tune, hikonv_layout_t *out);
+// Layout for 64-bit operands and a 128-bit product (1-D rule); fields as in hikonv_layout_t with
+// 64 / 128 in place of 32 / 64.
+int make_layout_emu64(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune, hikonv_layout_t *out);
+SplitConsts128 make_split_consts128(const hikonv_layout_t &L, int p, int q, int f_signed, int g_signed, int K);
 SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int f_signed, int g_signed, int K, int M);
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -248,6 +248,118 @@ static int search_layout(int p, int q, int fs, int gs, int K, int dims, int tota
     return HIKONV_OK;
 }
 
+// ---- the 64x64 -> 128 multiplier (the paper's remark that wider multipliers are handled the same way) ----
+// Same rules as the 1-D search above with 64-bit operands and a 128-bit product: both packed operands
+// must fit a 64-bit register, the N + Kc - 1 slots must fit 128 bits, and every slot must hold the
+// extreme sum it can receive once the carry of the previous block has been added (Theorem 2).
+static bool operand_fits64(Range r, int count, int S, bool signed_mul) {
+    if ((long long)S * (count - 1) > 63) return false;
+    i128 lo, hi;
+    packed_range(r, count, S, &lo, &hi);
+    if (signed_mul) return lo >= -((i128)1 << 63) && hi <= ((i128)1 << 63) - 1;
+    return lo >= 0 && hi <= ((i128)1 << 64) - 1;
+}
+
+static bool check_candidate_emu64(int p, int q, int fs, int gs, int K, int N, int S, hikonv_layout_t *L) {
+    if (S < 1 || S > 31 || N < 1) return false;
+    const bool sp = fs || gs;
+    const Range fr = code_range(p, fs), gr = code_range(q, gs);
+    if (!operand_fits64(fr, N, S, sp)) return false;
+    int Kc, J;
+    if (K <= N + 1 && operand_fits64(gr, K, S, sp)) {
+        Kc = K;
+        J = 1;
+    } else {
+        Kc = N;
+        J = ceil_div(K, N);
+        if (!operand_fits64(gr, Kc, S, sp)) return false;
+    }
+    if (J > kMaxJ) return false;
+    const int NS = N + Kc - 1;
+    if (NS > kMaxSegments) return false;
+    if ((long long)S * (NS - 1) >= 128) return false;
+    const int top_bits = std::min(S, 128 - S * (NS - 1));
+    const long long prods[4] = {fr.lo * gr.lo, fr.lo * gr.hi, fr.hi * gr.lo, fr.hi * gr.hi};
+    const long long pmin = *std::min_element(prods, prods + 4), pmax = *std::max_element(prods, prods + 4);
+    int T[kMaxSegments] = {0};
+    for (int j = 0; j < J; ++j) {
+        const int kc = std::min(Kc, K - j * Kc);
+        for (int m = 0; m < NS; ++m) T[m] += pair_count(m, N, kc);
+    }
+    for (int m = 0; m < NS; ++m) {
+        const int w = (m == NS - 1) ? top_bits : S;
+        if (!slot_fits((i128)T[m] * pmin, (i128)T[m] * pmax, w)) return false;
+    }
+    for (int m = 0; m < N; ++m) {       // after the carry of the previous block has been added
+        const int t = T[m] + (m + N < NS ? T[m + N] : 0);
+        if (!slot_fits((i128)t * pmin, (i128)t * pmax, S)) return false;
+    }
+    L->N = N;
+    L->S = S;
+    L->Kc = Kc;
+    L->J = J;
+    L->segments = NS;
+    L->top_bits = top_bits;
+    L->M = 1;
+    L->signed_prod = sp ? 1 : 0;
+    L->carry_bits = 0;
+    return true;
+}
+
+int make_layout_emu64(int p, int q, int fs, int gs, int K, const hikonv_tuning_t *tune, hikonv_layout_t *out) {
+    if (validate_codes(p, q) != HIKONV_OK || K < 1 || K > kMaxK || !out) return HIKONV_ERR_INVALID_ARG;
+    fs = fs ? 1 : 0;
+    gs = gs ? 1 : 0;
+    const int forceN = tune ? tune->N : 0, forceS = tune ? tune->S : 0;
+    if (forceN < 0 || forceS < 0) return HIKONV_ERR_INVALID_ARG;
+    std::memset(out, 0, sizeof(*out));
+    const int S_paper = slice_bits(p, q, guard_bits(HIKONV_GB_1D, 1, K, 1));
+    hikonv_layout_t best;
+    bool found = false;
+    for (int S = forceS ? forceS : S_paper; S <= (forceS ? forceS : 31) && !found; ++S) {
+        double best_rate = 0.0;
+        for (int N = forceN ? forceN : 1; N <= (forceN ? forceN : kMaxNEmu64); ++N) {
+            hikonv_layout_t c;
+            if (!check_candidate_emu64(p, q, fs, gs, K, N, S, &c)) continue;
+            const double rate = (double)c.N / c.J;      // outputs per 64x64 multiply
+            if (rate > best_rate + 1e-9) {
+                best_rate = rate;
+                best = c;
+                found = true;
+            }
+        }
+    }
+    if (!found) return HIKONV_ERR_NO_FIT;
+    best.S_paper = S_paper;
+    *out = best;
+    return HIKONV_OK;
+}
+
+SplitConsts128 make_split_consts128(const hikonv_layout_t &L, int p, int q, int fs, int gs, int K) {
+    SplitConsts128 c;
+    std::memset(&c, 0, sizeof(c));
+    c.slot_mask = (1u << L.S) - 1u;
+    const Range fr = code_range(p, fs ? 1 : 0), gr = code_range(q, gs ? 1 : 0);
+    const long long prods[4] = {fr.lo * gr.lo, fr.lo * gr.hi, fr.hi * gr.lo, fr.hi * gr.hi};
+    const long long pmin = *std::min_element(prods, prods + 4);
+    int T[kMaxSegments] = {0};
+    for (int j = 0; j < L.J; ++j) {
+        const int kc = std::min(L.Kc, K - j * L.Kc);
+        for (int m = 0; m < L.segments; ++m) T[m] += pair_count(m, L.N, kc);
+    }
+    int32_t seg_bias[kMaxSegments];
+    unsigned __int128 bias = 0;
+    for (int m = 0; m < L.segments; ++m) {
+        seg_bias[m] = (int32_t)(-(long long)T[m] * pmin);     // >= 0: lifts the most negative sum to 0
+        bias += (unsigned __int128)(uint32_t)seg_bias[m] << (L.S * m);
+    }
+    c.bias_lo = (uint64_t)bias;
+    c.bias_hi = (uint64_t)(bias >> 64);
+    for (int m = 0; m < L.N; ++m)
+        c.carry_bias[m] = seg_bias[m] + (m + L.N < L.segments ? seg_bias[m + L.N] : 0);
+    return c;
+}
+
 // The search above costs about a hundred microseconds of host time, as much as a layer takes on the
 // device, and its result depends on its arguments alone: keep the most recent results.
 namespace {
@@ -355,6 +467,11 @@ extern "C" int hikonv_layout(int p, int q, int f_signed, int g_signed, int K, in
     return make_layout(p, q, f_signed, g_signed, K, dims, total_terms, 0, tune, out);
 }
 
+extern "C" int hikonv_layout_emu64(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune,
+                                   hikonv_layout_t *out) {
+    return make_layout_emu64(p, q, f_signed, g_signed, K, tune, out);
+}
+
 extern "C" const char *hikonv_status_string(int status) {
     switch (status) {
         case HIKONV_OK: return "ok";
@@ -364,6 +481,7 @@ extern "C" const char *hikonv_status_string(int status) {
         case HIKONV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case HIKONV_ERR_CUDA: return "CUDA runtime error";
         case HIKONV_ERR_TOO_LARGE: return "layer needs more scratch than the built-in static buffer holds";
+        case HIKONV_ERR_RANGE: return "a stored code lies outside its bit range";
         default: return "unknown status";
     }
 }

@@ -89,16 +89,16 @@ def _extreme_vectors(p, q, fs, gs, n, K):
     return out
 
 
-def _model_conv1d(f, g, L, bias_per_slot):
+def _model_conv1d(f, g, L, bias_per_slot, word_bits=32):
     """The kernel's arithmetic in big integers: chunked kernel, carries added before the split,
-    slots lifted by a bias instead of Eq. 29's borrow increment; 32-bit operands, 64-bit product."""
+    slots lifted by a bias instead of Eq. 29's borrow increment; operands of `word_bits`, product of twice as many."""
     N, S, Kc, J = L["N"], L["S"], L["Kc"], L["J"]
     n_out = len(f) + len(g) - 1
     nb = (n_out + N - 1) // N
     fpad = list(f) + [0] * ((nb + 1) * N)
     A = [pm.pack(fpad[x * N:(x + 1) * N], S) for x in range(nb)]
     Bw = [pm.pack(g[j * Kc:(j + 1) * Kc], S) for j in range(J)]
-    lim = 1 << 31
+    lim = 1 << (word_bits - 1)
     for a in A:
         assert (-lim <= a < lim) if L["signed_prod"] else (0 <= a < 2 * lim)
     for b in Bw:
@@ -107,7 +107,7 @@ def _model_conv1d(f, g, L, bias_per_slot):
     y, prev_hi = [], bias >> (S * N)
     for x in range(nb):
         Q = bias + sum(A[x - j] * Bw[j] for j in range(J) if x - j >= 0)
-        assert 0 <= Q < (1 << 64)
+        assert 0 <= Q < (1 << (2 * word_bits))
         D = Q + prev_hi
         for m in range(N):
             carry_bias = bias_per_slot[m] + (bias_per_slot[m + N] if m + N < len(bias_per_slot) else 0)
@@ -139,6 +139,35 @@ def test_layout_1d_is_exact_on_extreme_codes(signed):
                 assert _model_conv1d(f, g, L, bias) == direct.conv1d_full(f, g).tolist()
 
 
+@pytest.mark.parametrize("signed", [False, True])
+def test_layout_emu64_is_exact_on_extreme_codes(signed):
+    # the 64x64 -> 128 variant: same check with 64-bit operands and a 128-bit product, and a wider
+    # multiplier never yields fewer outputs per multiply than the 32-bit one
+    for p in range(1, 9):
+        for K in (1, 2, 3, 5, 7, 9):
+            L = hk.layout_emu64(p, p, signed, signed, K)
+            L32 = hk.layout(p, p, signed, signed, K, 1)
+            assert L["J"] == -(-K // L["Kc"]) and L["segments"] == L["N"] + L["Kc"] - 1
+            assert L["S"] >= L["S_paper"] and L["S"] * (L["segments"] - 1) < 128 and 1 <= L["N"] <= 16
+            assert L["N"] / L["J"] >= min(L32["N"], 16) / L32["J"]
+            lo_f = -(1 << (p - 1)) if signed else 0
+            hi_f = (1 << (p - 1)) - 1 if signed else (1 << p) - 1
+            pmin = min(a * b for a in (lo_f, hi_f) for b in (lo_f, hi_f))
+            T = [0] * L["segments"]
+            for j in range(L["J"]):
+                kc = min(L["Kc"], K - j * L["Kc"])
+                for n in range(L["N"]):
+                    for k in range(kc):
+                        T[n + k] += 1
+            bias = [-t * pmin for t in T]
+            for f, g in _extreme_vectors(p, p, signed, signed, 3 * L["N"] + 2, K):
+                assert _model_conv1d(f, g, L, bias, word_bits=64) == direct.conv1d_full(f, g).tolist()
+    # the printed 4-bit slot width (S = 10 at K = 3) holds six codes in 64 bits... and seven: 4 + 6 * 10 = 64
+    assert hk.layout_emu64(4, 4, False, False, 3, {"S": 10})["N"] == 7
+    with pytest.raises(hk.HikonvError):
+        hk.layout_emu64(4, 4, False, False, 3, {"S": 10, "N": 8})       # 4 + 7 * 10 = 74 bits
+
+
 def test_layout_2d_known_cases():
     c3 = hk.layout(4, 4, True, True, 3, 2, 64 * 3)
     assert c3["J"] == 1 and c3["Kc"] == 3 and c3["M"] >= 1 and c3["S"] * (c3["segments"] - 1) < 64
@@ -154,7 +183,8 @@ def test_device_entry_points_validate_before_touching_cuda():
     lib = hk.lib()
     assert lib.hikonv_conv1d(None, 10, None, 3, 4, 4, 0, 0, None, 0, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_conv1d(8, 10, 8, 3, 9, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
-    assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 8, 1, None, None) == hk.ERR_UNSUPPORTED     # 64x64 emulation not built
+    assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 8, 3, None, None) == hk.ERR_INVALID_ARG     # no such algorithm
+    assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 9, 1, None, None) == hk.ERR_INVALID_ARG     # misaligned output
     assert lib.hikonv_conv1d(8, 10, 8, 0, 4, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
     # dense input: null pointers, widths that straddle bytes, layouts that are not instantiated
     assert lib.hikonv_conv1d_dense(None, 10, 8, 3, 4, 4, 0, 0, 8, None, None) == hk.ERR_INVALID_ARG
@@ -162,6 +192,9 @@ def test_device_entry_points_validate_before_touching_cuda():
     assert lib.hikonv_conv1d_dense(8, 10, 8, 3, 4, 4, 0, 1, 8, None, None) == hk.ERR_UNSUPPORTED     # mixed signs
     assert lib.hikonv_conv1d_dense(8, 10, 8, 9, 4, 4, 0, 0, 8, None, None) == hk.ERR_UNSUPPORTED     # K = 9
     assert lib.hikonv_pack(None, 10, 4, 0, 10, 3, 32, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_check_range(None, 10, 4, 0, 8, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_check_range(8, 10, 9, 0, 8, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_check_range(8, 10, 4, 0, 12, None, None) == hk.ERR_INVALID_ARG     # count word not 8-byte aligned
     assert lib.hikonv_pack(8, 10, 4, 0, 10, 4, 32, 8, None) == hk.ERR_NO_FIT
     assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 2, 1, 4, 4, 0, 0, 8, 0, 0, 0, 0, 256, 1 << 20, 0, None, None) == hk.ERR_UNSUPPORTED
     assert lib.hikonv_conv2d(8, 1, 1, 4, 4, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 0, 0, 0, 0, None, 0, 0, None, None) == hk.ERR_WORKSPACE
@@ -178,6 +211,7 @@ def test_multiply_counts():
     n = 3000
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 3)
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_UNPACKED_IMAD) == (n + 2) * 3
+    assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED64EMU) == -(-(n + 2) // hk.layout_emu64(4, 4, False, False, 3)["N"])
     packed = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_PACKED32)
     unpacked = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_UNPACKED_IMAD)
     macs = 2 * 16 * 10 * 12 * 8 * 9

@@ -62,3 +62,36 @@ def test_maxpool():
         out = hk.maxpool2x2_i8(buf[8:8 + v.size].view(2, 3, 4, 32), signed)
         torch.cuda.synchronize()
         assert np.array_equal(inputs.from_storage(out.cpu().numpy(), signed), direct.maxpool2x2(v))
+
+
+def test_check_range_counts_codes_outside_their_range():
+    # 8-bit values checked against every narrower range: sizes around the 16-byte pieces, unaligned starts
+    rng = np.random.default_rng(21)
+    for signed in (False, True):
+        for n in (1, 15, 16, 17, 47, 1000, 1000003):
+            v = inputs.uniform_codes(rng, (n + 3,), 8, signed)
+            d = dev(v)
+            for off in (0, 1, 3):
+                for bits in range(1, 9):
+                    want = direct.count_out_of_range(v[off:off + n], bits, signed)
+                    assert hk.check_range(d[off:off + n], bits, signed) == want, (signed, n, off, bits)
+    # in-range data of every width, the extremes included, passes; one bad code is found wherever it sits
+    for signed in (False, True):
+        for bits in range(1, 8):
+            lo, hi = inputs.code_range(bits, signed)
+            v = inputs.uniform_codes(rng, (5000,), bits, signed)
+            v[:2] = (lo, hi)
+            assert hk.check_range(dev(v), bits, signed) == 0
+            for pos in (0, 7, 16, 4999):
+                w = v.copy()
+                w[pos] = hi + 1
+                assert hk.check_range(dev(w), bits, signed) == 1
+                w[pos] = lo - 1
+                assert hk.check_range(dev(w), bits, signed) == 1
+    # the status code of the C interface
+    bad = dev(np.array([0, 1, 16, 3]))
+    count = torch.zeros(1, dtype=torch.int64, device="cuda")
+    assert hk.lib().hikonv_check_range(bad.data_ptr(), 4, 4, 0, count.data_ptr(), None, None) == hk.ERR_RANGE
+    assert int(count.item()) == 1
+    assert hk.lib().hikonv_check_range(bad.data_ptr(), 4, 5, 0, count.data_ptr(), None, None) == hk.OK
+    assert hk.status_string(hk.ERR_RANGE)

@@ -211,3 +211,19 @@ def test_pack_words_against_python_ints():
             for x, wv in enumerate(words):
                 exact = sum(int(padded[x * N + n]) << (S * n) for n in range(N))
                 assert int(wv) == exact % (1 << bits)
+
+
+def test_count_out_of_range_against_enumeration():
+    # every int8 value against every width, by the definition of a p-bit code: representable values are
+    # exactly those that survive a round trip through p bits
+    vals = np.arange(-128, 256)
+    for bits in range(1, 9):
+        for signed in (False, True):
+            def representable(v):
+                u = v & ((1 << bits) - 1)
+                back = u - (1 << bits) if signed and (u >> (bits - 1)) else u
+                return back == v
+            want = sum(0 if representable(int(v)) else 1 for v in vals)
+            assert direct.count_out_of_range(vals, bits, signed) == want
+    assert direct.count_out_of_range([0, 15, 16, -1], 4, False) == 2
+    assert direct.count_out_of_range([-8, 7, 8, -9], 4, True) == 2
