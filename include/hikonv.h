@@ -157,6 +157,10 @@ int hikonv_check_range(const int8_t *d_in, size_t n, int bits, int is_signed, un
  * algo: HIKONV_ALGO_PACKED32, HIKONV_ALGO_UNPACKED_IMAD, or HIKONV_ALGO_PACKED64EMU (64-bit packed
  * words, layout of hikonv_layout_emu64; same results, kept as the wider-multiplier variant).
  * tune may be NULL.  len >= 1, 1 <= K <= 64.
+ * The packed algorithm is bound by HBM on this input format, not by the multiplier, so without a forced
+ * layout the call lowers the planner's N to the block size its kernel streams fastest with (8 in place of
+ * 9..12, 4 in place of 5) when the slot width and the number of kernel chunks stay the same;
+ * hikonv_conv1d_multiplies counts the multiplies of the layout that runs.
  */
 int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p, int q,
                   int f_signed, int g_signed, int32_t *d_y, int algo, const hikonv_tuning_t *tune,

@@ -256,6 +256,25 @@ static int launch_unpacked(const Conv1dUnpackedParams &p, unsigned grid, cudaStr
     return launch_status();
 }
 
+// The layout hikonv_conv1d runs with on one-code-per-byte input: the planner's choice (most outputs per
+// multiply), with N lowered to the block size the register-resident kernel streams fastest with when that
+// needs the same slot width and no more kernel chunks (the path is HBM-bound; the extra multiplies are free).
+// A forced N, S or kernel choice (tune) is taken as it is.
+static int layout_for_byte_input(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune,
+                                 hikonv_layout_t *L) {
+    int rc = make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, L);
+    if (rc != HIKONV_OK) return rc;
+    if (tune && (tune->N > 0 || tune->S > 0 || tune->tile > 0)) return rc;
+    const int n_pref = conv1d_tc_preferred_n(L->N);
+    if (n_pref == L->N) return rc;
+    hikonv_tuning_t forced = {n_pref, L->S, 0, 0};
+    hikonv_layout_t alt;
+    if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, &forced, &alt) == HIKONV_OK && alt.J <= L->J &&
+        conv1d_packed_tc_available(alt.N, alt.J))
+        *L = alt;
+    return HIKONV_OK;
+}
+
 static int check_conv1d_args(const void *f, size_t len, const void *g, int K, int p, int q, const void *y, int algo) {
     if (!f || !g || !y || len < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
     if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
@@ -304,7 +323,7 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     }
 
     hikonv_layout_t L;
-    rc = make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L);
+    rc = layout_for_byte_input(p, q, f_signed, g_signed, K, tune, &L);
     if (rc != HIKONV_OK) return rc;
     if (L.N > kMaxN1D) return HIKONV_ERR_UNSUPPORTED;
     const SplitConsts sc = make_split_consts(L, p, q, f_signed, g_signed, K, 1);
@@ -408,7 +427,7 @@ extern "C" double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int 
     hikonv_layout_t L;
     if (algo == HIKONV_ALGO_PACKED64EMU) {
         if (make_layout_emu64(p, q, f_signed, g_signed, K, tune, &L) != HIKONV_OK) return 0.0;
-    } else if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, &L) != HIKONV_OK) return 0.0;
+    } else if (layout_for_byte_input(p, q, f_signed, g_signed, K, tune, &L) != HIKONV_OK) return 0.0;
     const double blocks = (double)(((long long)n_out + L.N - 1) / L.N);
     return blocks * L.J;
 }

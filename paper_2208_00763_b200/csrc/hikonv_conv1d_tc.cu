@@ -10,6 +10,7 @@
 // touch the ends of the signal, and unaligned buffers, take a guarded byte-wise path in the same kernel.
 // The comparator uses the same loads and stores with one 32-bit multiply-add per product.
 #include <mutex>
+#include <type_traits>
 #include <unordered_map>
 
 #include "hikonv_cuda.cuh"
@@ -205,40 +206,47 @@ __global__ void __launch_bounds__(kThreadsTc, ((N >= 9 && P == 0) ? 3 : 4)) conv
             load_tile(next0, fast_n, wn);
         }
 
-        // A_x for x = -J .. R-1 (index x + J); element n of block x is code FRONT + x N + n of w
-        uint32_t A[R + J];
+        // the arithmetic of one tile; `fast_c` is a compile-time copy of `fast`, so that on interior tiles the
+        // staging stores can be issued while later blocks are still being computed (fewer live registers)
+        auto tile_body = [&](auto fast_c) {
+            // A_x for x = -J .. R-1 (index x + J); element n of block x is code FRONT + x N + n of w
+            uint32_t A[R + J];
 #pragma unroll
-        for (int x = -J; x < R; ++x) {
-            uint32_t a = 0;
+            for (int x = -J; x < R; ++x) {
+                uint32_t a = 0;
 #pragma unroll
-            for (int n = 0; n < N; ++n) {
-                const int pos = FRONT + x * N + n;
-                uint32_t c;
-                if constexpr (P == 0) c = extract_code<FS>(w[pos / 4], pos % 4);
-                else c = extract_dense<FS, (P == 0 ? 8 : P)>(w, pos);
-                a = (n == 0) ? c : a + c * slot_pow[n];
-            }
-            A[x + J] = a;
-        }
-        // Q_x for x = -1 .. R-1, carry chain, split
-        int32_t out[L];
-        uint32_t carry = 0;
-#pragma unroll
-        for (int x = -1; x < R; ++x) {
-            uint64_t Q = p.bias;
-#pragma unroll
-            for (int j = 0; j < J; ++j) mad_wide<SP>(Q, A[x - j + J], Bw[j]);
-            if (x >= 0) {
-                const uint64_t D = Q + (uint64_t)carry;
-#pragma unroll
-                for (int m = 0; m < N; ++m) {
-                    const int sh = SC > 0 ? SC * m : p.seg_shift[m];
-                    out[x * N + m] = (int32_t)(shr64_lo(D, sh) & mask) - p.carry_bias[m];
+                for (int n = 0; n < N; ++n) {
+                    const int pos = FRONT + x * N + n;
+                    uint32_t c;
+                    if constexpr (P == 0) c = extract_code<FS>(w[pos / 4], pos % 4);
+                    else c = extract_dense<FS, (P == 0 ? 8 : P)>(w, pos);
+                    a = (n == 0) ? c : a + c * slot_pow[n];
                 }
+                A[x + J] = a;
             }
-            carry = shr64_lo(Q, hi_shift);
-        }
-        store_run<L>(p.y, p.n_out, tile0, lane, fast, s_stage[threadIdx.x >> 5], out);
+            // Q_x for x = -1 .. R-1, carry chain, split
+            int32_t out[L];
+            uint32_t carry = 0;
+#pragma unroll
+            for (int x = -1; x < R; ++x) {
+                uint64_t Q = SP ? p.bias : 0;           // unsigned products are never negative: every slot bias is zero
+#pragma unroll
+                for (int j = 0; j < J; ++j) mad_wide<SP>(Q, A[x - j + J], Bw[j]);
+                if (x >= 0) {
+                    const uint64_t D = Q + (uint64_t)carry;
+#pragma unroll
+                    for (int m = 0; m < N; ++m) {
+                        const int sh = SC > 0 ? SC * m : p.seg_shift[m];
+                        const int32_t field = (int32_t)(shr64_lo(D, sh) & mask);
+                        out[x * N + m] = SP ? field - p.carry_bias[m] : field;
+                    }
+                }
+                carry = shr64_lo(Q, hi_shift);
+            }
+            store_run<L>(p.y, p.n_out, tile0, lane, decltype(fast_c)::value, s_stage[threadIdx.x >> 5], out);
+        };
+        if (fast) tile_body(std::true_type{});
+        else tile_body(std::false_type{});
     }
 }
 
@@ -339,6 +347,15 @@ static int launch_packed_tc_njs(const Conv1dTcParams &p, bool sp, bool fs, cudaS
     return launch_persistent(conv1d_packed_tc_kernel<N, J, SC, true, false>, p, st);
 }
 
+// The 1-D kernels are bound by HBM, not by the multiplier, and run fastest with per-lane runs of 24 to 28
+// outputs at four resident CTAs per SM.  N = 5 (runs of 20) and N >= 9 (runs of 36 to 44, three CTAs) miss
+// that; the block sizes 4 and 8 reach it with the same slot width and a few more multiplies.
+int conv1d_tc_preferred_n(int N) {
+    if (N == 5) return 4;
+    if (N >= 9) return 8;
+    return N;
+}
+
 bool conv1d_packed_tc_available(int N, int J) {
     if (J == 1) return N >= 1 && N <= 12;
     if (J == 2) return N >= 2 && N <= 6;
@@ -350,7 +367,7 @@ bool conv1d_packed_tc_available(int N, int J) {
 int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool sp, bool fs, cudaStream_t st) {
     // layouts of the p = q bitwidth sweep (K = 3, 5, 7) with the slot width as a compile-time constant
 #define HK_NJS(n, j, sc) if (N == n && J == j && p.S == sc) return launch_packed_tc_njs<n, j, sc>(p, sp, fs, st);
-    HK_NJS(11, 1, 3) HK_NJS(8, 1, 4) HK_NJS(6, 1, 6) HK_NJS(5, 1, 6) HK_NJS(5, 1, 7) HK_NJS(5, 2, 7) HK_NJS(4, 1, 8) HK_NJS(4, 2, 9)
+    HK_NJS(11, 1, 3) HK_NJS(8, 1, 3) HK_NJS(8, 1, 4) HK_NJS(4, 1, 6) HK_NJS(4, 1, 7) HK_NJS(4, 2, 7) HK_NJS(6, 1, 6) HK_NJS(5, 1, 6) HK_NJS(5, 1, 7) HK_NJS(5, 2, 7) HK_NJS(4, 1, 8) HK_NJS(4, 2, 9)
     HK_NJS(3, 1, 10) HK_NJS(3, 2, 11) HK_NJS(3, 3, 11) HK_NJS(3, 1, 12) HK_NJS(3, 2, 13) HK_NJS(3, 3, 13)
     HK_NJS(2, 2, 14) HK_NJS(2, 3, 15) HK_NJS(2, 4, 15) HK_NJS(2, 2, 16) HK_NJS(2, 3, 17) HK_NJS(2, 4, 17)
     HK_NJS(2, 2, 18) HK_NJS(2, 3, 19) HK_NJS(2, 4, 19)

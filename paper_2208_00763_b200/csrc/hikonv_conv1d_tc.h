@@ -26,6 +26,8 @@ struct Conv1dTcParams {
 };
 
 int conv1d_tc_outputs_per_tile(int N);
+// Block size the register-resident kernel runs fastest with when the planner chose N (N itself, or a smaller one).
+int conv1d_tc_preferred_n(int N);
 bool conv1d_packed_tc_available(int N, int J);
 int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool signed_prod, bool f_signed, cudaStream_t st);
 // Dense input (P = 1, 2 or 4 bits per code, 8 / P codes per byte): the layouts that are instantiated.
