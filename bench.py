@@ -390,6 +390,17 @@ def run_ours(args):
                     vals = inputs.from_storage(host_f[i].numpy(), c["f_signed"])
                     d_fd[i] = torch.from_numpy(inputs.to_dense(vals, c["p"])).to(dev)
             extra["c2_by_bits"] = per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd)
+            # packed against comparator per bitwidth (the six cases of a width summed) and the cells where packed is not faster
+            by_width = {}
+            for name, row in extra["c2_by_bits"].items():
+                w = by_width.setdefault(name.split("_")[0], {"packed_us": 0.0, "unpacked_us": 0.0})
+                w["packed_us"] += row["packed_us"]
+                w["unpacked_us"] += row["unpacked_us"]
+            for w in by_width.values():
+                w["unpacked_over_packed"] = w["unpacked_us"] / w["packed_us"]
+            extra["c2_packed_vs_unpacked"] = {
+                "by_bitwidth": by_width,
+                "cases_packed_not_faster": sorted(n for n, r in extra["c2_by_bits"].items() if r["packed_us"] >= r["unpacked_us"])}
             del d_fd
             del d_f, d_g
             torch.cuda.empty_cache()
