@@ -212,6 +212,17 @@ def test_multiply_counts():
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 3)
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_UNPACKED_IMAD) == (n + 2) * 3
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED64EMU) == -(-(n + 2) // hk.layout_emu64(4, 4, False, False, 3)["N"])
+    # byte input: the HBM-bound 1-D kernel runs blocks of 8 where the planner says 11 (1-bit, K = 3) and of 4
+    # where it says 5 (2-bit, K = 5), unless the layout is forced; hikonv_layout keeps the planner's answer
+    assert hk.layout(1, 1, False, False, 3, 1)["N"] == 11 and hk.layout(2, 2, False, False, 5, 1)["N"] == 5
+    assert hk.conv1d_multiplies(n, 3, 1, 1, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 8)
+    assert hk.conv1d_multiplies(n, 5, 2, 2, False, False, hk.ALGO_PACKED32) == -(-(n + 4) // 4)
+    assert hk.conv1d_multiplies(n, 3, 1, 1, False, False, hk.ALGO_PACKED32, {"N": 11}) == -(-(n + 2) // 11)
+    # a smaller block that would need more kernel chunks is not taken: 1-bit codes x signed 2-bit taps, K = 9
+    # fit two chunks of N = 5 taps but would need three of N = 4
+    L9 = hk.layout(1, 2, False, True, 9, 1)
+    assert (L9["N"], L9["J"]) == (5, 2)
+    assert hk.conv1d_multiplies(n, 9, 1, 2, False, True, hk.ALGO_PACKED32) == 2 * -(-(n + 8) // 5)
     packed = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_PACKED32)
     unpacked = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_UNPACKED_IMAD)
     macs = 2 * 16 * 10 * 12 * 8 * 9

@@ -95,6 +95,24 @@ def test_forced_layouts():
         assert_exact(_run(fs, gs, 3, 3, True, True, hk.ALGO_PACKED32, tune), direct.conv1d_full(fs, gs), str(tune))
 
 
+@pytest.mark.parametrize("signed", [False, True])
+def test_planner_block_sizes_that_the_automatic_choice_replaces(signed):
+    # without a forced layout the call runs N = 8 / N = 4 where the planner says 11 / 5; the planner's own
+    # layouts stay reachable by forcing N, and both must give the oracle's result
+    for bits, K in ((1, 3), (2, 3), (2, 5), (2, 7)):
+        f, g = inputs.conv1d_case(60013, K, bits, bits, signed, signed, seed=300 + 10 * bits + K)
+        ref = direct.conv1d_full(f, g)
+        n_plan = hk.layout(bits, bits, signed, signed, K, 1)["N"]
+        assert_exact(_run(f, g, bits, bits, signed, signed, hk.ALGO_PACKED32), ref, "automatic p=%d K=%d" % (bits, K))
+        assert_exact(_run(f, g, bits, bits, signed, signed, hk.ALGO_PACKED32, {"N": n_plan}), ref,
+                     "planner N=%d p=%d K=%d" % (n_plan, bits, K))
+    # a layout whose smaller block would need one more kernel chunk keeps the planner's block size
+    rng = np.random.default_rng(31)
+    f = inputs.uniform_codes(rng, (60013,), 1, False)
+    g = inputs.uniform_codes(rng, (9,), 2, True)
+    assert_exact(_run(f, g, 1, 2, False, True, hk.ALGO_PACKED32), direct.conv1d_full(f, g), "1-bit x s2, K=9")
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_unaligned_pointers(algo):
     rng = np.random.default_rng(8)
