@@ -37,12 +37,12 @@ IMAD32_PER_CLK_PER_SM = 64
 IMAD_WIDE_PER_CLK_PER_SM = 32
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of the kernel (two
-# launches of the p=q=4, K=3 signed case at 2^24: 16.80 MB read both times, 8.47 and 8.26 MB written
+# launches of the p=q=4, K=3 signed case at 2^24: 16.80 MB read both times, 9.27 and 8.46 MB written
 # before the counters stopped; the rest of the 67 MB output was still in the 126 MB L2), with the
 # SHA-256 of the kernel source at capture time (a changed source voids the figure).
 NCU_TRAFFIC = {
-    "conv1d_packed_tc": {"sha256": "bb38eab824b7b9394315b32d3bf260fae6d50d46049c11c95bfe8bb3ff24d6a8",
-                         "bytes_per_output": (16.804e6 + 8.362e6) / 16777218.0},
+    "conv1d_packed_tc": {"sha256": "f6fdbe051c664c7fd9d281b6bdff69b91c1bd4aa5514dfcfb6bf19a67880c073",
+                         "bytes_per_output": (16.805e6 + 8.865e6) / 16777218.0},
 }
 
 
@@ -539,7 +539,7 @@ def small_case(torch, hk, inputs, dev):
 
 def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
     """Microseconds per launch for every sweep case, packed, comparator and the packed method on an emulated
-    64x64 multiplier (`emu64_us`), and for the 1-, 2- and 4-bit cases
+    64x64 multiplier (`emu64_us`), the byte dot-product comparator (`dp4a_us`), and for the 1-, 2- and 4-bit cases
     the packed kernel on dense input (8 / p codes per byte; `dense_hbm_bytes_per_output` = 4 + p / 8).  Each
     timed graph holds 12 launches that rotate over the three inputs of the same bitwidth and signedness and
     over three output buffers (240 MB per cycle), so no launch finds its data in L2."""
@@ -548,7 +548,8 @@ def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
     for i, c in enumerate(cases):
         same = [j for j, o in enumerate(cases) if o["p"] == c["p"] and o["f_signed"] == c["f_signed"]]
         row = {}
-        kinds = [("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD), ("emu64_us", hk.ALGO_PACKED64EMU)]
+        kinds = [("packed_us", hk.ALGO_PACKED32), ("unpacked_us", hk.ALGO_UNPACKED_IMAD), ("emu64_us", hk.ALGO_PACKED64EMU),
+                 ("dp4a_us", hk.ALGO_DP4A)]
         if i in d_fd:
             kinds.append(("dense_us", None))
             row["dense_hbm_bytes_per_output"] = 4.0 + c["p"] / 8.0

@@ -47,7 +47,9 @@ typedef enum {
     HIKONV_ALGO_PACKED32 = 0,      /* packed operands, 32x32->64 multiply (mad.wide)                    */
     HIKONV_ALGO_PACKED64EMU = 1,   /* packed operands of 64 bits, 64x64->128 product built from 32-bit
                                       multiplies (Section IV-C's wider multiplier); hikonv_conv1d only */
-    HIKONV_ALGO_UNPACKED_IMAD = 2  /* comparator: one product per 32-bit multiply-add, int32 accumulate */
+    HIKONV_ALGO_UNPACKED_IMAD = 2, /* comparator: one product per 32-bit multiply-add, int32 accumulate */
+    HIKONV_ALGO_DP4A = 3           /* second comparator: four products per byte dot-product instruction
+                                      (dp4a), int32 accumulate; hikonv_conv1d only, K <= 8               */
 } hikonv_algo;
 
 typedef enum {
@@ -88,7 +90,8 @@ typedef struct {
     int M;          /* force the number of accumulated products between two splits  */
     int tile;       /* kernel-specific tile selector (0 = automatic); conv2d: > 0 output
                        rows per CTA, < 0 carry-save moves at stage ends instead of at
-                       fixed places inside channel groups; conv1d: > 0 the general kernel */
+                       fixed places inside channel groups; conv1d: > 0 the general kernel, -32 runs of
+                       32 outputs per lane in the two comparators (default 24) */
 } hikonv_tuning_t;
 
 /*
@@ -154,8 +157,10 @@ int hikonv_check_range(const int8_t *d_in, size_t n, int bits, int is_signed, un
  * hikonv_conv1d - full 1-D convolution F_{len,K}(f, g) (Eq. 2-4 via Theorems 1 and 2).
  * d_f: len codes of p bits; d_g: K codes of q bits; d_y: len + K - 1 int32 outputs (device, 4-byte
  * aligned), y[m] = sum_k f[m-k] g[k] with f zero outside [0, len).
- * algo: HIKONV_ALGO_PACKED32, HIKONV_ALGO_UNPACKED_IMAD, or HIKONV_ALGO_PACKED64EMU (64-bit packed
- * words, layout of hikonv_layout_emu64; same results, kept as the wider-multiplier variant).
+ * algo: HIKONV_ALGO_PACKED32, HIKONV_ALGO_UNPACKED_IMAD, HIKONV_ALGO_PACKED64EMU (64-bit packed
+ * words, layout of hikonv_layout_emu64; same results, kept as the wider-multiplier variant), or
+ * HIKONV_ALGO_DP4A (the SIMD byte dot product, reported beside the packed method; K <= 8, else
+ * HIKONV_ERR_UNSUPPORTED).
  * tune may be NULL.  len >= 1, 1 <= K <= 64.
  * The packed algorithm is bound by HBM on this input format, not by the multiplier, so without a forced
  * layout the call lowers the planner's N to the block size its kernel streams fastest with (8 in place of

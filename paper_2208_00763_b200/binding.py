@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libhikonv.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE, ERR_RANGE = range(8)
 STATIC_SCRATCH_BYTES = 4 << 20
-ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD = 0, 1, 2
+ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD, ALGO_DP4A = 0, 1, 2, 3
 GB_SINGLE, GB_1D, GB_DNN = 0, 1, 2
 
 

@@ -279,7 +279,8 @@ static int check_conv1d_args(const void *f, size_t len, const void *g, int K, in
     if (!f || !g || !y || len < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
     if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
     if (len > (size_t)1 << 40) return HIKONV_ERR_UNSUPPORTED;
-    if (algo != HIKONV_ALGO_PACKED32 && algo != HIKONV_ALGO_PACKED64EMU && algo != HIKONV_ALGO_UNPACKED_IMAD)
+    if (algo != HIKONV_ALGO_PACKED32 && algo != HIKONV_ALGO_PACKED64EMU && algo != HIKONV_ALGO_UNPACKED_IMAD &&
+        algo != HIKONV_ALGO_DP4A)
         return HIKONV_ERR_INVALID_ARG;
     if (((uintptr_t)y) % 4 != 0) return HIKONV_ERR_INVALID_ARG;
     return HIKONV_OK;
@@ -308,9 +309,18 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     tp.g_signed = g_signed ? 1 : 0;
     tp.aligned = (y_aligned16 && ((uintptr_t)d_f % 4 == 0)) ? 1 : 0;
 
+    if (algo == HIKONV_ALGO_DP4A) {
+        if (!conv1d_dp4a_tc_available(K)) return HIKONV_ERR_UNSUPPORTED;
+        const int run = (tune && tune->tile == -32) ? 32 : 24;
+        tp.n_tiles = (n_out + 32 * run - 1) / (32 * run);
+        return launch_conv1d_dp4a_tc(tp, K, f_signed != 0, g_signed != 0, run, st);
+    }
     if (algo == HIKONV_ALGO_UNPACKED_IMAD && want_tc && conv1d_unpacked_tc_available(K)) {
-        tp.n_tiles = (n_out + 32 * 32 - 1) / (32 * 32);
-        return launch_conv1d_unpacked_tc(tp, K, f_signed != 0, st);
+        // runs of 24 outputs per lane at four resident CTAs stream fastest (as for the packed kernel); -32 keeps
+        // the longer runs reachable
+        const int run = (tune && tune->tile == -32) ? 32 : 24;
+        tp.n_tiles = (n_out + 32 * run - 1) / (32 * run);
+        return launch_conv1d_unpacked_tc(tp, K, f_signed != 0, run, st);
     }
     if (algo == HIKONV_ALGO_UNPACKED_IMAD) {
         Conv1dUnpackedParams up;
@@ -424,6 +434,7 @@ extern "C" double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int 
     if (len < 1 || K < 1) return 0.0;
     const double n_out = (double)len + K - 1;
     if (algo == HIKONV_ALGO_UNPACKED_IMAD) return n_out * K;
+    if (algo == HIKONV_ALGO_DP4A) return n_out * ((K + 3) / 4);
     hikonv_layout_t L;
     if (algo == HIKONV_ALGO_PACKED64EMU) {
         if (make_layout_emu64(p, q, f_signed, g_signed, K, tune, &L) != HIKONV_OK) return 0.0;

@@ -250,10 +250,9 @@ __global__ void __launch_bounds__(kThreadsTc, ((N >= 9 && P == 0) ? 3 : 4)) conv
     }
 }
 
-// Comparator: 16 outputs per lane, one product per 32-bit multiply-add.
-template <int K, bool FS>
-__global__ void __launch_bounds__(kThreadsTc) conv1d_unpacked_tc_kernel(const Conv1dTcParams p) {
-    constexpr int L = 32;
+// Comparator: runs of L outputs per lane, one product per 32-bit multiply-add.
+template <int K, bool FS, int L>
+__global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_unpacked_tc_kernel(const Conv1dTcParams p) {
     constexpr int HW = (K - 1 + 3) / 4;
     constexpr int NWORDS = HW + L / 4;
     __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
@@ -298,6 +297,75 @@ __global__ void __launch_bounds__(kThreadsTc) conv1d_unpacked_tc_kernel(const Co
 #pragma unroll
             for (int k = 0; k < K; ++k) s += e[o + (K - 1) - k] * gk[k];      // y[m] = sum_k f[m-k] g[k]
             out[o] = s;
+        }
+        store_run<L>(p.y, p.n_out, tile0, lane, fast, s_stage[threadIdx.x >> 5], out);
+    }
+}
+
+// Second comparator: the byte dot-product instruction (dp4a: four 8-bit products summed into 32 bits), the
+// SIMD alternative to packing codes into a wide multiplier.  Output m needs the codes f[m-K+1 .. m]; tap word
+// t holds the taps g[4t+3], g[4t+2], g[4t+1], g[4t] in its bytes 0..3 (zero past K-1), and the matching window
+// f[m-4t-3 .. m-4t] is cut out of two neighbouring loaded words with one funnel shift.  32 outputs per lane.
+template <bool FS, bool GS>
+__device__ __forceinline__ int32_t dot4(uint32_t codes, uint32_t taps, int32_t acc) {
+    int32_t d;
+    if (FS && GS) asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(codes), "r"(taps), "r"(acc));
+    else if (FS) asm("dp4a.s32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(codes), "r"(taps), "r"(acc));
+    else if (GS) asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(codes), "r"(taps), "r"(acc));
+    else asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(codes), "r"(taps), "r"(acc));
+    return d;
+}
+
+template <int KW, bool FS, bool GS, int L>
+__global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_dp4a_tc_kernel(const Conv1dTcParams p) {
+    constexpr int HW = KW;                       // 4 KW codes in front of the run cover the K - 1 <= 4 KW - 1 it needs
+    constexpr int NWORDS = HW + L / 4;
+    __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
+    uint32_t gw[KW];
+#pragma unroll
+    for (int t = 0; t < KW; ++t) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int k = 4 * t + 3 - j;
+            if (k < p.K) v |= (uint32_t)(uint8_t)__ldg(p.g + k) << (8 * j);
+        }
+        gw[t] = v;
+    }
+    const int lane = threadIdx.x & 31;
+    const long long stride = (long long)gridDim.x * kWarpsTc;
+    long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5);
+    uint32_t wn[NWORDS];
+    bool fast_n = false;
+    if (t < p.n_tiles) {
+        const long long tile0 = t * (32 * L);
+        fast_n = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
+        load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast_n, wn);
+    }
+    while (t < p.n_tiles) {
+        const long long tile0 = t * (32 * L);
+        const bool fast = fast_n;
+        uint32_t w[NWORDS];
+#pragma unroll
+        for (int i = 0; i < NWORDS; ++i) w[i] = wn[i];
+        t += stride;
+        if (t < p.n_tiles) {
+            const long long next0 = t * (32 * L);
+            fast_n = p.aligned && next0 >= 4 * HW && next0 + 32 * L <= p.len;
+            load_words<NWORDS, HW>(p.f, p.len, next0 + lane * L, fast_n, wn);
+        }
+        int32_t out[L];
+#pragma unroll
+        for (int o = 0; o < L; ++o) {
+            int32_t acc = 0;
+#pragma unroll
+            for (int tw = 0; tw < KW; ++tw) {
+                const int rel = o - 4 * tw - 3 + 4 * HW;      // first code of the window, counted from the first loaded code
+                const int idx = rel / 4, r = rel % 4;
+                const uint32_t window = r == 0 ? w[idx] : __funnelshift_r(w[idx], w[idx + 1], 8 * r);
+                acc = dot4<FS, GS>(window, gw[tw], acc);
+            }
+            out[o] = acc;
         }
         store_run<L>(p.y, p.n_out, tile0, lane, fast, s_stage[threadIdx.x >> 5], out);
     }
@@ -410,14 +478,29 @@ int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, boo
 
 bool conv1d_unpacked_tc_available(int K) { return K == 3 || K == 5 || K == 7; }
 
-int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool fs, cudaStream_t st) {
-#define HK_K(k)                                                                                   \
-    if (K == k) {                                                                                 \
-        if (fs) return launch_persistent(conv1d_unpacked_tc_kernel<k, true>, p, st);              \
-        return launch_persistent(conv1d_unpacked_tc_kernel<k, false>, p, st);                     \
+int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool fs, int run, cudaStream_t st) {
+#define HK_K(k, run_c)                                                                                   \
+    if (K == k && run == run_c) {                                                                        \
+        if (fs) return launch_persistent(conv1d_unpacked_tc_kernel<k, true, run_c>, p, st);              \
+        return launch_persistent(conv1d_unpacked_tc_kernel<k, false, run_c>, p, st);                     \
     }
-    HK_K(3) HK_K(5) HK_K(7)
+    HK_K(3, 24) HK_K(5, 24) HK_K(7, 24) HK_K(3, 32) HK_K(5, 32) HK_K(7, 32)
 #undef HK_K
+    return HIKONV_ERR_UNSUPPORTED;
+}
+
+bool conv1d_dp4a_tc_available(int K) { return K >= 1 && K <= 8; }
+
+int launch_conv1d_dp4a_tc(const Conv1dTcParams &p, int K, bool fs, bool gs, int run, cudaStream_t st) {
+#define HK_KW(kw, run_c)                                                                                            \
+    if ((K + 3) / 4 == kw && run == run_c) {                                                                        \
+        if (fs && gs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, true, true, run_c>, p, st);                \
+        if (fs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, true, false, run_c>, p, st);                     \
+        if (gs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, false, true, run_c>, p, st);                     \
+        return launch_persistent(conv1d_dp4a_tc_kernel<kw, false, false, run_c>, p, st);                            \
+    }
+    HK_KW(1, 24) HK_KW(2, 24) HK_KW(1, 32) HK_KW(2, 32)
+#undef HK_KW
     return HIKONV_ERR_UNSUPPORTED;
 }
 

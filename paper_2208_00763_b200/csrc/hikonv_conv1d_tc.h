@@ -34,6 +34,10 @@ int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool signed_p
 bool conv1d_packed_dense_available(int P, int N, int J, int S, bool signed_prod, bool f_signed);
 int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, bool signed_prod, bool f_signed, cudaStream_t st);
 bool conv1d_unpacked_tc_available(int K);
-int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool f_signed, cudaStream_t st);
+int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool f_signed, int run /* outputs per lane: 24 or 32 */, cudaStream_t st);
+// Byte dot-product comparator (four products per dp4a): kernels of up to eight taps.
+bool conv1d_dp4a_tc_available(int K);
+int launch_conv1d_dp4a_tc(const Conv1dTcParams &p, int K, bool f_signed, bool g_signed, int run /* outputs per lane: 24 or 32 */,
+                          cudaStream_t st);
 
 }  // namespace hikonv

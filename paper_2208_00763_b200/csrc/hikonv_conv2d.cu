@@ -734,7 +734,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     if (B < 1 || Ci < 1 || H < 1 || W < 1 || Co < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
     if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
     if (stride != 1 || pad < 0 || pad >= K) return HIKONV_ERR_UNSUPPORTED;
-    if (algo == HIKONV_ALGO_PACKED64EMU) return HIKONV_ERR_UNSUPPORTED;
+    if (algo == HIKONV_ALGO_PACKED64EMU || algo == HIKONV_ALGO_DP4A) return HIKONV_ERR_UNSUPPORTED;
     if (algo != HIKONV_ALGO_PACKED32 && algo != HIKONV_ALGO_UNPACKED_IMAD) return HIKONV_ERR_INVALID_ARG;
     if (requant && (shift < 0 || shift > 31 || lo < -128 || hi > 255 || lo > hi)) return HIKONV_ERR_INVALID_ARG;
     const int Ho = H + 2 * pad - K + 1, Wo = W + 2 * pad - K + 1;

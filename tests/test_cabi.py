@@ -183,7 +183,8 @@ def test_device_entry_points_validate_before_touching_cuda():
     lib = hk.lib()
     assert lib.hikonv_conv1d(None, 10, None, 3, 4, 4, 0, 0, None, 0, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_conv1d(8, 10, 8, 3, 9, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
-    assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 8, 3, None, None) == hk.ERR_INVALID_ARG     # no such algorithm
+    assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 8, 9, None, None) == hk.ERR_INVALID_ARG     # no such algorithm
+    assert lib.hikonv_conv1d(8, 10, 8, 9, 4, 4, 0, 0, 8, hk.ALGO_DP4A, None, None) == hk.ERR_UNSUPPORTED   # dp4a comparator: K <= 8
     assert lib.hikonv_conv1d(8, 10, 8, 3, 4, 4, 0, 0, 9, 1, None, None) == hk.ERR_INVALID_ARG     # misaligned output
     assert lib.hikonv_conv1d(8, 10, 8, 0, 4, 4, 0, 0, 8, 0, None, None) == hk.ERR_INVALID_ARG
     # dense input: null pointers, widths that straddle bytes, layouts that are not instantiated
@@ -211,6 +212,7 @@ def test_multiply_counts():
     n = 3000
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 3)
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_UNPACKED_IMAD) == (n + 2) * 3
+    assert hk.conv1d_multiplies(n, 7, 4, 4, False, False, hk.ALGO_DP4A) == (n + 6) * 2
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED64EMU) == -(-(n + 2) // hk.layout_emu64(4, 4, False, False, 3)["N"])
     # byte input: the HBM-bound 1-D kernel runs blocks of 8 where the planner says 11 (1-bit, K = 3) and of 4
     # where it says 5 (2-bit, K = 5), unless the layout is forced; hikonv_layout keeps the planner's answer

@@ -113,6 +113,18 @@ def test_planner_block_sizes_that_the_automatic_choice_replaces(signed):
     assert_exact(_run(f, g, 1, 2, False, True, hk.ALGO_PACKED32), direct.conv1d_full(f, g), "1-bit x s2, K=9")
 
 
+@pytest.mark.parametrize("algo", [hk.ALGO_UNPACKED_IMAD, hk.ALGO_DP4A])
+def test_comparators_with_runs_of_32_outputs(algo):
+    # tile = -32 selects the longer per-lane runs of the two comparators (24 is the default)
+    for signed in (False, True):
+        for bits in (1, 4, 8):
+            for K in (3, 5, 7):
+                for n in (100003, 1023):
+                    f, g = inputs.conv1d_case(n, K, bits, bits, signed, signed, seed=500 + bits * 10 + K)
+                    assert_exact(_run(f, g, bits, bits, signed, signed, algo, {"tile": -32}), direct.conv1d_full(f, g),
+                                 "runs of 32: p=%d K=%d n=%d signed=%d" % (bits, K, n, signed))
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_unaligned_pointers(algo):
     rng = np.random.default_rng(8)
@@ -151,3 +163,52 @@ def test_full_size_sweep(algo):
         f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"], case["seed"])
         y = _run(f, g, case["p"], case["q"], case["f_signed"], case["g_signed"], algo)
         assert_exact(y, direct.conv1d_full(f, g), str(case))
+
+
+# ---- the byte dot-product comparator (dp4a), kernels of up to eight taps
+
+@pytest.mark.parametrize("signed", [False, True])
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_dp4a_bitwidth_sweep_and_extremes(bits, signed):
+    for K in (3, 5, 7):
+        for n in (100003, 4097):
+            f, g = inputs.conv1d_case(n, K, bits, bits, signed, signed, seed=bits * 100 + K + 1)
+            assert_exact(_run(f, g, bits, bits, signed, signed, hk.ALGO_DP4A), direct.conv1d_full(f, g),
+                         "dp4a p=%d K=%d n=%d signed=%d" % (bits, K, n, signed))
+        for f, g in inputs.extreme_1d(2051, K, bits, bits, signed, signed):
+            assert_exact(_run(f, g, bits, bits, signed, signed, hk.ALGO_DP4A), direct.conv1d_full(f, g),
+                         "dp4a extreme p=%d K=%d signed=%d" % (bits, K, signed))
+
+
+def test_dp4a_mixed_signs_every_kernel_length_and_tiny_signals():
+    rng = np.random.default_rng(41)
+    for (p, q, fs, gs) in ((4, 4, False, True), (8, 4, False, True), (4, 8, True, False), (8, 8, True, True), (8, 8, False, False)):
+        for K in range(1, 9):
+            for n in (1, 2, 5, 33, 1023, 1024, 1025, 5000):
+                f = inputs.uniform_codes(rng, (n,), p, fs)
+                g = inputs.uniform_codes(rng, (K,), q, gs)
+                assert_exact(_run(f, g, p, q, fs, gs, hk.ALGO_DP4A), direct.conv1d_full(f, g), "dp4a p=%d q=%d K=%d n=%d" % (p, q, K, n))
+    f = inputs.uniform_codes(rng, (100,), 4, False)
+    with pytest.raises(hk.HikonvError):
+        _run(f, inputs.uniform_codes(rng, (9,), 4, False), 4, 4, False, False, hk.ALGO_DP4A)
+
+
+def test_dp4a_unaligned_pointers_and_full_size():
+    rng = np.random.default_rng(42)
+    f = inputs.uniform_codes(rng, (20000,), 8, False)
+    g = inputs.uniform_codes(rng, (7,), 4, True)
+    ref = direct.conv1d_full(f, g)
+    for shift in (1, 3):
+        big_f = torch.zeros(20016, dtype=torch.int8, device="cuda")
+        big_y = torch.full((20032,), -7, dtype=torch.int32, device="cuda")
+        big_f[shift:shift + 20000] = dev(f)
+        y = big_y[shift:shift + 20006]
+        hk.conv1d(big_f[shift:shift + 20000], dev(g), 8, 4, False, True, algo=hk.ALGO_DP4A, out=y)
+        assert_exact(y, ref, "dp4a offset %d" % shift)
+        torch.cuda.synchronize()
+        assert int(big_y[shift - 1]) == -7 and int(big_y[shift + 20006]) == -7
+    for case in inputs.c2_cases():
+        if (case["p"], case["K"]) in ((1, 3), (4, 5), (8, 7)):
+            f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"], case["seed"])
+            y = _run(f, g, case["p"], case["q"], case["f_signed"], case["g_signed"], hk.ALGO_DP4A)
+            assert_exact(y, direct.conv1d_full(f, g), "dp4a " + str(case))
