@@ -10,6 +10,9 @@
 //   splits  y[xN+m] = ((D_x >> S m) & mask) - carry_bias[m],  m < N       (Algorithm 2's shift
 //           and mask; the per-slot bias replaces the sign-borrow increment of Eq. 29)
 // Outputs are staged per warp in shared memory and written with coalesced 16-byte stores.
+// This file holds the argument checks, the layout choice and the general (any N, J, K) kernels; the
+// register-resident kernels of the packed method and of the two comparators are in hikonv_conv1d_tc.cu,
+// the variant on an emulated 64x64 multiplier in hikonv_conv1d_emu64.cu.
 #include <cstring>
 
 #include "hikonv_cuda.cuh"
