@@ -36,13 +36,15 @@ HBM_FALLBACK_GBS = 6650.0            # earlier pool measurement, used only when 
 IMAD32_PER_CLK_PER_SM = 64
 IMAD_WIDE_PER_CLK_PER_SM = 32
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of the kernel (two
-# launches of the p=q=4, K=3 signed case at 2^24: 16.80 MB read both times, 9.27 and 8.46 MB written
-# before the counters stopped; the rest of the 67 MB output was still in the 126 MB L2), with the
-# SHA-256 of the kernel source at capture time (a changed source voids the figure).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of the kernel: six
+# consecutive launches of the p=q=4, K=3 signed case at 2^24 rotating over three input and three output
+# buffers, caches not flushed between launches (steady state): 14.2-14.7 MB read, 63.8-65.7 MB written.
+# (With the caches flushed before each launch the same kernel shows 16.8 MB read and 8-9 MB written: most
+# of a launch's output is then still in the 126 MB L2 when its counters stop.)  The SHA-256 is that of the
+# kernel source at capture time; a changed source voids the figure.
 NCU_TRAFFIC = {
     "conv1d_packed_tc": {"sha256": "f6fdbe051c664c7fd9d281b6bdff69b91c1bd4aa5514dfcfb6bf19a67880c073",
-                         "bytes_per_output": (16.805e6 + 8.865e6) / 16777218.0},
+                         "bytes_per_output": (14.443e6 + 65.167e6) / 16777218.0},
 }
 
 
@@ -319,8 +321,8 @@ def run_ours(args):
     roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": hbm_peak_gbs, "unit": "GB/s",
                 "frac": achieved_gbs / hbm_peak_gbs, "traffic": traffic, "peak_kind": "of " + peak_kind,
                 "kernel": "conv1d_packed_tc_kernel", "bytes_per_output": 5,
-                "traffic_note": "DRAM bytes of one launch under ncu; below the algorithmic bytes because most of a launch's "
-                                "output is still in L2 when its counters stop"}
+                "traffic_note": "DRAM bytes per launch under ncu in steady state (six consecutive launches over rotating buffers, "
+                                "caches not flushed between them): 0.95 of the algorithmic bytes, nothing is re-read"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
