@@ -2,6 +2,7 @@
 """Benchmark of the packed low-bit convolution path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+                    [--workload c2|c3|c4|c5] [--algo packed|unpacked|dp4a|emu64]
 
 A "step" is one pass of the whole hot path over the 1-D bitwidth sweep: 48 full convolutions of a
 2^24-element signal (p = q = 1..8, K in {3,5,7}, unsigned and signed), each launch reading its own
@@ -304,7 +305,9 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    total_ms = max_over_ranks(timed_graph(lambda: sweep(hk.ALGO_PACKED32), args.steps, args.warmup))
+    main_algo = {"packed": hk.ALGO_PACKED32, "unpacked": hk.ALGO_UNPACKED_IMAD, "dp4a": hk.ALGO_DP4A,
+                 "emu64": hk.ALGO_PACKED64EMU}[args.algo]
+    total_ms = max_over_ranks(timed_graph(lambda: sweep(main_algo), args.steps, args.warmup))
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step = total_ms / args.steps
     value = ranks.whole_job_rate(macs_per_step, args.steps, total_ms, world)
@@ -316,23 +319,24 @@ def run_ours(args):
     achieved_gbs = bytes_per_launch / avg_launch_s / 1e9
     traffic = None
     rec = NCU_TRAFFIC.get("conv1d_packed_tc")
-    if rec and rec.get("sha256") == _source_hash("hikonv_conv1d_tc.cu"):
+    if args.algo == "packed" and rec and rec.get("sha256") == _source_hash("hikonv_conv1d_tc.cu"):
         traffic = rec["bytes_per_output"] * outputs_per_step / launches_per_step
     roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": hbm_peak_gbs, "unit": "GB/s",
                 "frac": achieved_gbs / hbm_peak_gbs, "traffic": traffic, "peak_kind": "of " + peak_kind,
-                "kernel": "conv1d_packed_tc_kernel", "bytes_per_output": 5,
+                "kernel": {"packed": "conv1d_packed_tc_kernel", "unpacked": "conv1d_unpacked_tc_kernel",
+                           "dp4a": "conv1d_dp4a_tc_kernel", "emu64": "conv1d_emu64_kernel"}[args.algo], "bytes_per_output": 5,
                 "traffic_note": "DRAM bytes per launch under ncu in steady state (six consecutive launches over rotating buffers, "
                                 "caches not flushed between them): 0.95 of the algorithmic bytes, nothing is re-read"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int64", "data": "synthetic",
+        "dtype": {"packed": "int64", "emu64": "int128"}.get(args.algo, "int32"), "data": "synthetic",
         "config": {"workload": "c2: 1-D bitwidth sweep, %d full convolutions of length 2^%d (p=q=1..8, K=3/5/7, unsigned+signed), "
                                "int8-stored codes in, int32 out" % (len(cases), length.bit_length() - 1),
                    "l2": "inputs larger than L2: every launch of a step has its own input and output buffers (%.1f GB per step)"
                          % ((outputs_per_step * 4 + len(cases) * length) / 1e9),
-                   "launch": "one CUDA graph replay per step"},
+                   "launch": "one CUDA graph replay per step", "algo": args.algo},
         "gpu_launches": args.steps * launches_per_step,
         "roofline": roofline,
     }
@@ -353,7 +357,7 @@ def run_ours(args):
             for i, (c, f, g) in enumerate(zip(cases, pin_f, pin_g)):
                 k = i % 2
                 hk.conv1d_host(f, g, c["p"], c["q"], c["f_signed"], c["g_signed"], pin_ys[k][: length + c["K"] - 1], wss[k],
-                               stream=streams[k])
+                               algo=main_algo, stream=streams[k])
 
         def e2e_run(steps):
             cur = torch.cuda.current_stream(dev)
@@ -419,6 +423,8 @@ def run_ours(args):
 def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank, local_rank, barrier, max_over_ranks, imad_peak):
     """Main line for --workload c3/c4/c5: a step is one layer (or one network pass) on this rank's batch,
     timed with one event pair per step and an L2 flush (256 MB memset) before each step."""
+    if args.algo not in ("packed", "unpacked"):
+        raise SystemExit("--algo %s exists for the 1-D sweep only" % args.algo)
     algo = hk.ALGO_PACKED32 if args.algo == "packed" else hk.ALGO_UNPACKED_IMAD
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     launches = 0
@@ -661,7 +667,8 @@ def main():
     ap.add_argument("--cases", default="", help="c2 only: comma-separated subset such as p4_K3_s,p8_K7_u (for profiling)")
     ap.add_argument("--case-copies", type=int, default=3, help="with --cases: buffer copies per case")
     ap.add_argument("--batch", type=int, default=0, help="c3/c4/c5: override the batch size (for profiling)")
-    ap.add_argument("--algo", default="packed", choices=["packed", "unpacked"], help="c3/c4/c5: which kernel the main line times")
+    ap.add_argument("--algo", default="packed", choices=["packed", "unpacked", "dp4a", "emu64"],
+                    help="which kernel the main line times (dp4a and emu64: the 1-D sweep only)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
