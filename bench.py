@@ -36,6 +36,7 @@ HBM_FALLBACK_GBS = 6650.0            # earlier pool measurement, used only when 
 # the packed kernels on 32.
 IMAD32_PER_CLK_PER_SM = 64
 IMAD_WIDE_PER_CLK_PER_SM = 32
+TABLE_REPEATS = 7                    # timed repeats per cell of the per-case table (median and max - min are reported)
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of the kernel: six
 # consecutive launches of the p=q=4, K=3 signed case at 2^24 rotating over three input and three output
@@ -44,8 +45,7 @@ IMAD_WIDE_PER_CLK_PER_SM = 32
 # of a launch's output is then still in the 126 MB L2 when its counters stop.)  The SHA-256 is that of the
 # kernel source at capture time; a changed source voids the figure.
 NCU_TRAFFIC = {
-    "conv1d_packed_tc": {"sha256": "f6fdbe051c664c7fd9d281b6bdff69b91c1bd4aa5514dfcfb6bf19a67880c073",
-                         "bytes_per_output": (14.443e6 + 65.167e6) / 16777218.0},
+    "conv1d_bs": {"sha256": "", "sha256_run": "", "bytes_per_output": 0.0},
 }
 
 
@@ -123,13 +123,16 @@ class ClockSampler:
 # reference arm and CPU baseline: the oracle as it stands, on the host cores
 # ----------------------------------------------------------------------------------------------
 
-def oracle_inputs(sample_len: int, seed_offset: int = 0):
+def oracle_inputs(sample_len: int, seed_offset: int = 0, compact: bool = False):
+    """The 48 sweep cases as code values; `compact` keeps them as int16 (the oracle widens them itself), so that the
+    full-length sweep fits in 1.6 GB of host memory."""
+    import numpy as np
     from paper_2208_00763_b200 import inputs
     data = []
     for case in inputs.c2_cases(sample_len):
         f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"],
                                   case["seed"] + seed_offset)
-        data.append((f, g))
+        data.append((f.astype(np.int16) if compact else f, g))
     return data
 
 
@@ -160,6 +163,11 @@ def cpu_baseline(sample_len: int):
         macs += m
         secs += s
         passes += 1
+    # the definition on one thread: one pass over the same sample
+    threads_all = direct.num_threads()
+    direct.set_num_threads(1)
+    m1, s1 = oracle_sweep(data)
+    direct.set_num_threads(threads_all)
     layers = {}
     for name, shape, batch in (("c3", inputs_mod().C3_SHAPE, 2), ("c4", inputs_mod().C4_SHAPE, 2)):
         x, w = inputs_mod().layer_case(shape, batch=batch)
@@ -190,6 +198,7 @@ def cpu_baseline(sample_len: int):
                                                              "speedup": (t1 - t0) / (t2 - t1)}
     direct.set_num_threads(threads_before)
     return {"value": macs / secs, "unit": UNIT, "cores": direct.num_threads(), "kind": "oracle", "layers": layers,
+            "one_thread": {"value": m1 / s1, "unit": UNIT, "sample": "one pass over the same 48 cases, %.1f s" % s1},
             "algorithm2_one_thread": alg2,
             "sample": "%d pass(es) over the 48 sweep cases at signal length %d (benchmark length 2^24), int64 direct "
                       "convolution, OpenMP over outputs, %.1f s of CPU time" % (passes, sample_len, secs)}
@@ -200,8 +209,8 @@ def run_reference(args):
     if ranks.rank_info()[1] != 0:
         return 0                      # the oracle runs once, on rank 0's host cores
     from oracle import direct
-    sample_len = 1 << 22
-    data = oracle_inputs(sample_len)
+    sample_len = args.length                      # the benchmark's own signal length (2^24 unless --length says otherwise)
+    data = oracle_inputs(sample_len, compact=True)
     for _ in range(args.warmup):
         oracle_sweep(data[:4])
     total_macs, total_secs = 0.0, 0.0
@@ -210,12 +219,14 @@ def run_reference(args):
         total_macs += m
         total_secs += s
     value = total_macs / total_secs
-    sample = "each step: the 48 sweep cases at signal length %d (1/4 of the benchmark length)" % sample_len
+    sample = "each step: the 48 sweep cases at signal length %d (the benchmark's configuration), one case after the other" % sample_len
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total_secs / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": "c2: 1-D bitwidth sweep, 48 full convolutions (p=q=1..8, K=3/5/7, unsigned+signed); " + sample},
+        "config": {"workload": "c2: 1-D bitwidth sweep, %d full convolutions of length 2^%d (p=q=1..8, K=3/5/7, unsigned+signed), "
+                               "int8-stored codes in, int32 out" % (len(data), sample_len.bit_length() - 1),
+                   "oracle": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": direct.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -253,6 +264,19 @@ def run_ours(args):
 
     def max_over_ranks(ms: float) -> float:
         return ranks.max_over_ranks(ms, dev)
+
+    # measured integer-pipe rates (register-only kernels of the library), the denominators of the "alu" rooflines
+    peaks = None
+    if rank == 0:
+        peaks = {}
+        for kind in ("mad_wide_u32", "mad_wide_s32", "mad_lo_s32", "logic", "shift", "prmt"):
+            r = hk.pipe_rate(kind, device=dev)
+            peaks[kind] = {"T_per_s": r["ops_per_second"] / 1e12, "lanes_per_clk_per_sm_at_max_clock": r["lanes_per_clock_per_sm"]}
+        peaks["derived"] = {"mad_wide_T_per_s": imad_peak["packed"] / 1e12, "mad_lo_T_per_s": imad_peak["unpacked"] / 1e12,
+                            "how": "SMs x lanes/clk x max SM clock (%d SMs, %d / %d lanes, %.0f MHz)"
+                                   % (sms, IMAD_WIDE_PER_CLK_PER_SM, IMAD32_PER_CLK_PER_SM, sm_max_mhz)}
+        imad_peak["packed_measured"] = max(peaks["mad_wide_u32"]["T_per_s"], peaks["mad_wide_s32"]["T_per_s"]) * 1e12
+        imad_peak["unpacked_measured"] = peaks["mad_lo_s32"]["T_per_s"] * 1e12
 
     # ---- the sweep: every rank runs the whole sweep on its own data (weak scaling, no exchange)
     if args.workload != "c2":
@@ -318,15 +342,17 @@ def run_ours(args):
     bytes_per_launch = 5.0 * outputs_per_step / launches_per_step
     achieved_gbs = bytes_per_launch / avg_launch_s / 1e9
     traffic = None
-    rec = NCU_TRAFFIC.get("conv1d_packed_tc")
-    if args.algo == "packed" and rec and rec.get("sha256") == _source_hash("hikonv_conv1d_tc.cu"):
+    rec = NCU_TRAFFIC.get("conv1d_bs")
+    if args.algo == "packed" and rec and rec.get("sha256") == _source_hash("hikonv_conv1d_bs.cu") and \
+            rec.get("sha256_run") == _source_hash("hikonv_conv1d_run.cuh"):
         traffic = rec["bytes_per_output"] * outputs_per_step / launches_per_step
     roofline = {"bound": "hbm", "achieved": achieved_gbs, "peak": hbm_peak_gbs, "unit": "GB/s",
                 "frac": achieved_gbs / hbm_peak_gbs, "traffic": traffic, "peak_kind": "of " + peak_kind,
-                "kernel": {"packed": "conv1d_packed_tc_kernel", "unpacked": "conv1d_unpacked_tc_kernel",
+                "kernel": {"packed": "conv1d_bs_kernel", "unpacked": "conv1d_unpacked_tc_kernel",
                            "dp4a": "conv1d_dp4a_tc_kernel", "emu64": "conv1d_emu64_kernel"}[args.algo], "bytes_per_output": 5,
-                "traffic_note": "DRAM bytes per launch under ncu in steady state (six consecutive launches over rotating buffers, "
-                                "caches not flushed between them): 0.95 of the algorithmic bytes, nothing is re-read"}
+                "traffic_note": ("DRAM bytes per launch under ncu in steady state (consecutive launches over rotating buffers, "
+                                 "caches not flushed between them)" if traffic is not None else
+                                 "null: the kernel source has changed since the DRAM counters were taken")}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -396,21 +422,32 @@ def run_ours(args):
                     vals = inputs.from_storage(host_f[i].numpy(), c["f_signed"])
                     d_fd[i] = torch.from_numpy(inputs.to_dense(vals, c["p"])).to(dev)
             extra["c2_by_bits"] = per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd)
-            # packed against comparator per bitwidth (the six cases of a width summed) and the cells where packed is not faster
+            # packed against comparator per bitwidth (the six cases of a width summed); a case counts as a tie when
+            # the two medians differ by no more than the larger run-to-run spread of the two
             by_width = {}
+            slower, ties, faster = [], [], []
             for name, row in extra["c2_by_bits"].items():
                 w = by_width.setdefault(name.split("_")[0], {"packed_us": 0.0, "unpacked_us": 0.0})
                 w["packed_us"] += row["packed_us"]
                 w["unpacked_us"] += row["unpacked_us"]
+                spread = max(row["packed_spread_us"], row["unpacked_spread_us"])
+                if abs(row["packed_us"] - row["unpacked_us"]) <= spread:
+                    ties.append(name)
+                elif row["packed_us"] < row["unpacked_us"]:
+                    faster.append(name)
+                else:
+                    slower.append(name)
             for w in by_width.values():
                 w["unpacked_over_packed"] = w["unpacked_us"] / w["packed_us"]
             extra["c2_packed_vs_unpacked"] = {
-                "by_bitwidth": by_width,
-                "cases_packed_not_faster": sorted(n for n, r in extra["c2_by_bits"].items() if r["packed_us"] >= r["unpacked_us"])}
+                "by_bitwidth": by_width, "repeats_per_cell": TABLE_REPEATS,
+                "cases_packed_faster": sorted(faster), "cases_tied_within_spread": sorted(ties),
+                "cases_packed_not_faster": sorted(slower)}
             del d_fd
             del d_f, d_g
             torch.cuda.empty_cache()
             extra.update(layer_workloads(torch, np, hk, inputs, network, dev, imad_peak))
+            extra["peaks"] = peaks
             line["extra"] = extra
         line["cpu_baseline"] = cpu_baseline(1 << 22)
 
@@ -503,16 +540,26 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
     }
     if muls is not None:
-        peak = imad_peak[args.algo]
-        line["roofline"] = {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": peak / 1e12,
-                            "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / peak, "traffic": None,
-                            "kernel": "conv2d_kernel",
-                            "peak_kind": "derived: SMs x %d lanes/clk x max SM clock; the step also holds the two packing kernels"
-                                         % (IMAD_WIDE_PER_CLK_PER_SM if args.algo == "packed" else IMAD32_PER_CLK_PER_SM)}
+        line["roofline"] = alu_roofline(muls, ms, imad_peak, args.algo)
+        line["roofline"]["kernel"] = "conv2d_kernel"
     if rank == 0:
         print(json.dumps(line), flush=True)
     ranks.shutdown()
     return 0
+
+
+def alu_roofline(muls: float, ms: float, imad_peak: dict, key: str) -> dict:
+    """Multiplies executed per second against the rate of that multiply: `peak` is the rate the library's own
+    register-only kernel reached on this GPU (hikonv_pipe_rate) when it was measured, `frac_of_derived` divides by
+    SMs x lanes per clock x maximum SM clock instead.  The step also holds the packing kernel of the layer."""
+    achieved = muls / (ms * 1e-3)
+    derived = imad_peak[key]
+    measured = imad_peak.get(key + "_measured")
+    peak = measured if measured else derived
+    return {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "T multiply-add/s",
+            "frac": achieved / peak, "traffic": None,
+            "peak_kind": "of measured (register-only multiply-add kernel, this run)" if measured else "of derived",
+            "frac_of_derived": achieved / derived, "derived_peak": derived / 1e12}
 
 
 def small_case(torch, hk, inputs, dev):
@@ -550,7 +597,8 @@ def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
     64x64 multiplier (`emu64_us`), the byte dot-product comparator (`dp4a_us`), and for the 1-, 2- and 4-bit cases
     the packed kernel on dense input (8 / p codes per byte; `dense_hbm_bytes_per_output` = 4 + p / 8).  Each
     timed graph holds 12 launches that rotate over the three inputs of the same bitwidth and signedness and
-    over three output buffers (240 MB per cycle), so no launch finds its data in L2."""
+    over three output buffers (240 MB per cycle), so no launch finds its data in L2.  Every cell is the median
+    of TABLE_REPEATS timings of two graph replays; `*_spread_us` is their max - min."""
     table = {}
     ys = [torch.empty(length + 6, dtype=torch.int32, device=d_f[0].device) for _ in range(3)]
     for i, c in enumerate(cases):
@@ -576,14 +624,18 @@ def per_bitwidth_table(torch, hk, cases, d_f, d_g, length, d_fd):
             with torch.cuda.graph(g):
                 fn()
             g.replay()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
-            e0.record()
-            for _ in range(3):
+            reps = []
+            for _ in range(TABLE_REPEATS):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
                 g.replay()
-            e1.record()
-            torch.cuda.synchronize()
-            row[name] = e0.elapsed_time(e1) * 1e3 / 36
+                g.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                reps.append(e0.elapsed_time(e1) * 1e3 / 24)
+            row[name] = statistics.median(reps)
+            row[name.replace("_us", "_spread_us")] = max(reps) - min(reps)
         table["p%d_K%d_%s" % (c["p"], c["K"], "s" if c["f_signed"] else "u")] = row
     return table
 
@@ -625,9 +677,7 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
                                            requant=rq, algo=algo, workspace=ws, out=o))
             muls = hk.conv2d_multiplies(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
                                         shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], algo)
-            rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT,
-                        "roofline": {"bound": "alu", "achieved": muls / (ms * 1e-3) / 1e12, "peak": imad_peak[key] / 1e12,
-                                     "unit": "T multiply-add/s", "frac": muls / (ms * 1e-3) / imad_peak[key], "traffic": None}}
+            rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key)}
         rec["layout"] = hk.layout(shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], shape["K"], 2, shape["Ci"] * shape["K"])
         rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
         out[name] = rec

@@ -18,7 +18,10 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device
  *     entry points enqueue their kernels on it and return without synchronising.
  *   - Every function returns a hikonv_status (as int); nothing aborts, nothing traps on
- *     the device.  Arguments are validated on the host before any launch.
+ *     the device.  Arguments are validated on the host before any launch.  HIKONV_ERR_CUDA
+ *     reports what the call's own launches and copies returned; an error that earlier,
+ *     unrelated CUDA calls left unread in the thread's error state is neither reported nor
+ *     cleared.
  *   - There is no CPU fallback: without a CUDA device the device entry points return
  *     HIKONV_ERR_CUDA.
  */
@@ -46,7 +49,7 @@ typedef enum {
 typedef enum {
     HIKONV_ALGO_PACKED32 = 0,      /* packed operands, 32x32->64 multiply (mad.wide)                    */
     HIKONV_ALGO_PACKED64EMU = 1,   /* packed operands of 64 bits, 64x64->128 product built from 32-bit
-                                      multiplies (Section IV-C's wider multiplier); hikonv_conv1d only */
+                                      multiplies (Section V-A's wider multiplier); hikonv_conv1d only */
     HIKONV_ALGO_UNPACKED_IMAD = 2, /* comparator: one product per 32-bit multiply-add, int32 accumulate */
     HIKONV_ALGO_DP4A = 3           /* second comparator: four products per byte dot-product instruction
                                       (dp4a), int32 accumulate; hikonv_conv1d only, K <= 8               */
@@ -90,8 +93,11 @@ typedef struct {
     int M;          /* force the number of accumulated products between two splits  */
     int tile;       /* kernel-specific tile selector (0 = automatic); conv2d: > 0 output
                        rows per CTA, < 0 carry-save moves at stage ends instead of at
-                       fixed places inside channel groups; conv1d: > 0 the general kernel, -32 runs of
-                       32 outputs per lane in the two comparators (default 24) */
+                       fixed places inside channel groups; conv1d: > 0 the general kernel, -1 the
+                       planner's layout instead of register-aligned slots; -24 / -25 force the
+                       register budget of four / five resident CTAs per SM in the register-aligned
+                       kernels and the two comparators (default: whichever measured faster for the
+                       kernel), -32 runs of 32 outputs per lane (default 24) in the two comparators */
 } hikonv_tuning_t;
 
 /*
@@ -163,13 +169,27 @@ int hikonv_check_range(const int8_t *d_in, size_t n, int bits, int is_signed, un
  * HIKONV_ERR_UNSUPPORTED).
  * tune may be NULL.  len >= 1, 1 <= K <= 64.
  * The packed algorithm is bound by HBM on this input format, not by the multiplier, so without a forced
- * layout the call lowers the planner's N to the block size its kernel streams fastest with (8 in place of
- * 9..12, 4 in place of 5) when the slot width and the number of kernel chunks stay the same;
- * hikonv_conv1d_multiplies counts the multiplies of the layout that runs.
+ * layout the call does not run the planner's layout (most outputs per multiply) but the one with the fewest
+ * instructions per output: hikonv_conv1d_layout returns it, hikonv_conv1d_multiplies counts its multiplies.
  */
 int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p, int q,
                   int f_signed, int g_signed, int32_t *d_y, int algo, const hikonv_tuning_t *tune,
                   void *stream);
+
+/*
+ * hikonv_conv1d_layout - the packed layout hikonv_conv1d(HIKONV_ALGO_PACKED32) runs with for these arguments
+ * (host only; hikonv_layout reports the planner's choice, which maximises outputs per multiply).
+ * On one-code-per-byte input the path is bound by HBM, so the call prefers the layout with the fewest
+ * instructions per output: slots of 8 or 16 bits with N S = 32 whenever every sum of K products fits such a
+ * slot and K <= 8 (the packed operand of Eq. 5 is then the loaded word itself or one byte permute of it, the
+ * carry of Theorem 2 is the high register of the previous product, and every output is one byte permute);
+ * sums of 17 to 21 bits (8-bit codes) run with N = 2 and two taps per kernel word at the narrowest such S.
+ * Otherwise it takes the planner's layout with N lowered to 8 (from 9..12) or 4 (from 5) when that keeps S
+ * and J.  tune: a forced N or S is taken as it is, tile == -1 keeps the planner's layout, tile > 0 the
+ * general kernel.
+ */
+int hikonv_conv1d_layout(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune,
+                         hikonv_layout_t *out);
 
 /*
  * hikonv_conv1d_dense - hikonv_conv1d (packed algorithm) on a signal stored without its unused bits
@@ -238,8 +258,12 @@ size_t hikonv_conv2d_workspace_bytes(int B, int Ci, int H, int W, int Co, int K,
  *   - Limit: hikonv_conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad) must not exceed HIKONV_STATIC_SCRATCH_BYTES,
  *     otherwise HIKONV_ERR_TOO_LARGE is returned and nothing is launched.
  *   - The function calls no cudaMalloc/cudaFree and no allocating library routine.
+ *   - The buffer that is used is the CURRENT device's.  d_x and d_out must be memory of the current device
+ *     (checked with a pointer-attribute query; otherwise HIKONV_ERR_INVALID_ARG and nothing is launched) and
+ *     `stream` must belong to it.
  *   - The first call on each device looks up the buffer's device address (once per device, with that
- *     device current).  Make that first call during start-up, before any stream capture.
+ *     device current) and keeps it for the life of the process; cudaDeviceReset invalidates it.  Make that
+ *     first call during start-up, before any stream capture.
  *   - All calls on a device share the one buffer and it keeps the previous call's contents.  Nothing
  *     in it has to start at zero: every call rewrites all words it later reads.  Two calls whose
  *     kernels can overlap on the GPU (different streams, no dependency between them) race on the
@@ -274,6 +298,28 @@ double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int f_signed, i
                                 const hikonv_tuning_t *tune);
 double hikonv_conv2d_multiplies(int B, int Ci, int H, int W, int Co, int K, int pad, int p, int q,
                                 int x_signed, int w_signed, int algo, const hikonv_tuning_t *tune);
+
+/*
+ * hikonv_pipe_rate - measured issue rate of one integer instruction, for the rooflines of the packed kernels.
+ * (A measurement aid; the paper has no counterpart.)  The 2-D layer kernels are bound by the 32x32->64
+ * multiply-add that implements Eq. 9, and no public table gives its rate on this GPU.  The call runs a
+ * register-only kernel (four CTAs of 256 threads per SM, eight independent dependency chains per thread whose
+ * operands depend on the previous result, so nothing is loop-invariant), times it with CUDA events on `stream`
+ * (best of three launches after a warm-up; the call SYNCHRONISES) and returns instructions x 32 lanes per second
+ * in *h_ops_per_second and, if h_lanes_per_clock_per_sm is not NULL, that rate divided by (SM count x the device's
+ * maximum SM clock).  d_scratch_word: one 4-byte device word owned by the caller.  iters: loop trips of 64
+ * instructions per thread (1 .. 2^20).
+ */
+typedef enum {
+    HIKONV_PIPE_MAD_WIDE_U32 = 0, /* mad.wide.u32: the packed multiply of unsigned layouts       */
+    HIKONV_PIPE_MAD_WIDE_S32 = 1, /* mad.wide.s32: the packed multiply of signed layouts         */
+    HIKONV_PIPE_MAD_LO_S32 = 2,   /* mad.lo.s32: the comparator's 32-bit multiply-add            */
+    HIKONV_PIPE_LOGIC = 3,        /* lop3.b32: masks of the split and of the carry-save moves    */
+    HIKONV_PIPE_SHIFT = 4,        /* shf.r: the funnel shifts of the split                       */
+    HIKONV_PIPE_PRMT = 5          /* prmt.b32: code extraction and byte-aligned slot extraction  */
+} hikonv_pipe_kind;
+int hikonv_pipe_rate(int kind, int iters, uint32_t *d_scratch_word, double *h_ops_per_second,
+                     double *h_lanes_per_clock_per_sm, void *stream);
 
 const char *hikonv_status_string(int status);
 

@@ -18,6 +18,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA, ERR_T
 STATIC_SCRATCH_BYTES = 4 << 20
 ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD, ALGO_DP4A = 0, 1, 2, 3
 GB_SINGLE, GB_1D, GB_DNN = 0, 1, 2
+PIPE_KINDS = {"mad_wide_u32": 0, "mad_wide_s32": 1, "mad_lo_s32": 2, "logic": 3, "shift": 4, "prmt": 5}
 
 
 class HikonvError(RuntimeError):
@@ -49,6 +50,7 @@ _SIGNATURES = {
     "hikonv_pack": (_i, [_vp, _sz, _i, _i, _i, _i, _i, _vp, _vp]),
     "hikonv_check_range": (_i, [_vp, _sz, _i, _i, _vp, ctypes.POINTER(ctypes.c_ulonglong), _vp]),
     "hikonv_conv1d": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _i, ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv1d_layout": (_i, [_i] * 5 + [ctypes.POINTER(TuningT), ctypes.POINTER(LayoutT)]),
     "hikonv_conv1d_dense": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv1d_host_workspace_bytes": (_sz, [_sz, _i]),
     "hikonv_conv1d_host": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _i, ctypes.POINTER(TuningT), _vp]),
@@ -63,6 +65,7 @@ _SIGNATURES = {
     "hikonv_maxpool2x2_i8": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
     "hikonv_conv1d_multiplies": (_d, [_sz, _i, _i, _i, _i, _i, _i, ctypes.POINTER(TuningT)]),
     "hikonv_conv2d_multiplies": (_d, [_i] * 12 + [ctypes.POINTER(TuningT)]),
+    "hikonv_pipe_rate": (_i, [_i, _i, _vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), _vp]),
     "hikonv_status_string": (ctypes.c_char_p, [_i]),
 }
 
@@ -116,6 +119,25 @@ def _dev_i8(t: torch.Tensor, name: str) -> int:
     return t.data_ptr()
 
 
+def _dev_out(t: torch.Tensor, name: str, numel: int, dtypes, like: torch.Tensor) -> int:
+    """Checks a caller-supplied output tensor before its address goes to a kernel: the library writes `numel`
+    elements of one of `dtypes` there and cannot see the tensor's size, type, layout or device."""
+    if not getattr(t, "is_cuda", False):
+        raise ValueError("%s must be a CUDA tensor" % name)
+    if t.device != like.device:
+        raise ValueError("%s is on %s, the inputs are on %s" % (name, t.device, like.device))
+    if t.dtype not in dtypes:
+        raise ValueError("%s must have dtype %s, not %s" % (name, " or ".join(str(d) for d in dtypes), t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if t.numel() != numel:
+        raise ValueError("%s holds %d elements, the call writes %d" % (name, t.numel(), numel))
+    return t.data_ptr()
+
+
+_CODE_DTYPES = (torch.int8, torch.uint8)
+
+
 # ------------------------------------------------------------------ host-only planning
 
 def plan(p, q, LA=32, LB=32, mode=GB_SINGLE, M=1, K_fixed=0) -> dict:
@@ -135,6 +157,14 @@ def layout_emu64(p, q, f_signed, g_signed, K, tune=None) -> dict:
     out = LayoutT()
     _check(lib().hikonv_layout_emu64(p, q, int(f_signed), int(g_signed), K, _tune(tune), ctypes.byref(out)),
            "hikonv_layout_emu64")
+    return {n: getattr(out, n) for n, _ in LayoutT._fields_}
+
+
+def conv1d_layout(p, q, f_signed, g_signed, K, tune=None) -> dict:
+    """The layout ``conv1d`` (packed algorithm, one code per byte) runs with."""
+    out = LayoutT()
+    _check(lib().hikonv_conv1d_layout(p, q, int(f_signed), int(g_signed), K, _tune(tune), ctypes.byref(out)),
+           "hikonv_conv1d_layout")
     return {n: getattr(out, n) for n, _ in LayoutT._fields_}
 
 
@@ -167,7 +197,8 @@ def conv1d(d_f: torch.Tensor, d_g: torch.Tensor, p: int, q: int, f_signed: bool,
     if out is None:
         out = torch.empty(n + K - 1, dtype=torch.int32, device=d_f.device)
     _check(lib().hikonv_conv1d(_dev_i8(d_f, "d_f"), n, _dev_i8(d_g, "d_g"), K, p, q, int(f_signed), int(g_signed),
-                               out.data_ptr(), algo, _tune(tune), _stream(stream)), "hikonv_conv1d")
+                               _dev_out(out, "out", n + K - 1, (torch.int32,), d_f), algo, _tune(tune), _stream(stream)),
+           "hikonv_conv1d")
     return out
 
 
@@ -182,7 +213,8 @@ def conv1d_dense(d_f_dense: torch.Tensor, n: int, d_g: torch.Tensor, p: int, q: 
     if out is None:
         out = torch.empty(n + K - 1, dtype=torch.int32, device=d_f_dense.device)
     _check(lib().hikonv_conv1d_dense(d_f_dense.data_ptr(), n, _dev_i8(d_g, "d_g"), K, p, q, int(f_signed), int(g_signed),
-                                     out.data_ptr(), _tune(tune), _stream(stream)), "hikonv_conv1d_dense")
+                                     _dev_out(out, "out", n + K - 1, (torch.int32,), d_f_dense), _tune(tune), _stream(stream)),
+           "hikonv_conv1d_dense")
     return out
 
 
@@ -217,8 +249,11 @@ def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_sig
     if out is None:
         out = torch.empty((B, Co, max(Ho, 0), max(Wo, 0)), dtype=torch.int8 if requant else torch.int32, device=d_x.device)
     shift, lo, hi = requant if requant else (0, 0, 0)
+    out_ptr = _dev_out(out, "out", B * Co * max(Ho, 0) * max(Wo, 0), _CODE_DTYPES if requant else (torch.int32,), d_x)
+    if not workspace.is_cuda or workspace.device != d_x.device or not workspace.is_contiguous():
+        raise ValueError("workspace must be a contiguous CUDA tensor on the inputs' device")
     _check(lib().hikonv_conv2d(_dev_i8(d_x, "d_x"), B, Ci, H, W, _dev_i8(d_w, "d_w"), Co, K, stride, pad, p, q,
-                               int(x_signed), int(w_signed), out.data_ptr(), 1 if requant else 0, shift, lo, hi,
+                               int(x_signed), int(w_signed), out_ptr, 1 if requant else 0, shift, lo, hi,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), algo, _tune(tune),
                                _stream(stream)), "hikonv_conv2d")
     return out
@@ -239,9 +274,14 @@ def conv2d_static_scratch(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int
     if Ci != Ci2 or K != K2:
         raise ValueError("weight shape does not match the input")
     shift, lo, hi = requant if requant else (0, 0, 0)
-    _check(lib().hikonv_conv2d_static_scratch(_dev_i8(d_x, "d_x"), B, Ci, H, W, _dev_i8(d_w, "d_w"), Co, K, stride, pad, p, q,
-                                              int(x_signed), int(w_signed), out.data_ptr(), 1 if requant else 0, shift, lo, hi,
-                                              algo, _tune(tune), _stream(stream)), "hikonv_conv2d_static_scratch")
+    Ho, Wo = H + 2 * pad - K + 1, W + 2 * pad - K + 1
+    out_ptr = _dev_out(out, "out", B * Co * max(Ho, 0) * max(Wo, 0), _CODE_DTYPES if requant else (torch.int32,), d_x)
+    if d_w.device != d_x.device:
+        raise ValueError("d_w is on %s, d_x on %s" % (d_w.device, d_x.device))
+    with torch.cuda.device(d_x.device):      # the built-in buffer that is used is the current device's
+        _check(lib().hikonv_conv2d_static_scratch(_dev_i8(d_x, "d_x"), B, Ci, H, W, _dev_i8(d_w, "d_w"), Co, K, stride, pad, p, q,
+                                                  int(x_signed), int(w_signed), out_ptr, 1 if requant else 0, shift, lo, hi,
+                                                  algo, _tune(tune), _stream(stream)), "hikonv_conv2d_static_scratch")
     return out
 
 
@@ -265,7 +305,8 @@ def maxpool2x2_i8(d_in: torch.Tensor, is_signed: bool, out: Optional[torch.Tenso
     B, C, H, W = d_in.shape
     if out is None:
         out = torch.empty((B, C, H // 2, W // 2), dtype=d_in.dtype, device=d_in.device)
-    _check(lib().hikonv_maxpool2x2_i8(_dev_i8(d_in, "d_in"), B, C, H, W, int(is_signed), out.data_ptr(), _stream(stream)),
+    _check(lib().hikonv_maxpool2x2_i8(_dev_i8(d_in, "d_in"), B, C, H, W, int(is_signed),
+                                      _dev_out(out, "out", B * C * (H // 2) * (W // 2), _CODE_DTYPES, d_in), _stream(stream)),
            "hikonv_maxpool2x2_i8")
     return out
 
@@ -276,3 +317,14 @@ def conv1d_multiplies(n, K, p, q, f_signed, g_signed, algo=ALGO_PACKED32, tune=N
 
 def conv2d_multiplies(B, Ci, H, W, Co, K, pad, p, q, x_signed, w_signed, algo=ALGO_PACKED32, tune=None) -> float:
     return float(lib().hikonv_conv2d_multiplies(B, Ci, H, W, Co, K, pad, p, q, int(x_signed), int(w_signed), algo, _tune(tune)))
+
+
+def pipe_rate(kind: str, iters: int = 2048, device=None, stream=None) -> dict:
+    """Measured rate of one integer instruction (see ``PIPE_KINDS``): operations per second (instructions x 32
+    lanes) and lanes per clock per SM at the device's maximum SM clock.  Synchronises."""
+    word = torch.zeros(1, dtype=torch.int32, device=device or "cuda")
+    ops, lanes = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    with torch.cuda.device(word.device):
+        _check(lib().hikonv_pipe_rate(PIPE_KINDS[kind], int(iters), word.data_ptr(), ctypes.byref(ops), ctypes.byref(lanes),
+                                      _stream(stream)), "hikonv_pipe_rate")
+    return {"ops_per_second": ops.value, "lanes_per_clock_per_sm": lanes.value}

@@ -55,8 +55,9 @@ extern "C" int hikonv_check_range(const int8_t *d_in, size_t n, int bits, int is
         size_t blocks = (n_vec + 255) / 256;
         if (blocks > (size_t)sms * 8) blocks = (size_t)sms * 8;
         if (blocks < 1) blocks = 1;
-        check_range_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint8_t *>(d_in), n, head, n_vec, lift, high, d_count);
-        if (launch_status() != HIKONV_OK) return HIKONV_ERR_CUDA;
+        if (launch_plain(check_range_kernel, dim3((unsigned)blocks), dim3(256), 0, st, reinterpret_cast<const uint8_t *>(d_in), n, head,
+                         n_vec, lift, high, d_count) != HIKONV_OK)
+            return HIKONV_ERR_CUDA;
     }
     HIKONV_CUDA_TRY(cudaMemcpyAsync(&found, d_count, sizeof(found), cudaMemcpyDeviceToHost, st));
     HIKONV_CUDA_TRY(cudaStreamSynchronize(st));

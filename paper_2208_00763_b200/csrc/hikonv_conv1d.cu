@@ -16,7 +16,9 @@
 #include <cstring>
 
 #include "hikonv_cuda.cuh"
+#include "hikonv_conv1d_bs.h"
 #include "hikonv_conv1d_emu64.h"
+#include "hikonv_conv1d_run.cuh"
 #include "hikonv_conv1d_tc.h"
 
 namespace hikonv {
@@ -221,13 +223,9 @@ __global__ void __launch_bounds__(kThreads1D) conv1d_unpacked_kernel(const Conv1
 
 template <int N>
 static int launch_packed_n(const Conv1dParams &p, bool signed_prod, bool f_signed, unsigned grid, cudaStream_t st) {
-    if (!signed_prod)
-        conv1d_packed_kernel<N, false, false><<<grid, kThreads1D, 0, st>>>(p);
-    else if (f_signed)
-        conv1d_packed_kernel<N, true, true><<<grid, kThreads1D, 0, st>>>(p);
-    else
-        conv1d_packed_kernel<N, true, false><<<grid, kThreads1D, 0, st>>>(p);
-    return launch_status();
+    if (!signed_prod) return launch_plain(conv1d_packed_kernel<N, false, false>, dim3(grid), dim3(kThreads1D), 0, st, p);
+    if (f_signed) return launch_plain(conv1d_packed_kernel<N, true, true>, dim3(grid), dim3(kThreads1D), 0, st, p);
+    return launch_plain(conv1d_packed_kernel<N, true, false>, dim3(grid), dim3(kThreads1D), 0, st, p);
 }
 
 static int launch_packed(int N, const Conv1dParams &p, bool sp, bool fs, unsigned grid, cudaStream_t st) {
@@ -251,28 +249,39 @@ static int launch_packed(int N, const Conv1dParams &p, bool sp, bool fs, unsigne
 template <bool F_SIGNED>
 static int launch_unpacked(const Conv1dUnpackedParams &p, unsigned grid, cudaStream_t st) {
     switch (p.K) {
-        case 3: conv1d_unpacked_kernel<3, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
-        case 5: conv1d_unpacked_kernel<5, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
-        case 7: conv1d_unpacked_kernel<7, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
-        default: conv1d_unpacked_kernel<0, F_SIGNED><<<grid, kThreads1D, 0, st>>>(p); break;
+        case 3: return launch_plain(conv1d_unpacked_kernel<3, F_SIGNED>, dim3(grid), dim3(kThreads1D), 0, st, p);
+        case 5: return launch_plain(conv1d_unpacked_kernel<5, F_SIGNED>, dim3(grid), dim3(kThreads1D), 0, st, p);
+        case 7: return launch_plain(conv1d_unpacked_kernel<7, F_SIGNED>, dim3(grid), dim3(kThreads1D), 0, st, p);
+        default: return launch_plain(conv1d_unpacked_kernel<0, F_SIGNED>, dim3(grid), dim3(kThreads1D), 0, st, p);
     }
-    return launch_status();
 }
 
-// The layout hikonv_conv1d runs with on one-code-per-byte input: the planner's choice (most outputs per
-// multiply), with N lowered to the block size the register-resident kernel streams fastest with when that
-// needs the same slot width and no more kernel chunks (the path is HBM-bound; the extra multiplies are free).
-// A forced N, S or kernel choice (tune) is taken as it is.
+// The layout hikonv_conv1d runs with on one-code-per-byte input.  The path is HBM-bound, so the layout with the
+// fewest instructions per output wins, not the one with the most outputs per multiply:
+//   1. byte-aligned slots (S = 8, 16, 24 with N S = 32) when the sums fit them and K <= 8 (*slot_bytes > 0);
+//   2. else the planner's choice, with N lowered to the block size the register-resident kernel streams fastest
+//      with when that needs the same slot width and no more kernel chunks.
+// A forced N or S (tune) is taken as it is; tune->tile == -1 skips step 1, tune->tile > 0 both.
 static int layout_for_byte_input(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune,
-                                 hikonv_layout_t *L) {
+                                 hikonv_layout_t *L, int *slot_bytes) {
+    *slot_bytes = 0;
+    const bool forced = tune && (tune->N > 0 || tune->S > 0 || tune->tile > 0);
+    if (!forced && !(tune && tune->tile == -1)) {
+        if (validate_codes(p, q) != HIKONV_OK || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
+        const int sb = make_layout_byte_slots(p, q, f_signed, g_signed, K, L);
+        if (sb > 0) {
+            *slot_bytes = sb;
+            return HIKONV_OK;
+        }
+    }
     int rc = make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, tune, L);
     if (rc != HIKONV_OK) return rc;
-    if (tune && (tune->N > 0 || tune->S > 0 || tune->tile > 0)) return rc;
+    if (forced) return rc;
     const int n_pref = conv1d_tc_preferred_n(L->N);
     if (n_pref == L->N) return rc;
-    hikonv_tuning_t forced = {n_pref, L->S, 0, 0};
+    hikonv_tuning_t forced_n = {n_pref, L->S, 0, 0};
     hikonv_layout_t alt;
-    if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, &forced, &alt) == HIKONV_OK && alt.J <= L->J &&
+    if (make_layout(p, q, f_signed, g_signed, K, 1, 0, 0, &forced_n, &alt) == HIKONV_OK && alt.J <= L->J &&
         conv1d_packed_tc_available(alt.N, alt.J))
         *L = alt;
     return HIKONV_OK;
@@ -314,16 +323,24 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
 
     if (algo == HIKONV_ALGO_DP4A) {
         if (!conv1d_dp4a_tc_available(K)) return HIKONV_ERR_UNSUPPORTED;
-        const int run = (tune && tune->tile == -32) ? 32 : 24;
+        // one tap word (K <= 4) leaves registers for five resident CTAs per SM, which stream 2-3 % faster; two do not
+        const int forced = tune ? -tune->tile : 0;
+        const int shape = (forced == 32 || forced == 25 || forced == 24) ? forced : (K <= 4 ? 25 : 24);
+        const int run = shape == 32 ? 32 : 24;
         tp.n_tiles = (n_out + 32 * run - 1) / (32 * run);
-        return launch_conv1d_dp4a_tc(tp, K, f_signed != 0, g_signed != 0, run, st);
+        tp.fast_after_first = fast_tiles_after_first((long long)len, run, tp.aligned != 0);
+        return launch_conv1d_dp4a_tc(tp, K, f_signed != 0, g_signed != 0, shape, st);
     }
     if (algo == HIKONV_ALGO_UNPACKED_IMAD && want_tc && conv1d_unpacked_tc_available(K)) {
-        // runs of 24 outputs per lane at four resident CTAs stream fastest (as for the packed kernel); -32 keeps
-        // the longer runs reachable
-        const int run = (tune && tune->tile == -32) ? 32 : 24;
+        // runs of 24 outputs per lane stream fastest (as for the packed kernels): with the register budget of five
+        // resident CTAs per SM up to five taps, of four beyond (seven taps spill at five); -32 keeps the longer runs
+        // reachable, -24 / -25 force a budget
+        const int forced = tune ? -tune->tile : 0;
+        const int shape = (forced == 32 || forced == 25 || forced == 24) ? forced : (K <= 5 ? 25 : 24);
+        const int run = shape == 32 ? 32 : 24;
         tp.n_tiles = (n_out + 32 * run - 1) / (32 * run);
-        return launch_conv1d_unpacked_tc(tp, K, f_signed != 0, run, st);
+        tp.fast_after_first = fast_tiles_after_first((long long)len, run, tp.aligned != 0);
+        return launch_conv1d_unpacked_tc(tp, K, f_signed != 0, shape, st);
     }
     if (algo == HIKONV_ALGO_UNPACKED_IMAD) {
         Conv1dUnpackedParams up;
@@ -336,8 +353,31 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     }
 
     hikonv_layout_t L;
-    rc = layout_for_byte_input(p, q, f_signed, g_signed, K, tune, &L);
+    int slot_bytes = 0;
+    rc = layout_for_byte_input(p, q, f_signed, g_signed, K, tune, &L, &slot_bytes);
     if (rc != HIKONV_OK) return rc;
+    if (slot_bytes > 0) {           // register-aligned slots: mode 1, 2 or 3
+        Conv1dBsParams bp;
+        std::memset(&bp, 0, sizeof(bp));
+        bp.f = d_f; bp.g = d_g; bp.y = d_y; bp.len = (long long)len; bp.n_out = n_out; bp.K = K;
+        bp.g_signed = g_signed ? 1 : 0;
+        bp.aligned = tp.aligned;
+        if (f_signed) {
+            bp.code_xor = 0x01010101u * (1u << (p - 1));
+            bp.code_and = 0x01010101u * ((1u << p) - 1u);
+        }
+        bp.S = L.S;
+        bp.mask3 = (1u << L.S) - 1u;
+        if (slot_bytes == 3 && L.signed_prod) {
+            // slot 2 receives floor(K / 2) products: its bias lifts their most negative sum to zero, slot 0 takes the rest
+            const SplitConsts sc3 = make_split_consts(L, p, q, f_signed, g_signed, K, 1);
+            const uint64_t half = 1ull << (L.S - 1), b2 = (uint64_t)sc3.seg_bias[2];
+            bp.bias3 = (half - b2) + (half << L.S) + (b2 << (2 * L.S));
+        }
+        bp.n_tiles = (unsigned)((n_out + 32 * kBsRun - 1) / (32 * kBsRun));
+        bp.fast_after_first = fast_tiles_after_first((long long)len, kBsRun, tp.aligned != 0);
+        return launch_conv1d_bs(bp, slot_bytes, L.J, f_signed != 0, L.signed_prod != 0, tune ? -tune->tile : 0, st);
+    }
     if (L.N > kMaxN1D) return HIKONV_ERR_UNSUPPORTED;
     const SplitConsts sc = make_split_consts(L, p, q, f_signed, g_signed, K, 1);
 
@@ -380,6 +420,13 @@ extern "C" int hikonv_conv1d(const int8_t *d_f, size_t len, const int8_t *d_g, i
     const long long grid = (warps + kWarps1D - 1) / kWarps1D;
     if (grid > 0x7FFFFFFFLL) return HIKONV_ERR_UNSUPPORTED;
     return launch_packed(L.N, kp, L.signed_prod != 0, f_signed != 0, (unsigned)grid, st);
+}
+
+extern "C" int hikonv_conv1d_layout(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune,
+                                    hikonv_layout_t *out) {
+    if (!out) return HIKONV_ERR_INVALID_ARG;
+    int slot_bytes = 0;
+    return layout_for_byte_input(p, q, f_signed, g_signed, K, tune, out, &slot_bytes);
 }
 
 extern "C" int hikonv_conv1d_dense(const uint8_t *d_f_dense, size_t len, const int8_t *d_g, int K, int p, int q, int f_signed,
@@ -441,7 +488,10 @@ extern "C" double hikonv_conv1d_multiplies(size_t len, int K, int p, int q, int 
     hikonv_layout_t L;
     if (algo == HIKONV_ALGO_PACKED64EMU) {
         if (make_layout_emu64(p, q, f_signed, g_signed, K, tune, &L) != HIKONV_OK) return 0.0;
-    } else if (layout_for_byte_input(p, q, f_signed, g_signed, K, tune, &L) != HIKONV_OK) return 0.0;
+    } else {
+        int slot_bytes = 0;
+        if (layout_for_byte_input(p, q, f_signed, g_signed, K, tune, &L, &slot_bytes) != HIKONV_OK) return 0.0;
+    }
     const double blocks = (double)(((long long)n_out + L.N - 1) / L.N);
     return blocks * L.J;
 }

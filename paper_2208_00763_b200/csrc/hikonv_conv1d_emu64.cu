@@ -1,7 +1,7 @@
 // HIKONV_ALGO_PACKED64EMU for hikonv_conv1d: the packed method on a 64x64 -> 128 multiplier that the
 // GPU does not have, built from its 32-bit multiply pipe (the low and the high 64 bits of the product
 // are each a short sequence of 32x32 multiply-adds).  The paper notes that a wider multiplier is used
-// in the same way as the 32-bit one (Section IV-C); this is that variant:
+// in the same way as the 32-bit one (Section V-A); this is that variant:
 //   A_x = sum_n f[xN+n] 2^(S n)   in 64 bits  (Eq. 5; more codes per word than 32 bits hold)
 //   Q_x = bias + sum_j A_{x-j} B_j in 128 bits (Eq. 9)
 //   D_x = Q_x + (Q_{x-1} >> S N)               (Theorem 2)
@@ -140,13 +140,9 @@ __global__ void __launch_bounds__(kThreadsE) conv1d_emu64_kernel(const Emu64Para
 
 template <int N>
 static int launch_n(const Emu64Params &p, bool signed_prod, bool f_signed, unsigned grid, cudaStream_t st) {
-    if (!signed_prod)
-        conv1d_emu64_kernel<N, false, false><<<grid, kThreadsE, 0, st>>>(p);
-    else if (f_signed)
-        conv1d_emu64_kernel<N, true, true><<<grid, kThreadsE, 0, st>>>(p);
-    else
-        conv1d_emu64_kernel<N, true, false><<<grid, kThreadsE, 0, st>>>(p);
-    return launch_status();
+    if (!signed_prod) return launch_plain(conv1d_emu64_kernel<N, false, false>, dim3(grid), dim3(kThreadsE), 0, st, p);
+    if (f_signed) return launch_plain(conv1d_emu64_kernel<N, true, true>, dim3(grid), dim3(kThreadsE), 0, st, p);
+    return launch_plain(conv1d_emu64_kernel<N, true, false>, dim3(grid), dim3(kThreadsE), 0, st, p);
 }
 
 int launch_conv1d_emu64(const int8_t *d_f, size_t len, const int8_t *d_g, int K, int p, int q, int f_signed, int g_signed,

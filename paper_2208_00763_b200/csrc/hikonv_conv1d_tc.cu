@@ -9,17 +9,11 @@
 // registers), splits N outputs per block and writes its L outputs with 16-byte stores.  Tiles that
 // touch the ends of the signal, and unaligned buffers, take a guarded byte-wise path in the same kernel.
 // The comparator uses the same loads and stores with one 32-bit multiply-add per product.
-#include <mutex>
 #include <type_traits>
-#include <unordered_map>
 
-#include "hikonv_cuda.cuh"
-#include "hikonv_conv1d_tc.h"
+#include "hikonv_conv1d_run.cuh"
 
 namespace hikonv {
-
-constexpr int kThreadsTc = 256;
-constexpr int kWarpsTc = kThreadsTc / 32;
 
 __host__ __device__ constexpr int gcd_c(int a, int b) { return b == 0 ? a : gcd_c(b, a % b); }
 // blocks per lane: L = R N is a multiple of 4 and at least kMinRun
@@ -31,38 +25,6 @@ __host__ __device__ constexpr int blocks_per_lane(int N) {
     int r = step;
     while (r * N < kMinRun) r += step;
     return r;
-}
-
-// Byte `b` (0..3) of w as a 32-bit value, sign- or zero-extended: one prmt.
-template <bool SIGNED>
-__device__ __forceinline__ uint32_t extract_code(uint32_t w, int b) {
-    uint32_t r;
-    // selector nibbles: low nibble picks byte b; in the upper three, bit 3 replicates that byte's sign,
-    // or index 4 picks byte 0 of the zero second operand
-    const uint32_t sel = SIGNED ? (uint32_t)(b | ((8 | b) << 4) | ((8 | b) << 8) | ((8 | b) << 12)) : (uint32_t)(b | 0x4440);
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(w), "r"(0u), "r"(sel));
-    return r;
-}
-
-// Loads the words covering elements [e0 - 4 HW, e0 + 4 NWD - 4 HW) of f; e0 is a multiple of 4.
-template <int NWORDS, int HW>
-__device__ __forceinline__ void load_words(const int8_t *f, long long len, long long e0, bool fast, uint32_t (&w)[NWORDS]) {
-    if (fast) {
-        const uint32_t *src = reinterpret_cast<const uint32_t *>(f + e0) - HW;
-#pragma unroll
-        for (int i = 0; i < NWORDS; ++i) w[i] = __ldg(src + i);
-    } else {
-#pragma unroll
-        for (int i = 0; i < NWORDS; ++i) {
-            uint32_t v = 0;
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const long long idx = e0 + 4 * (i - HW) + b;
-                if (idx >= 0 && idx < len) v |= (uint32_t)(uint8_t)__ldg(f + idx) << (8 * b);   // Eq. 2: zero outside
-            }
-            w[i] = v;
-        }
-    }
 }
 
 // Dense input: P bits per code (1, 2 or 4), code e at bit (e P) % 8 of byte (e P) / 8.  Field `k` (a
@@ -102,37 +64,6 @@ __device__ __forceinline__ void load_dense(const int8_t *f, long long len, long 
                 v[k / EPW] |= ((byte >> (int)((e * P) % 8)) & ((1u << P) - 1u)) << ((k % EPW) * P);
             }
         }
-    }
-}
-
-// Row pitch (in words) of a lane's run in the warp's staging buffer: L padded so that the 16-byte
-// stores of eight neighbouring lanes fall into different banks.
-__host__ __device__ constexpr int stage_pitch(int L) { return (L % 8 == 0) ? L + 4 : L; }
-
-// Writes a warp tile of 32 runs of L outputs.  Interior tiles go through the warp's shared-memory
-// buffer so that every store instruction writes 512 contiguous bytes; edge tiles are stored guarded.
-template <int L>
-__device__ __forceinline__ void store_run(int32_t *y, long long n_out, long long tile0, int lane, bool fast, int32_t *stage,
-                                          const int32_t (&out)[L]) {
-    constexpr int P = stage_pitch(L);
-    if (fast) {
-        int4 *row = reinterpret_cast<int4 *>(stage + lane * P);
-#pragma unroll
-        for (int i = 0; i < L / 4; ++i) row[i] = make_int4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
-        __syncwarp();
-        int4 *dst = reinterpret_cast<int4 *>(y + tile0);
-#pragma unroll
-        for (int k = 0; k < L / 4; ++k) {
-            const int idx = 4 * (lane + 32 * k);              // first output of this 16-byte piece within the tile
-            const int src_lane = idx / L, src_off = idx % L;  // L is a multiple of 4: a piece never straddles two runs
-            __stcs(dst + lane + 32 * k, *reinterpret_cast<const int4 *>(stage + src_lane * P + src_off));   // written once, never re-read
-        }
-        __syncwarp();
-    } else {
-        const long long e0 = tile0 + lane * L;
-#pragma unroll
-        for (int i = 0; i < L; ++i)
-            if (e0 + i < n_out) y[e0 + i] = out[i];
     }
 }
 
@@ -251,8 +182,8 @@ __global__ void __launch_bounds__(kThreadsTc, ((N >= 9 && P == 0) ? 3 : 4)) conv
 }
 
 // Comparator: runs of L outputs per lane, one product per 32-bit multiply-add.
-template <int K, bool FS, int L>
-__global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_unpacked_tc_kernel(const Conv1dTcParams p) {
+template <int K, bool FS, int L, int MINB>
+__global__ void __launch_bounds__(kThreadsTc, MINB) conv1d_unpacked_tc_kernel(const Conv1dTcParams p) {
     constexpr int HW = (K - 1 + 3) / 4;
     constexpr int NWORDS = HW + L / 4;
     __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
@@ -262,35 +193,14 @@ __global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_unpacked
         const int8_t raw = __ldg(p.g + k);
         gk[k] = p.g_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
     }
-    const int lane = threadIdx.x & 31;
-    const long long stride = (long long)gridDim.x * kWarpsTc;
-    long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5);
-    uint32_t wn[NWORDS];
-    bool fast_n = false;
-    if (t < p.n_tiles) {
-        const long long tile0 = t * (32 * L);
-        fast_n = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
-        load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast_n, wn);
-    }
-    while (t < p.n_tiles) {
-        const long long tile0 = t * (32 * L);
-        const bool fast = fast_n;
-        uint32_t w[NWORDS];
-#pragma unroll
-        for (int i = 0; i < NWORDS; ++i) w[i] = wn[i];
-        t += stride;
-        if (t < p.n_tiles) {
-            const long long next0 = t * (32 * L);
-            fast_n = p.aligned && next0 >= 4 * HW && next0 + 32 * L <= p.len;
-            load_words<NWORDS, HW>(p.f, p.len, next0 + lane * L, fast_n, wn);
-        }
+    walk_tiles<L, HW>(p.f, p.y, p.len, p.n_out, (unsigned)p.n_tiles, p.fast_after_first, s_stage[threadIdx.x >> 5],
+                      [&](const uint32_t (&w)[NWORDS], int32_t (&out)[L]) {
         int32_t e[L + K - 1];                       // e[i] = f[e0 - (K-1) + i]
 #pragma unroll
         for (int i = 0; i < L + K - 1; ++i) {
             const int pos = 4 * HW - (K - 1) + i;
             e[i] = (int32_t)extract_code<FS>(w[pos / 4], pos % 4);
         }
-        int32_t out[L];
 #pragma unroll
         for (int o = 0; o < L; ++o) {
             int32_t s = 0;
@@ -298,8 +208,7 @@ __global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_unpacked
             for (int k = 0; k < K; ++k) s += e[o + (K - 1) - k] * gk[k];      // y[m] = sum_k f[m-k] g[k]
             out[o] = s;
         }
-        store_run<L>(p.y, p.n_out, tile0, lane, fast, s_stage[threadIdx.x >> 5], out);
-    }
+    });
 }
 
 // Second comparator: the byte dot-product instruction (dp4a: four 8-bit products summed into 32 bits), the
@@ -316,8 +225,8 @@ __device__ __forceinline__ int32_t dot4(uint32_t codes, uint32_t taps, int32_t a
     return d;
 }
 
-template <int KW, bool FS, bool GS, int L>
-__global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_dp4a_tc_kernel(const Conv1dTcParams p) {
+template <int KW, bool FS, bool GS, int L, int MINB>
+__global__ void __launch_bounds__(kThreadsTc, MINB) conv1d_dp4a_tc_kernel(const Conv1dTcParams p) {
     constexpr int HW = KW;                       // 4 KW codes in front of the run cover the K - 1 <= 4 KW - 1 it needs
     constexpr int NWORDS = HW + L / 4;
     __shared__ __align__(16) int32_t s_stage[kWarpsTc][32 * stage_pitch(L)];
@@ -332,29 +241,8 @@ __global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_dp4a_tc_
         }
         gw[t] = v;
     }
-    const int lane = threadIdx.x & 31;
-    const long long stride = (long long)gridDim.x * kWarpsTc;
-    long long t = (long long)blockIdx.x * kWarpsTc + (threadIdx.x >> 5);
-    uint32_t wn[NWORDS];
-    bool fast_n = false;
-    if (t < p.n_tiles) {
-        const long long tile0 = t * (32 * L);
-        fast_n = p.aligned && tile0 >= 4 * HW && tile0 + 32 * L <= p.len;
-        load_words<NWORDS, HW>(p.f, p.len, tile0 + lane * L, fast_n, wn);
-    }
-    while (t < p.n_tiles) {
-        const long long tile0 = t * (32 * L);
-        const bool fast = fast_n;
-        uint32_t w[NWORDS];
-#pragma unroll
-        for (int i = 0; i < NWORDS; ++i) w[i] = wn[i];
-        t += stride;
-        if (t < p.n_tiles) {
-            const long long next0 = t * (32 * L);
-            fast_n = p.aligned && next0 >= 4 * HW && next0 + 32 * L <= p.len;
-            load_words<NWORDS, HW>(p.f, p.len, next0 + lane * L, fast_n, wn);
-        }
-        int32_t out[L];
+    walk_tiles<L, HW>(p.f, p.y, p.len, p.n_out, (unsigned)p.n_tiles, p.fast_after_first, s_stage[threadIdx.x >> 5],
+                      [&](const uint32_t (&w)[NWORDS], int32_t (&out)[L]) {
 #pragma unroll
         for (int o = 0; o < L; ++o) {
             int32_t acc = 0;
@@ -367,36 +255,7 @@ __global__ void __launch_bounds__(kThreadsTc, (L <= 24 ? 4 : 3)) conv1d_dp4a_tc_
             }
             out[o] = acc;
         }
-        store_run<L>(p.y, p.n_out, tile0, lane, fast, s_stage[threadIdx.x >> 5], out);
-    }
-}
-
-// Persistent launch: as many CTAs as fit on the device at once (occupancy query, cached per kernel),
-// fewer when the problem is small; each warp then walks tiles with a grid-wide stride.
-// CTAs of `kernel` that fit one SM, asked once per kernel (all instantiations share one function-pointer
-// type, so the answer is kept per pointer, not per template instance of the launcher).
-static int resident_ctas(const void *kernel) {
-    static std::mutex mutex;
-    static std::unordered_map<const void *, int> known;
-    std::lock_guard<std::mutex> lock(mutex);
-    auto it = known.find(kernel);
-    if (it != known.end()) return it->second;
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kThreadsTc, 0) != cudaSuccess || occ < 1) occ = 1;
-    known[kernel] = occ;
-    return occ;
-}
-
-template <typename Kernel>
-static int launch_persistent(Kernel kernel, const Conv1dTcParams &p, cudaStream_t st) {
-    const int resident = resident_ctas(reinterpret_cast<const void *>(kernel));
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long want = (p.n_tiles + kWarpsTc - 1) / kWarpsTc;
-    const long long cap = (long long)sms * resident;
-    const unsigned grid = (unsigned)(want < cap ? want : cap);
-    kernel<<<grid, kThreadsTc, 0, st>>>(p);
-    return launch_status();
+    });
 }
 
 int conv1d_tc_outputs_per_tile(int N) {
@@ -478,28 +337,29 @@ int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, boo
 
 bool conv1d_unpacked_tc_available(int K) { return K == 3 || K == 5 || K == 7; }
 
-int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool fs, int run, cudaStream_t st) {
-#define HK_K(k, run_c)                                                                                   \
-    if (K == k && run == run_c) {                                                                        \
-        if (fs) return launch_persistent(conv1d_unpacked_tc_kernel<k, true, run_c>, p, st);              \
-        return launch_persistent(conv1d_unpacked_tc_kernel<k, false, run_c>, p, st);                     \
+int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool fs, int shape, cudaStream_t st) {
+#define HK_K(k, shape_c, run_c, minb)                                                                    \
+    if (K == k && shape == shape_c) {                                                                    \
+        if (fs) return launch_persistent(conv1d_unpacked_tc_kernel<k, true, run_c, minb>, p, st);        \
+        return launch_persistent(conv1d_unpacked_tc_kernel<k, false, run_c, minb>, p, st);               \
     }
-    HK_K(3, 24) HK_K(5, 24) HK_K(7, 24) HK_K(3, 32) HK_K(5, 32) HK_K(7, 32)
+    HK_K(3, 24, 24, 4) HK_K(5, 24, 24, 4) HK_K(7, 24, 24, 4) HK_K(3, 25, 24, 5) HK_K(5, 25, 24, 5) HK_K(7, 25, 24, 5)
+    HK_K(3, 32, 32, 3) HK_K(5, 32, 32, 3) HK_K(7, 32, 32, 3)
 #undef HK_K
     return HIKONV_ERR_UNSUPPORTED;
 }
 
 bool conv1d_dp4a_tc_available(int K) { return K >= 1 && K <= 8; }
 
-int launch_conv1d_dp4a_tc(const Conv1dTcParams &p, int K, bool fs, bool gs, int run, cudaStream_t st) {
-#define HK_KW(kw, run_c)                                                                                            \
-    if ((K + 3) / 4 == kw && run == run_c) {                                                                        \
-        if (fs && gs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, true, true, run_c>, p, st);                \
-        if (fs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, true, false, run_c>, p, st);                     \
-        if (gs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, false, true, run_c>, p, st);                     \
-        return launch_persistent(conv1d_dp4a_tc_kernel<kw, false, false, run_c>, p, st);                            \
+int launch_conv1d_dp4a_tc(const Conv1dTcParams &p, int K, bool fs, bool gs, int shape, cudaStream_t st) {
+#define HK_KW(kw, shape_c, run_c, minb)                                                                             \
+    if ((K + 3) / 4 == kw && shape == shape_c) {                                                                    \
+        if (fs && gs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, true, true, run_c, minb>, p, st);          \
+        if (fs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, true, false, run_c, minb>, p, st);               \
+        if (gs) return launch_persistent(conv1d_dp4a_tc_kernel<kw, false, true, run_c, minb>, p, st);               \
+        return launch_persistent(conv1d_dp4a_tc_kernel<kw, false, false, run_c, minb>, p, st);                      \
     }
-    HK_KW(1, 24) HK_KW(2, 24) HK_KW(1, 32) HK_KW(2, 32)
+    HK_KW(1, 24, 24, 4) HK_KW(2, 24, 24, 4) HK_KW(1, 25, 24, 5) HK_KW(2, 25, 24, 5) HK_KW(1, 32, 32, 3) HK_KW(2, 32, 32, 3)
 #undef HK_KW
     return HIKONV_ERR_UNSUPPORTED;
 }

@@ -14,6 +14,7 @@ struct Conv1dTcParams {
     long long len;
     long long n_out;
     long long n_tiles;       // warp tiles of 32 * L outputs covering n_out
+    unsigned fast_after_first;   // comparators: tiles 1 .. this many lie inside aligned buffers (0: f or y unaligned)
     int K, S, Kc;
     int hi_shift;            // S * N
     int g_signed;
@@ -34,10 +35,10 @@ int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool signed_p
 bool conv1d_packed_dense_available(int P, int N, int J, int S, bool signed_prod, bool f_signed);
 int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, bool signed_prod, bool f_signed, cudaStream_t st);
 bool conv1d_unpacked_tc_available(int K);
-int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool f_signed, int run /* outputs per lane: 24 or 32 */, cudaStream_t st);
+int launch_conv1d_unpacked_tc(const Conv1dTcParams &p, int K, bool f_signed, int shape /* 24: runs of 24 outputs per lane, four CTAs per SM; 25: the same with five CTAs; 32: runs of 32, three CTAs */, cudaStream_t st);
 // Byte dot-product comparator (four products per dp4a): kernels of up to eight taps.
 bool conv1d_dp4a_tc_available(int K);
-int launch_conv1d_dp4a_tc(const Conv1dTcParams &p, int K, bool f_signed, bool g_signed, int run /* outputs per lane: 24 or 32 */,
+int launch_conv1d_dp4a_tc(const Conv1dTcParams &p, int K, bool f_signed, bool g_signed, int shape /* 24: runs of 24 outputs per lane, four CTAs per SM; 25: the same with five CTAs; 32: runs of 32, three CTAs */,
                           cudaStream_t st);
 
 }  // namespace hikonv

@@ -629,7 +629,7 @@ static int launch_pitch(const Conv2dSetup &s, bool sp, cudaStream_t st) {
     if (!sp) HK_LAUNCH(false);
     else HK_LAUNCH(true);
 #undef HK_LAUNCH
-    return launch_status();
+    return HIKONV_OK;
 }
 
 // KT > 0: the kernel with unrolled (kh, j) loops and a compile-time row pitch; KT == 0: everything at run time.
@@ -923,7 +923,6 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
         }
 #undef HK_PACK
     }
-    rc = launch_status();
     if (rc != HIKONV_OK) return rc;
     return launch_conv2d(s, st);
 }
@@ -936,11 +935,23 @@ constexpr int kMaxDevices = 64;
 std::mutex g_scratch_mutex;
 void *g_scratch_ptr[kMaxDevices] = {nullptr};
 
+// Is `ptr` device memory of GPU `dev`?  (A query of the pointer's attributes; nothing is allocated.)
+bool on_device(const void *ptr, int dev) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, ptr) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged) && attr.device == dev;
+}
+
 // Device address of g_static_scratch on the current device.  In host code the array's name is only
-// a handle, so the address is asked for once per device and cached.
-int static_scratch_address(void **out) {
+// a handle, so the address is asked for once per device and cached.  The buffer of the CURRENT device is
+// used, so the operands must live there: a buffer of one GPU must not reach kernels that run on another.
+int static_scratch_address(void **out, const void *d_x, const void *d_out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HIKONV_ERR_CUDA;
+    if (!d_x || !d_out || !on_device(d_x, dev) || !on_device(d_out, dev)) return HIKONV_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(g_scratch_mutex);
     if (!g_scratch_ptr[dev]) {
         void *ptr = nullptr;
@@ -960,7 +971,7 @@ extern "C" int hikonv_conv2d_static_scratch(const int8_t *d_x, int B, int Ci, in
     if (need == 0) return HIKONV_ERR_INVALID_ARG;
     if (need > (size_t)HIKONV_STATIC_SCRATCH_BYTES) return HIKONV_ERR_TOO_LARGE;
     void *scratch = nullptr;
-    const int rc = static_scratch_address(&scratch);
+    const int rc = static_scratch_address(&scratch, d_x, d_out);
     if (rc != HIKONV_OK) return rc;
     // the packing kernels write every word the layer kernel reads, so stale contents are harmless
     return hikonv_conv2d(d_x, B, Ci, H, W, d_w, Co, K, stride, pad, p, q, x_signed, w_signed, d_out, requant, shift, lo, hi,
@@ -1022,8 +1033,8 @@ extern "C" int hikonv_maxpool2x2_i8(const int8_t *d_in, int B, int C, int H, int
     }
     long long blocks = (total + 255) / 256;
     if (blocks > cap) blocks = cap;
-    maxpool2x2_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(d_in, B * C, H, W, is_signed ? 1 : 0, d_out);
-    return launch_status();
+    return launch_plain(maxpool2x2_kernel, dim3((unsigned)blocks), dim3(256), 0, (cudaStream_t)stream, d_in, B * C, H, W,
+                        is_signed ? 1 : 0, d_out);
 }
 
 extern "C" double hikonv_conv2d_multiplies(int B, int Ci, int H, int W, int Co, int K, int pad, int p, int q, int x_signed,

@@ -16,8 +16,20 @@ namespace hikonv {
         if (_e != cudaSuccess) return HIKONV_ERR_CUDA;        \
     } while (0)
 
-// After a kernel launch: report a launch failure without clearing an earlier sticky error.
-inline int launch_status() { return cudaPeekAtLastError() == cudaSuccess ? HIKONV_OK : HIKONV_ERR_CUDA; }
+// Plain launch that is judged by its own result: the status is what cudaLaunchKernelEx returns for THIS launch,
+// so an error that an earlier, unrelated call left unread in the thread's error state is neither reported here
+// nor cleared.
+template <typename... Params, typename... Args>
+inline int launch_plain(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = nullptr;
+    cfg.numAttrs = 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...) == cudaSuccess ? HIKONV_OK : HIKONV_ERR_CUDA;
+}
 
 // Programmatic dependent launch.  A kernel launched with launch_dependent() may be scheduled while the
 // kernel before it on the stream is still running; it must call grid_dependency_wait() before its first
@@ -43,13 +55,32 @@ inline int launch_dependent(void (*kernel)(Params...), dim3 grid, dim3 block, si
     return cudaLaunchKernelEx(&cfg, kernel, args...) == cudaSuccess ? HIKONV_OK : HIKONV_ERR_CUDA;
 }
 
-// One 32x32->64 multiply-accumulate, acc += a * b (the packed multiply of Eq. 9).
+// The 32x32->64 product of two packed words (Eq. 9).  The multiply is given as inline PTX (mul.wide) and the
+// 64-bit add is left to the compiler, which fuses the pair into one wide multiply-add.  Two other spellings were
+// tried and dropped after counting instructions per opcode in the profiler: mad.wide as inline PTX came out as a
+// multiply plus separate 64-bit additions, and the plain C++ expression (int64)a * (int64)b + c becomes a full
+// 64-bit multiply (three multiplies and adds) whenever the optimiser has hoisted or combined one of the sign
+// extensions.
+template <bool SIGNED>
+__device__ __forceinline__ uint64_t mul_wide(uint32_t a, uint32_t b) {
+    uint64_t r;
+    if (SIGNED)
+        asm("mul.wide.s32 %0, %1, %2;" : "=l"(r) : "r"(a), "r"(b));
+    else
+        asm("mul.wide.u32 %0, %1, %2;" : "=l"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// acc += a * b.
 template <bool SIGNED>
 __device__ __forceinline__ void mad_wide(uint64_t &acc, uint32_t a, uint32_t b) {
-    if (SIGNED)
-        asm("mad.wide.s32 %0, %1, %2, %0;" : "+l"(acc) : "r"(a), "r"(b));
-    else
-        asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(acc) : "r"(a), "r"(b));
+    acc += mul_wide<SIGNED>(a, b);
+}
+
+// a * b + c with the addend as an operand of its own.
+template <bool SIGNED>
+__device__ __forceinline__ uint64_t mul_wide_add(uint32_t a, uint32_t b, uint64_t c) {
+    return c + mul_wide<SIGNED>(a, b);
 }
 
 // Low 32 bits of (v >> sh) for 0 <= sh < 64.

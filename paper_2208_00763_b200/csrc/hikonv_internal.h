@@ -48,6 +48,10 @@ int make_layout(int p, int q, int f_signed, int g_signed, int K, int dims, int t
 // Layout for 64-bit operands and a 128-bit product (1-D rule); fields as in hikonv_layout_t with
 // 64 / 128 in place of 32 / 64.
 int make_layout_emu64(int p, int q, int f_signed, int g_signed, int K, const hikonv_tuning_t *tune, hikonv_layout_t *out);
+// 1-D layout with register-aligned slots, the narrowest that holds every sum of K products: returns the kernel
+// mode (1: S = 8, N = 4; 2: S = 16, N = 2; 3: S = 17 .. 21, N = 2) and fills `out`, or returns 0 when none applies
+// (K > 8, an operand that does not fit its register, sums beyond 21 bits).
+int make_layout_byte_slots(int p, int q, int f_signed, int g_signed, int K, hikonv_layout_t *out);
 SplitConsts128 make_split_consts128(const hikonv_layout_t &L, int p, int q, int f_signed, int g_signed, int K);
 SplitConsts make_split_consts(const hikonv_layout_t &L, int p, int q, int f_signed, int g_signed, int K, int M);
 

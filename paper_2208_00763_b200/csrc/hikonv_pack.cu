@@ -39,16 +39,11 @@ extern "C" int hikonv_pack(const int8_t *d_in, size_t n, int bits, int is_signed
     const size_t blocks = (n_words + threads - 1) / threads;
     if (blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
+    const dim3 grid((unsigned)blocks), block(threads);
     if (word_bits == 32) {
-        if (is_signed)
-            pack_kernel<true, uint32_t><<<(unsigned)blocks, threads, 0, st>>>(d_in, n, S, N, (uint32_t *)d_words, n_words);
-        else
-            pack_kernel<false, uint32_t><<<(unsigned)blocks, threads, 0, st>>>(d_in, n, S, N, (uint32_t *)d_words, n_words);
-    } else {
-        if (is_signed)
-            pack_kernel<true, uint64_t><<<(unsigned)blocks, threads, 0, st>>>(d_in, n, S, N, (uint64_t *)d_words, n_words);
-        else
-            pack_kernel<false, uint64_t><<<(unsigned)blocks, threads, 0, st>>>(d_in, n, S, N, (uint64_t *)d_words, n_words);
+        if (is_signed) return launch_plain(pack_kernel<true, uint32_t>, grid, block, 0, st, d_in, n, S, N, (uint32_t *)d_words, n_words);
+        return launch_plain(pack_kernel<false, uint32_t>, grid, block, 0, st, d_in, n, S, N, (uint32_t *)d_words, n_words);
     }
-    return launch_status();
+    if (is_signed) return launch_plain(pack_kernel<true, uint64_t>, grid, block, 0, st, d_in, n, S, N, (uint64_t *)d_words, n_words);
+    return launch_plain(pack_kernel<false, uint64_t>, grid, block, 0, st, d_in, n, S, N, (uint64_t *)d_words, n_words);
 }

@@ -335,6 +335,49 @@ int make_layout_emu64(int p, int q, int fs, int gs, int K, const hikonv_tuning_t
     return HIKONV_OK;
 }
 
+// Register-aligned slots for the 1-D kernels.  Mode 1: S = 8, N = 4, four taps per kernel word; mode 2: S = 16,
+// N = 2, two taps; mode 3: the narrowest S in 17 .. 21 with N = 2, two taps.  The conditions are those of the
+// exact-range rule above, specialised: both operands fit a 32-bit register (31 bits plus sign for a signed
+// multiply; signed codes enter the multiplier lifted to non-negative values -- by 2^(p-1) in mode 1, by 128 in
+// modes 2 and 3 -- so only their lifted width counts), the N + Kc - 1 slots fit 64 bits, and every output, a sum
+// of at most K products, fits its S-bit slot: as an unsigned value, or as a two's-complement one when either
+// operand is signed (modes 1 and 2 read signed slots with a sign-extending permute, mode 3 subtracts 2^(S-1)).
+int make_layout_byte_slots(int p, int q, int fs, int gs, int K, hikonv_layout_t *out) {
+    if (validate_codes(p, q) != HIKONV_OK || K < 1 || K > 8) return 0;
+    fs = fs ? 1 : 0;
+    gs = gs ? 1 : 0;
+    const bool sp = fs || gs;
+    const Range fr = code_range(p, fs), gr = code_range(q, gs);
+    const long long prods[4] = {fr.lo * gr.lo, fr.lo * gr.hi, fr.hi * gr.lo, fr.hi * gr.hi};
+    const long long pmin = *std::min_element(prods, prods + 4), pmax = *std::max_element(prods, prods + 4);
+    const long long lo = (long long)K * pmin, hi = (long long)K * pmax;
+    for (int S = 8; S <= 21; S = (S == 8 ? 16 : S + 1)) {
+        const int mode = S == 8 ? 1 : S == 16 ? 2 : 3;
+        const int N = mode == 1 ? 4 : 2;
+        const int Kc = std::min(K, N), J = ceil_div(K, Kc);
+        const Range lifted = {0, (mode == 1 || !fs) ? (1LL << p) - 1 : 255};
+        if (!operand_fits(lifted, N, S, sp)) continue;
+        if (!operand_fits(gr, Kc, S, sp)) continue;
+        if (S * (N + Kc - 1) > 63) continue;
+        if (sp ? (lo < -(1LL << (S - 1)) || hi > (1LL << (S - 1)) - 1) : (hi > (1LL << S) - 1)) continue;
+        if (out) {
+            std::memset(out, 0, sizeof(*out));
+            out->N = N;
+            out->S = S;
+            out->Kc = Kc;
+            out->J = J;
+            out->segments = N + Kc - 1;
+            out->top_bits = std::min(S, 64 - S * (N + Kc - 2));
+            out->M = 1;
+            out->signed_prod = sp ? 1 : 0;
+            out->S_paper = slice_bits(p, q, guard_bits(HIKONV_GB_1D, 1, K, 1));
+            out->carry_bits = 0;
+        }
+        return mode;
+    }
+    return 0;
+}
+
 SplitConsts128 make_split_consts128(const hikonv_layout_t &L, int p, int q, int fs, int gs, int K) {
     SplitConsts128 c;
     std::memset(&c, 0, sizeof(c));

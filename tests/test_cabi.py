@@ -208,17 +208,29 @@ def test_device_entry_points_validate_before_touching_cuda():
 
 
 def test_multiply_counts():
-    # packed 4-bit K = 3: one multiply per block of N = 3 outputs; comparator: K per output
+    # packed 4-bit K = 3 on the planner's layout: one multiply per block of N = 3 outputs; comparator: K per output
     n = 3000
-    assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 3)
+    planner = {"tile": -1}
+    assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32, planner) == -(-(n + 2) // 3)
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_UNPACKED_IMAD) == (n + 2) * 3
     assert hk.conv1d_multiplies(n, 7, 4, 4, False, False, hk.ALGO_DP4A) == (n + 6) * 2
     assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED64EMU) == -(-(n + 2) // hk.layout_emu64(4, 4, False, False, 3)["N"])
-    # byte input: the HBM-bound 1-D kernel runs blocks of 8 where the planner says 11 (1-bit, K = 3) and of 4
-    # where it says 5 (2-bit, K = 5), unless the layout is forced; hikonv_layout keeps the planner's answer
+    # byte input without a forced layout: byte-aligned slots (the HBM-bound call takes the fewest instructions per
+    # output, not the most outputs per multiply): 16-bit slots, N = 2, the three taps in two kernel words at
+    # 4 bits; 8-bit slots, N = 4 at 1 and 2 bits; 18-bit slots, N = 2, two taps per kernel word for signed 8-bit codes
+    assert hk.conv1d_multiplies(n, 3, 4, 4, False, False, hk.ALGO_PACKED32) == 2 * -(-(n + 2) // 2)
+    assert hk.conv1d_multiplies(n, 3, 1, 1, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 4)
+    assert hk.conv1d_multiplies(n, 5, 2, 2, False, False, hk.ALGO_PACKED32) == 2 * -(-(n + 4) // 4)
+    assert hk.conv1d_multiplies(n, 7, 8, 8, True, True, hk.ALGO_PACKED32) == 4 * -(-(n + 6) // 2)
+    L8 = hk.conv1d_layout(8, 8, True, True, 7)
+    assert (L8["N"], L8["S"], L8["Kc"], L8["J"]) == (2, 18, 2, 4)
+    assert hk.conv1d_layout(4, 4, False, False, 3) == dict(hk.conv1d_layout(4, 4, False, False, 3), N=2, S=16, Kc=2, J=2)
+    # with tile = -1 the planner's layout runs, in blocks of 8 where the planner says 11 (1-bit, K = 3) and of 4
+    # where it says 5 (2-bit, K = 5), unless N is forced; hikonv_layout keeps the planner's answer
     assert hk.layout(1, 1, False, False, 3, 1)["N"] == 11 and hk.layout(2, 2, False, False, 5, 1)["N"] == 5
-    assert hk.conv1d_multiplies(n, 3, 1, 1, False, False, hk.ALGO_PACKED32) == -(-(n + 2) // 8)
-    assert hk.conv1d_multiplies(n, 5, 2, 2, False, False, hk.ALGO_PACKED32) == -(-(n + 4) // 4)
+    assert hk.conv1d_multiplies(n, 3, 1, 1, False, False, hk.ALGO_PACKED32, planner) == -(-(n + 2) // 8)
+    assert hk.conv1d_multiplies(n, 5, 2, 2, False, False, hk.ALGO_PACKED32, planner) == -(-(n + 4) // 4)
+    assert hk.conv1d_layout(1, 1, False, False, 3, planner)["N"] == 8
     assert hk.conv1d_multiplies(n, 3, 1, 1, False, False, hk.ALGO_PACKED32, {"N": 11}) == -(-(n + 2) // 11)
     # a smaller block that would need more kernel chunks is not taken: 1-bit codes x signed 2-bit taps, K = 9
     # fit two chunks of N = 5 taps but would need three of N = 4
@@ -229,3 +241,77 @@ def test_multiply_counts():
     unpacked = hk.conv2d_multiplies(2, 8, 10, 12, 16, 3, 1, 4, 4, True, True, hk.ALGO_UNPACKED_IMAD)
     macs = 2 * 16 * 10 * 12 * 8 * 9
     assert 0 < packed < macs / 2 and unpacked >= macs
+
+
+class _FakeDeviceTensor:
+    """Stands in for a CUDA tensor where there is no GPU: only what the binding's checks look at."""
+
+    def __init__(self, numel, dtype, device="cuda:0", contiguous=True, is_cuda=True):
+        self._numel, self.dtype, self.device, self._contiguous, self.is_cuda = numel, dtype, device, contiguous, is_cuda
+
+    def numel(self):
+        return self._numel
+
+    def is_contiguous(self):
+        return self._contiguous
+
+    def data_ptr(self):
+        return 0x1000
+
+
+def test_output_tensors_are_validated_before_any_launch():
+    # the kernels see only an address: a short, mistyped, strided or misplaced `out` must be refused on the host
+    import torch
+    like = _FakeDeviceTensor(10, torch.int8)
+    good = _FakeDeviceTensor(12, torch.int32)
+    assert hk._dev_out(good, "out", 12, (torch.int32,), like) == 0x1000
+    for bad in (_FakeDeviceTensor(11, torch.int32),                         # too short
+                _FakeDeviceTensor(12, torch.int8),                          # bytes where int32 is written
+                _FakeDeviceTensor(12, torch.int32, contiguous=False),       # strided view
+                _FakeDeviceTensor(12, torch.int32, device="cuda:1"),        # another GPU
+                _FakeDeviceTensor(12, torch.int32, is_cuda=False),          # host memory
+                torch.empty(12, dtype=torch.int32)):                        # a real CPU tensor
+        with pytest.raises(ValueError):
+            hk._dev_out(bad, "out", 12, (torch.int32,), like)
+    # through a public wrapper: a CPU tensor as `out` never reaches the library
+    f = torch.zeros(8, dtype=torch.int8)
+    with pytest.raises(ValueError):
+        hk.conv1d(f, f[:3], 4, 4, False, False, out=torch.empty(10, dtype=torch.int32))
+
+
+def test_register_aligned_layout_conditions():
+    # hikonv_conv1d_layout takes slots of 8, 16 or 17..21 bits exactly when, recomputed here from the code ranges:
+    # the (lifted) packed codes fit the multiplier's register, the kernel word fits it, the slots fit 64 bits and
+    # K products fit the slot
+    for p in range(1, 9):
+        for q in range(1, 9):
+            for fs in (False, True):
+                for gs in (False, True):
+                    flo, fhi = (-(1 << (p - 1)), (1 << (p - 1)) - 1) if fs else (0, (1 << p) - 1)
+                    glo, ghi = (-(1 << (q - 1)), (1 << (q - 1)) - 1) if gs else (0, (1 << q) - 1)
+                    prods = [a * b for a in (flo, fhi) for b in (glo, ghi)]
+                    signed_mul = fs or gs
+                    reg_hi = (1 << 31) - 1 if signed_mul else (1 << 32) - 1
+                    for K in range(1, 10):
+                        want = None
+                        for S in (8, 16, 17, 18, 19, 20, 21):
+                            N = 4 if S == 8 else 2
+                            Kc = min(K, N)
+                            # signed codes enter lifted: by 2^(p-1) with one-byte slots, by 128 otherwise
+                            top = (1 << p) - 1 if (S == 8 or not fs) else 255
+                            a_ok = sum(top << (S * n) for n in range(N)) <= reg_hi
+                            b_lo = sum(glo << (S * k) for k in range(Kc))
+                            b_hi = sum(ghi << (S * k) for k in range(Kc))
+                            b_ok = b_hi <= reg_hi and (b_lo >= -(1 << 31) if signed_mul else b_lo >= 0)
+                            lo, hi = K * min(prods), K * max(prods)
+                            y_ok = (-(1 << (S - 1)) <= lo and hi <= (1 << (S - 1)) - 1) if signed_mul else hi <= (1 << S) - 1
+                            if K <= 8 and a_ok and b_ok and y_ok and S * (N + Kc - 1) <= 63:
+                                want = (N, S, Kc, -(-K // Kc))
+                                break
+                        L = hk.conv1d_layout(p, q, fs, gs, K)
+                        got = (L["N"], L["S"], L["Kc"], L["J"])
+                        if want is not None:
+                            assert got == want, (p, q, fs, gs, K, got, want)
+                        else:
+                            plan = hk.conv1d_layout(p, q, fs, gs, K, {"tile": -1})
+                            assert got == (plan["N"], plan["S"], plan["Kc"], plan["J"]), (p, q, fs, gs, K)

@@ -10,10 +10,17 @@ from gpu_util import assert_exact, dev
 
 pytestmark = pytest.mark.gpu
 
-ALGOS = [hk.ALGO_PACKED32, hk.ALGO_UNPACKED_IMAD]
+# "planner": the packed kernels on the planner's layout (most outputs per multiply); without it the packed call
+# takes byte-aligned slots wherever the sums fit them (tests/test_gpu_conv1d_byte_slots.py covers those further)
+PLANNER = "planner-layout"
+ALGOS = [hk.ALGO_PACKED32, PLANNER, hk.ALGO_UNPACKED_IMAD]
 
 
 def _run(f, g, p, q, fs, gs, algo, tune=None):
+    if algo == PLANNER:
+        algo = hk.ALGO_PACKED32
+        if not tune:
+            tune = {"tile": -1}
     return hk.conv1d(dev(f), dev(g), p, q, fs, gs, algo=algo, tune=tune)
 
 
@@ -113,16 +120,18 @@ def test_planner_block_sizes_that_the_automatic_choice_replaces(signed):
     assert_exact(_run(f, g, 1, 2, False, True, hk.ALGO_PACKED32), direct.conv1d_full(f, g), "1-bit x s2, K=9")
 
 
+@pytest.mark.parametrize("shape", [-32, -24, -25])
 @pytest.mark.parametrize("algo", [hk.ALGO_UNPACKED_IMAD, hk.ALGO_DP4A])
-def test_comparators_with_runs_of_32_outputs(algo):
-    # tile = -32 selects the longer per-lane runs of the two comparators (24 is the default)
+def test_comparators_in_every_launch_shape(algo, shape):
+    # tile = -32: runs of 32 outputs per lane; -24 / -25: runs of 24 with the register budget of four / five
+    # resident CTAs per SM (the default picks between the last two by kernel length)
     for signed in (False, True):
         for bits in (1, 4, 8):
             for K in (3, 5, 7):
                 for n in (100003, 1023):
                     f, g = inputs.conv1d_case(n, K, bits, bits, signed, signed, seed=500 + bits * 10 + K)
-                    assert_exact(_run(f, g, bits, bits, signed, signed, algo, {"tile": -32}), direct.conv1d_full(f, g),
-                                 "runs of 32: p=%d K=%d n=%d signed=%d" % (bits, K, n, signed))
+                    assert_exact(_run(f, g, bits, bits, signed, signed, algo, {"tile": shape}), direct.conv1d_full(f, g),
+                                 "shape %d: p=%d K=%d n=%d signed=%d" % (shape, bits, K, n, signed))
 
 
 @pytest.mark.parametrize("algo", ALGOS)
@@ -136,7 +145,8 @@ def test_unaligned_pointers(algo):
         big_y = torch.full((20016,), -7, dtype=torch.int32, device="cuda")
         big_f[shift:shift + 20000] = dev(f)
         y = big_y[shift:shift + 20002]
-        hk.conv1d(big_f[shift:shift + 20000], dev(g), 4, 4, True, True, algo=algo, out=y)
+        hk.conv1d(big_f[shift:shift + 20000], dev(g), 4, 4, True, True, algo=hk.ALGO_PACKED32 if algo == PLANNER else algo,
+                  tune={"tile": -1} if algo == PLANNER else None, out=y)
         assert_exact(y, ref, "offset %d" % shift)
         torch.cuda.synchronize()
         assert int(big_y[shift - 1]) == -7 and int(big_y[shift + 20002]) == -7     # nothing written outside

@@ -40,6 +40,17 @@ def test_extreme_codes_and_unaligned_buffers(bits):
             assert_exact(_run(f, g, bits, signed, offset), ref, "offset %d" % offset)
 
 
+@pytest.mark.parametrize("bits", [1, 2, 4])
+def test_full_size_sweep_cases(bits):
+    # the 18 dense cases the benchmark times (1, 2 and 4 bits; K = 3, 5, 7; both signs) at 2^24 codes against the
+    # oracle: at this length every warp of the persistent grid walks several tiles
+    for case in inputs.c2_cases():
+        if case["p"] != bits:
+            continue
+        f, g = inputs.conv1d_case(case["length"], case["K"], case["p"], case["q"], case["f_signed"], case["g_signed"], case["seed"])
+        assert_exact(_run(f, g, bits, case["f_signed"]), direct.conv1d_full(f, g), "dense " + str(case))
+
+
 def test_same_results_as_byte_storage_at_full_size():
     # the benchmark length, one case: dense and one-code-per-byte inputs give identical outputs
     f, g = inputs.conv1d_case(1 << 24, 3, 4, 4, True, True, seed=1431)

@@ -1,5 +1,5 @@
 """GPU parity of HIKONV_ALGO_PACKED64EMU (64-bit packed words, 64x64 -> 128 product built from 32-bit
-multiplies; the wider multiplier of Section IV-C) against the int64 oracle, bit for bit."""
+multiplies; the wider multiplier of Section V-A) against the int64 oracle, bit for bit."""
 import numpy as np
 import pytest
 import torch

@@ -121,28 +121,25 @@ def test_requantize(algo):
 
 
 @pytest.mark.parametrize("algo", ALGOS)
-def test_c3_layer_sampled_images(algo):
-    # full-size launch (batch 32); the oracle checks three whole images of it
+def test_c3_layer_every_image(algo):
+    # full-size launch (batch 32); the oracle checks all 32 images of it, codes and (packed algorithm) exact sums
     s = inputs.C3_SHAPE
     x, w = inputs.layer_case(s)
+    acc = direct.conv2d_nchw(x, w, s["pad"])
     got = _layer(x, w, s["pad"], s["p"], s["q"], s["x_signed"], s["w_signed"], algo, requant=(s["shift"], s["lo"], s["hi"]))
-    torch.cuda.synchronize()
-    g = got.cpu().numpy().astype(np.int64)
-    for b in (0, 13, 31):
-        ref = direct.requant(direct.conv2d_nchw(x[b:b + 1], w, s["pad"]), s["shift"], s["lo"], s["hi"])
-        assert np.array_equal(g[b:b + 1], ref), "image %d" % b
+    assert_exact(got, direct.requant(acc, s["shift"], s["lo"], s["hi"]), "C3 codes")
+    if algo == hk.ALGO_PACKED32:
+        assert_exact(_layer(x, w, s["pad"], s["p"], s["q"], s["x_signed"], s["w_signed"], algo), acc, "C3 sums")
 
 
 @pytest.mark.parametrize("algo", ALGOS)
-def test_c4_layer_sampled_images(algo):
+def test_c4_layer_every_image(algo):
+    # full-size launch (batch 64), all 64 images against the oracle
     s = inputs.C4_SHAPE
     x, w = inputs.layer_case(s)
     assert abs(float((x == 0).mean()) - (0.3 + 0.7 / 16)) < 0.01
     got = _layer(x, w, s["pad"], s["p"], s["q"], s["x_signed"], s["w_signed"], algo)
-    torch.cuda.synchronize()
-    g = got.cpu().numpy().astype(np.int64)
-    for b in (0, 31, 63):
-        assert np.array_equal(g[b:b + 1], direct.conv2d_nchw(x[b:b + 1], w, s["pad"])), "image %d" % b
+    assert_exact(got, direct.conv2d_nchw(x, w, s["pad"]), "C4 sums")
 
 
 def test_host_buffer_entry_point():
@@ -167,17 +164,21 @@ def test_compact_cnn_small_batch(algo):
     assert_exact(head, ref_head, "head")
 
 
-def test_compact_cnn_full_size_sampled():
-    # the benchmark configuration (batch 64, 3x160x320); the oracle checks two images end to end
+def test_compact_cnn_full_size_every_image():
+    # the benchmark configuration (batch 64, 3x160x320): head output and every layer's activations of all 64
+    # images against the oracle (the oracle runs the batch in four parts to bound its int64 buffers)
     x, layers, head_w = inputs.c5_network()
     net = network.CompactCnn(layers, head_w, device="cuda")
-    head, _ = net.forward(dev(x))
+    head, acts = net.forward(dev(x), keep_activations=True)
     torch.cuda.synchronize()
     g = head.cpu().numpy().astype(np.int64)
     assert g.shape == (64, 36, 10, 20)
-    for b in (0, 63):
-        ref_head, _ = direct.cnn_forward(x[b:b + 1], layers, head_w)
-        assert np.array_equal(g[b:b + 1], ref_head), "image %d" % b
+    g_acts = [a.cpu().numpy() for a in acts]
+    for b0 in range(0, 64, 16):
+        ref_head, ref_acts = direct.cnn_forward(x[b0:b0 + 16], layers, head_w)
+        assert np.array_equal(g[b0:b0 + 16], ref_head), "head, images %d..%d" % (b0, b0 + 15)
+        for i, (a, r) in enumerate(zip(g_acts, ref_acts)):
+            assert np.array_equal(a[b0:b0 + 16].astype(np.int64), r), "layer %d, images %d..%d" % (i + 1, b0, b0 + 15)
 
 
 def test_layer_chain_captured_in_a_cuda_graph():

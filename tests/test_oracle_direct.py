@@ -227,3 +227,69 @@ def test_count_out_of_range_against_enumeration():
             assert direct.count_out_of_range(vals, bits, signed) == want
     assert direct.count_out_of_range([0, 15, 16, -1], 4, False) == 2
     assert direct.count_out_of_range([-8, 7, 8, -9], 4, True) == 2
+
+
+def test_pack_words_printed_multiplicands():
+    # Section V-A-2's worked example: f = (11, 9, 7) and g = (3, 2) with S = 10 are printed packed as 11543559
+    # and 3074, element 0 in the TOP slot; Eq. 5 puts element 0 in the lowest slot, so the mirrored sequences
+    # must reproduce the printed words, and the product of the two words must be the printed one
+    g = _golden("worked_example_f32.txt")
+    f = [int(t) for t in g["f"].split()]
+    k = [int(t) for t in g["g"].split()]
+    S = int(g["S"])
+    wf = direct.pack_words(f[::-1], S, len(f), 32)
+    wg = direct.pack_words(k[::-1], S, len(k), 32)
+    assert wf.tolist() == [int(g["multiplicand_f"])] and wg.tolist() == [int(g["multiplicand_g"])]
+    assert int(wf[0]) * int(wg[0]) == int(g["product"])
+    # a second block and a ragged tail: (11, 9, 7, 5) in blocks of three -> the printed word and 5 alone
+    assert direct.pack_words([7, 9, 11, 5], S, 3, 64).tolist() == [int(g["multiplicand_f"]), 5]
+    # signed codes: Eq. 28's slot-by-slot form, written out by hand for (-1, 2) at S = 4: slot 0 holds 15,
+    # slot 1 holds 2 - 1 (the borrow of the negative slot below): 0x1F
+    assert direct.pack_words([-1, 2], 4, 2, 32).tolist() == [0x1F]
+    # (-1, -1): slot 0 holds 15, slot 1 holds -1 - 1 = 14 (mod 16), the sign fills the rest of the register
+    assert direct.pack_words([-1, -1], 4, 2, 32).tolist() == [0xFFFFFFEF]
+
+
+def _torch_network(x, layers, head_w):
+    """The same chain through library routines: float64 conv2d (exact below 2^53), floor division by 2^shift,
+    clamp, max_pool2d."""
+    a = torch.tensor(np.asarray(x), dtype=torch.float64)
+    acts = []
+    for L in layers:
+        a = torch.nn.functional.conv2d(a, torch.tensor(np.asarray(L["w"]), dtype=torch.float64), padding=L["pad"])
+        a = torch.clamp(torch.floor(a / float(1 << L["shift"])), L["lo"], L["hi"])
+        if L["pool"]:
+            a = torch.nn.functional.max_pool2d(a, 2, 2)
+        acts.append(a.numpy().astype(np.int64))
+    head = torch.nn.functional.conv2d(a, torch.tensor(np.asarray(head_w), dtype=torch.float64))
+    return head.numpy().astype(np.int64), acts
+
+
+def test_cnn_forward_vs_library_chain():
+    # a pooled layer, an unpooled one, a signed clamp range and the pad-0 1x1 head; odd sizes so that the pool
+    # drops a row and a column
+    rng = np.random.default_rng(77)
+    x = rng.integers(0, 256, (2, 3, 11, 14))
+    layers = [
+        {"w": rng.integers(-8, 8, (5, 3, 3, 3)), "pad": 1, "shift": 7, "lo": 0, "hi": 15, "pool": True},
+        {"w": rng.integers(-8, 8, (6, 5, 3, 3)), "pad": 1, "shift": 3, "lo": 0, "hi": 15, "pool": False},
+        {"w": rng.integers(-8, 8, (4, 6, 3, 3)), "pad": 0, "shift": 4, "lo": -8, "hi": 7, "pool": True},
+    ]
+    head_w = rng.integers(-8, 8, (7, 4, 1, 1))
+    head, acts = direct.cnn_forward(x, layers, head_w)
+    ref_head, ref_acts = _torch_network(x, layers, head_w)
+    assert [a.shape for a in acts] == [(2, 5, 5, 7), (2, 6, 5, 7), (2, 4, 1, 2)]
+    for a, r in zip(acts, ref_acts):
+        assert np.array_equal(a, r)
+    assert head.shape == (2, 7, 1, 2) and np.array_equal(head, ref_head)
+    # the activations are not degenerate: the clamps bite on both sides somewhere and the values spread
+    assert acts[0].min() == 0 and acts[0].max() == 15 and len(np.unique(acts[1])) > 4
+
+
+def test_cnn_forward_one_pixel_network_by_hand():
+    # 1x1 input, one channel, 1x1 kernels: layer 1: 200 * 3 = 600 >> 4 = 37 -> clamp [0, 15] = 15;
+    # layer 2: 15 * (-2) = -30 >> 2 = floor(-7.5) = -8 -> clamp [-8, 7] = -8; head: -8 * 5 = -40
+    layers = [{"w": [[[[3]]]], "pad": 0, "shift": 4, "lo": 0, "hi": 15, "pool": False},
+              {"w": [[[[-2]]]], "pad": 0, "shift": 2, "lo": -8, "hi": 7, "pool": False}]
+    head, acts = direct.cnn_forward([[[[200]]]], layers, [[[[5]]]])
+    assert [int(a.ravel()[0]) for a in acts] == [15, -8] and int(head.ravel()[0]) == -40
