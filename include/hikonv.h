@@ -240,6 +240,32 @@ int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *
                   int requant, int shift, int lo, int hi, void *d_workspace, size_t workspace_bytes,
                   int algo, const hikonv_tuning_t *tune, void *stream);
 
+/*
+ * hikonv_conv2d_dense - hikonv_conv2d on tensors stored without their unused bits (Section V-B, "Single convolver
+ * architecture": weights are kept compressed in memory, and "the same compression can also be applied to the
+ * feature data during runtime"), with the layer's requantised output written in the same compressed form and,
+ * optionally, max-pooled on the way out.
+ *   Dense storage of a tensor of b-bit codes, b in {1, 2, 4}: the codes in their NCHW (OIHW) order, 8 / b per
+ *   byte, code e in bits [(e b) % 8, (e b) % 8 + b) of byte (e b) / 8, two's complement when signed;
+ *   ceil(count b / 8) bytes.
+ *   x_store_bits: 8 (one code per byte, as hikonv_conv2d reads) or p (dense, p in {1, 2, 4});
+ *   w_store_bits: 8 or q (dense, q in {1, 2, 4});
+ *   out_store_bits: 32 with requant == 0 (int32 sums, 4-byte aligned);
+ *                   with requant != 0: 8 (one code per byte) or 1 / 2 / 4 (dense; [lo, hi] must lie in the
+ *                   code range of that width, signed when lo < 0, and every output row must fill whole bytes:
+ *                   Wo' * out_store_bits a multiple of 8, else HIKONV_ERR_UNSUPPORTED);
+ *   pool: 0, or 1 = 2x2 maximum with stride 2 after requantisation (requant != 0, Ho and Wo even); the output is
+ *         then [B][Co][Ho / 2][Wo / 2] (Ho' = Ho / 2, Wo' = Wo / 2), else [B][Co][Ho][Wo].
+ * The packing stage unpacks dense codes as it reads them; the layer kernel stages a CTA's requantised codes in
+ * shared memory and writes whole bytes.  All other arguments, the workspace and the error behaviour are those of
+ * hikonv_conv2d; combinations that are not built return HIKONV_ERR_UNSUPPORTED and launch nothing.
+ */
+int hikonv_conv2d_dense(const void *d_x, int x_store_bits, int B, int Ci, int H, int W, const void *d_w,
+                        int w_store_bits, int Co, int K, int stride, int pad, int p, int q, int x_signed,
+                        int w_signed, void *d_out, int out_store_bits, int requant, int shift, int lo, int hi,
+                        int pool, void *d_workspace, size_t workspace_bytes, int algo,
+                        const hikonv_tuning_t *tune, void *stream);
+
 /* Workspace needed by hikonv_conv2d for this layer shape (an upper bound over all layouts and both algorithms). */
 size_t hikonv_conv2d_workspace_bytes(int B, int Ci, int H, int W, int Co, int K, int pad);
 

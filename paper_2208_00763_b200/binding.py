@@ -56,6 +56,8 @@ _SIGNATURES = {
     "hikonv_conv1d_host": (_i, [_vp, _sz, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _i, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _vp, _sz, _i,
                            ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv2d_dense": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz,
+                                 _i, ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d_workspace_bytes": (_sz, [_i] * 7),
     "hikonv_conv2d_static_scratch": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i,
                                           ctypes.POINTER(TuningT), _vp]),
@@ -256,6 +258,44 @@ def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_sig
                                int(x_signed), int(w_signed), out_ptr, 1 if requant else 0, shift, lo, hi,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), algo, _tune(tune),
                                _stream(stream)), "hikonv_conv2d")
+    return out
+
+
+def conv2d_dense(d_x: torch.Tensor, x_shape, x_store_bits: int, d_w: torch.Tensor, w_shape, w_store_bits: int, pad: int, p: int,
+                 q: int, x_signed: bool, w_signed: bool, requant: Optional[tuple] = None, out_store_bits: int = 8,
+                 pool: bool = False, algo: int = ALGO_PACKED32, tune=None, workspace: Optional[torch.Tensor] = None,
+                 out: Optional[torch.Tensor] = None, stride: int = 1, stream=None) -> torch.Tensor:
+    """``conv2d`` on densely stored tensors.  ``d_x`` / ``d_w`` are flat uint8 (dense) or int8 (one code per byte)
+    tensors holding the codes of ``x_shape`` = (B, Ci, H, W) / ``w_shape`` = (Co, Ci, K, K).  Returns int32
+    [B, Co, Ho, Wo] without ``requant``; with it a flat uint8 tensor of the (optionally pooled) output codes,
+    ``out_store_bits`` per code (8: shaped [B, Co, Ho', Wo'] int8)."""
+    B, Ci, H, W = x_shape
+    Co, Ci2, K, K2 = w_shape
+    if Ci != Ci2 or K != K2:
+        raise ValueError("weight shape does not match the input")
+    for t, n, bits, name in ((d_x, B * Ci * H * W, x_store_bits, "d_x"), (d_w, Co * Ci * K * K, w_store_bits, "d_w")):
+        if not t.is_cuda or not t.is_contiguous() or t.dtype not in _CODE_DTYPES or t.numel() * 8 < n * bits:
+            raise ValueError("%s must be a contiguous CUDA byte tensor holding all codes" % name)
+    Ho, Wo = H + 2 * pad - K + 1, W + 2 * pad - K + 1
+    Hq, Wq = (Ho // 2, Wo // 2) if pool else (Ho, Wo)
+    count = B * Co * max(Hq, 0) * max(Wq, 0)
+    if workspace is None:
+        workspace = torch.empty(conv2d_workspace_bytes(B, Ci, H, W, Co, K, pad), dtype=torch.uint8, device=d_x.device)
+    if not requant:
+        if out is None:
+            out = torch.empty((B, Co, max(Ho, 0), max(Wo, 0)), dtype=torch.int32, device=d_x.device)
+        out_ptr, store = _dev_out(out, "out", B * Co * max(Ho, 0) * max(Wo, 0), (torch.int32,), d_x), 32
+    else:
+        nbytes = (count * out_store_bits + 7) // 8
+        if out is None:
+            out = (torch.empty((B, Co, Hq, Wq), dtype=torch.int8, device=d_x.device) if out_store_bits == 8
+                   else torch.empty(nbytes, dtype=torch.uint8, device=d_x.device))
+        out_ptr, store = _dev_out(out, "out", nbytes, _CODE_DTYPES, d_x), out_store_bits
+    shift, lo, hi = requant if requant else (0, 0, 0)
+    _check(lib().hikonv_conv2d_dense(d_x.data_ptr(), x_store_bits, B, Ci, H, W, d_w.data_ptr(), w_store_bits, Co, K, stride, pad, p, q,
+                                     int(x_signed), int(w_signed), out_ptr, store, 1 if requant else 0, shift, lo, hi,
+                                     1 if pool else 0, workspace.data_ptr(), workspace.numel() * workspace.element_size(), algo,
+                                     _tune(tune), _stream(stream)), "hikonv_conv2d_dense")
     return out
 
 

@@ -67,6 +67,16 @@ struct Conv2dParams {
     uint64_t bias, mask_low, mask_high;
     uint32_t slot_mask, top_mask;
     int32_t slot_bias[kMaxN2DSeg];
+    // requantised output: the CTA's codes are staged as bytes in shared memory ([channel][row][column], WTP bytes
+    // per row) and leave in pieces of `vec` bytes along a row; with pool != 0 rows and columns are first reduced
+    // by a 2x2 maximum (output [B][Co][Ho/2][Wo/2]; TR and Ho are even then)
+    int stage_out;             // 1: staged (every requantised layer), 0: direct stores
+    int tile_off;              // word offset of the byte tile in shared memory
+    int WTP;                   // bytes per tile row (a multiple of 16)
+    int vec;                   // bytes per output piece: 16, 8, 4 or 1
+    int pool;                  // 2x2 max-pool fused into the copy-out
+    int out_signed;            // pooled codes compare as signed bytes
+    int out_bits;              // 8: one code per byte; 1 / 2 / 4: dense output, 8 / out_bits codes per byte (vec: 4 or 1 bytes)
 };
 
 template <bool UNPACKED>
@@ -99,6 +109,18 @@ __device__ __forceinline__ void mac(typename AccType<UNPACKED>::type &acc, uint3
     } else {
         acc += (uint64_t)a * (uint64_t)b;
     }
+}
+
+// VEC input bytes of two rows per thread (VEC = 8: two 8-byte loads, one 4-byte store; VEC = 16: two
+// 16-byte loads, one 8-byte store), per-byte maxima; needs W % VEC == 0 and VEC-byte aligned input,
+// VEC/2-byte aligned output.
+template <bool SIGNED>
+__device__ __forceinline__ uint32_t pool_pairs(uint32_t a0, uint32_t a1, uint32_t b0, uint32_t b1) {
+    uint32_t v0 = SIGNED ? __vmaxs4(a0, b0) : __vmaxu4(a0, b0);     // the two rows
+    uint32_t v1 = SIGNED ? __vmaxs4(a1, b1) : __vmaxu4(a1, b1);
+    v0 = SIGNED ? __vmaxs4(v0, v0 >> 8) : __vmaxu4(v0, v0 >> 8);    // bytes 0 and 2 hold the pair maxima
+    v1 = SIGNED ? __vmaxs4(v1, v1 >> 8) : __vmaxu4(v1, v1 >> 8);
+    return __byte_perm(v0, v1, 0x6420);
 }
 
 // N: pixels per packed word; SC: slot width when known at compile time (0: read from the parameters);
@@ -404,11 +426,13 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     // where each position's pixels go (channel 0): element offset and number of pixels to store (0: none)
     size_t pix_off[TM];
     int pix_n[TM];
+    int tile_pos[TM];                                                // staged output: byte offset of the position's first pixel in a channel's tile
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
         const int pos = wpos0 + i * lanes_m + lm;
         pix_off[i] = 0;
         pix_n[i] = 0;
+        tile_pos[i] = 0;
         if (pos < TP) {
             const int r = small_div(pos, p.XB, inv_xb), xbl = pos - r * p.XB;
             const int xg = seg * p.XO + xbl - p.J;                   // output block in the row; halo positions give no pixels
@@ -417,11 +441,15 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 const int b = b0 + db, h = h0 + r - db * p.Ho;
                 pix_off[i] = (((size_t)b * p.Co) * p.Ho + h) * p.Wo + (size_t)xg * N;
                 pix_n[i] = min(N, p.Wo - xg * N);
+                tile_pos[i] = r * p.WTP + (xbl - p.J) * N;
             }
         }
     }
     const size_t chan_stride = (size_t)p.Ho * p.Wo;
 
+    if (UNPACKED && p.requant && p.stage_out) __syncthreads();     // the staged tile reuses the operand buffers of the main loop
+    int8_t *tile = reinterpret_cast<int8_t *>(smem + p.tile_off);
+    const int tile_chan = p.TR * p.WTP;                              // bytes per channel of the staged tile
     // ---- overlap-add, optional requantisation (arithmetic shift, clamp), store
     auto finish = [&](auto requant_tag) {
         constexpr bool REQ = decltype(requant_tag)::value;
@@ -459,7 +487,10 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                     int32_t v = (int32_t)Y[m];
                     if constexpr (REQ) {
                         v = max(p.lo, min(p.hi, v >> p.shift));
-                        if (m < n_store) ((int8_t *)p.out)[o + m] = (int8_t)v;
+                        if (m < n_store) {
+                            if (p.stage_out) tile[(tn * TN + t) * tile_chan + tile_pos[i] + m] = (int8_t)v;
+                            else ((int8_t *)p.out)[o + m] = (int8_t)v;
+                        }
                     } else {
                         if (m < n_store) ((int32_t *)p.out)[o + m] = v;
                     }
@@ -469,6 +500,92 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     };
     if (p.requant) finish(std::true_type());
     else finish(std::false_type());
+    if (!(p.requant && p.stage_out)) return;
+
+    // ---- staged codes leave the CTA: whole rows in pieces of `vec` bytes, optionally max-pooled 2x2 on the way
+    __syncthreads();
+    const int col0 = seg * p.XO * N;                                 // first output column of this row segment
+    const int wn = min(p.Wo - col0, p.XO * N);                       // columns of this segment
+    const int ncv = min(p.TCO, p.Co - co0);                          // channels of this tile that exist
+    if (p.out_bits < 8) {
+        // dense codes: every output byte gathers 8 / out_bits neighbouring codes of a row (rows and segments start on
+        // byte boundaries, checked on the host); with pool each code is the maximum of a 2x2 window first
+        const int ob = p.out_bits, cpb = 8 / ob, sh = p.pool ? 1 : 0;
+        const uint32_t cmask = (1u << ob) - 1u;
+        const int Hq = p.Ho >> sh, Wq = p.Wo >> sh, TRq = TRe >> sh;
+        const int ppr = ((((wn >> sh) * ob) >> 3)) / p.vec;          // pieces of `vec` dense bytes per row
+        const float inv_ppr = 1.0f / (float)ppr, inv_tr = 1.0f / (float)TRq;
+        for (int idx = tid; idx < ncv * TRq * ppr; idx += nthreads) {
+            const int rr = small_div(idx, ppr, inv_ppr), piece = idx - rr * ppr;
+            const int cl = small_div(rr, TRq, inv_tr), rq = rr - cl * TRq;
+            const int r = rq << sh;
+            const int db = small_div(h0 + r, p.Ho, inv_ho);
+            const int b = b0 + db, h = h0 + r - db * p.Ho;
+            const int8_t *src = tile + cl * tile_chan + r * p.WTP;
+            const size_t e0 = ((((size_t)b * p.Co + co0 + cl) * Hq + (h >> sh)) * Wq + (col0 >> sh));   // first code of this segment's row
+            uint8_t *dst = (uint8_t *)p.out + ((e0 * ob) >> 3) + piece * p.vec;
+            uint32_t word = 0;
+            for (int u = 0; u < p.vec; ++u) {
+                uint32_t byte = 0;
+                for (int c = 0; c < cpb; ++c) {
+                    const int col = (piece * p.vec + u) * cpb + c;           // code index within the segment's (pooled) row
+                    int v;
+                    if (p.pool) {
+                        int a0 = src[2 * col], a1 = src[2 * col + 1], c0 = src[p.WTP + 2 * col], c1 = src[p.WTP + 2 * col + 1];
+                        if (!p.out_signed) { a0 &= 0xFF; a1 &= 0xFF; c0 &= 0xFF; c1 &= 0xFF; }
+                        v = max(max(a0, a1), max(c0, c1));
+                    } else {
+                        v = src[col];
+                    }
+                    byte |= ((uint32_t)v & cmask) << (ob * c);
+                }
+                word |= byte << (8 * u);
+            }
+            if (p.vec == 4) *reinterpret_cast<uint32_t *>(dst) = word;
+            else *dst = (uint8_t)word;
+        }
+    } else if (!p.pool) {
+        const int ppr = wn / p.vec;                                  // pieces per row (vec divides Wo and col0)
+        const float inv_ppr = 1.0f / (float)ppr, inv_tr = 1.0f / (float)TRe;
+        for (int idx = tid; idx < ncv * TRe * ppr; idx += nthreads) {
+            const int rr = small_div(idx, ppr, inv_ppr), piece = idx - rr * ppr;
+            const int cl = small_div(rr, TRe, inv_tr), r = rr - cl * TRe;
+            const int db = small_div(h0 + r, p.Ho, inv_ho);
+            const int b = b0 + db, h = h0 + r - db * p.Ho;
+            const int8_t *src = tile + cl * tile_chan + r * p.WTP + piece * p.vec;
+            int8_t *dst = (int8_t *)p.out + (((size_t)b * p.Co + co0 + cl) * p.Ho + h) * p.Wo + col0 + piece * p.vec;
+            if (p.vec == 16) *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(src);
+            else if (p.vec == 8) *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(src);
+            else if (p.vec == 4) *reinterpret_cast<uint32_t *>(dst) = *reinterpret_cast<const uint32_t *>(src);
+            else *dst = *src;
+        }
+    } else {
+        const int Hq = p.Ho >> 1, Wq = p.Wo >> 1, TRq = TRe >> 1;
+        const int ppr = (wn >> 1) / p.vec;                           // pooled pieces per row
+        const float inv_ppr = 1.0f / (float)ppr, inv_tr = 1.0f / (float)TRq;
+        for (int idx = tid; idx < ncv * TRq * ppr; idx += nthreads) {
+            const int rr = small_div(idx, ppr, inv_ppr), piece = idx - rr * ppr;
+            const int cl = small_div(rr, TRq, inv_tr), rq = rr - cl * TRq;
+            const int r = 2 * rq;
+            const int db = small_div(h0 + r, p.Ho, inv_ho);
+            const int b = b0 + db, h = h0 + r - db * p.Ho;
+            const int8_t *src = tile + cl * tile_chan + r * p.WTP + piece * 2 * p.vec;
+            int8_t *dst = (int8_t *)p.out + (((size_t)b * p.Co + co0 + cl) * Hq + (h >> 1)) * Wq + (col0 >> 1) + piece * p.vec;
+            if (p.vec == 8) {
+                const uint4 r0 = *reinterpret_cast<const uint4 *>(src), r1 = *reinterpret_cast<const uint4 *>(src + p.WTP);
+                const uint2 v = p.out_signed ? make_uint2(pool_pairs<true>(r0.x, r0.y, r1.x, r1.y), pool_pairs<true>(r0.z, r0.w, r1.z, r1.w))
+                                             : make_uint2(pool_pairs<false>(r0.x, r0.y, r1.x, r1.y), pool_pairs<false>(r0.z, r0.w, r1.z, r1.w));
+                *reinterpret_cast<uint2 *>(dst) = v;
+            } else if (p.vec == 4) {
+                const uint2 r0 = *reinterpret_cast<const uint2 *>(src), r1 = *reinterpret_cast<const uint2 *>(src + p.WTP);
+                *reinterpret_cast<uint32_t *>(dst) = p.out_signed ? pool_pairs<true>(r0.x, r0.y, r1.x, r1.y) : pool_pairs<false>(r0.x, r0.y, r1.x, r1.y);
+            } else {
+                int a0 = src[0], a1 = src[1], c0 = src[p.WTP], c1 = src[p.WTP + 1];
+                if (!p.out_signed) { a0 &= 0xFF; a1 &= 0xFF; c0 &= 0xFF; c1 &= 0xFF; }
+                *dst = (int8_t)max(max(a0, a1), max(c0, c1));
+            }
+        }
+    }
 }
 
 // Reversed, packed kernel rows (Theorem 3: g = W[co][ci][kh][K-1:0], then Eq. 5 per chunk of Kc taps).
@@ -478,7 +595,19 @@ struct WeightPackParams {
     const int8_t *w;
     uint32_t *wp;
     int Co, Ci, K, J, Kc, S, w_signed, CoP, total;
+    int w_bits;                // storage: 8 = one code per byte, 1 / 2 / 4 = dense (8 / w_bits codes per byte)
 };
+
+// Code number e of a tensor stored densely with `bits` (1, 2, 4 or 8) bits per code: code e occupies bits
+// [(e bits) % 8, (e bits) % 8 + bits) of byte (e bits) / 8, two's complement when signed (Section V-B: weights and
+// features kept compressed in memory and unpacked as they are read).
+__device__ __forceinline__ int32_t load_dense_code(const int8_t *base, size_t e, int bits, bool is_signed) {
+    const size_t bit = e * (size_t)bits;
+    const uint32_t byte = (uint8_t)__ldg(base + (bit >> 3));
+    const uint32_t v = (byte >> (int)(bit & 7)) & ((1u << bits) - 1u);
+    const uint32_t sb = 1u << (bits - 1);
+    return is_signed ? (int32_t)((v ^ sb) - sb) : (int32_t)v;
+}
 
 __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int idx) {
     if (idx >= q.total) return;
@@ -490,12 +619,17 @@ __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int 
     const int ci = rest / q.K;
     uint32_t word = 0;
     if (co < q.Co) {
-        const int8_t *row = q.w + (((size_t)co * q.Ci + ci) * q.K + kh) * q.K;
+        const size_t row_e = (((size_t)co * q.Ci + ci) * q.K + kh) * q.K;       // first code of the kernel row
         for (int k = 0; k < q.Kc; ++k) {
             const int g_idx = j * q.Kc + k;              // index into the reversed row
             if (g_idx < q.K) {
-                const int8_t raw = __ldg(row + (q.K - 1 - g_idx));
-                const int32_t v = q.w_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+                int32_t v;
+                if (q.w_bits == 8) {
+                    const int8_t raw = __ldg(q.w + row_e + (q.K - 1 - g_idx));
+                    v = q.w_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+                } else {
+                    v = load_dense_code(q.w, row_e + (q.K - 1 - g_idx), q.w_bits, q.w_signed != 0);
+                }
                 word += (uint32_t)v << (q.S * k);
             }
         }
@@ -509,10 +643,12 @@ __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int 
 // One thread packs four consecutive words of a row (one 16-byte store); a CTA stays within one
 // (ci, b) plane, whose rows are contiguous in both the input and the packed layout.  The CTAs past the
 // activation planes pack the kernel rows (one word per thread), so that a layer needs one packing launch.
+// x_bits: storage of the activations, 8 = one code per byte, 1 / 2 / 4 = dense.
 template <bool XS, int N>
 __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
                                                             int pad, int K, int J, int S, int XBT, int blocks_per_plane,
-                                                            uint32_t *__restrict__ ap, int act_blocks, const WeightPackParams wq) {
+                                                            uint32_t *__restrict__ ap, int act_blocks, const WeightPackParams wq,
+                                                            int x_bits) {
     grid_dependency_release();
     grid_dependency_wait();                                          // the input may come from the kernel before; the workspace may still be read by it
     if ((int)blockIdx.x >= act_blocks) {
@@ -528,29 +664,28 @@ __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__rest
     const int hi = hp - pad;
     uint32_t word[4] = {0u, 0u, 0u, 0u};
     if (hi >= 0 && hi < H) {
-        const int8_t *row = x + (((size_t)b * Ci + ci) * H + hi) * W;
+        const size_t row_e = (((size_t)b * Ci + ci) * H + hi) * W;  // first code of the input row
         const int col0 = (4 * q - J) * N + K - 1 - pad;              // input column of slot 0 of the first word
+        if (x_bits == 8) {
+            const int8_t *row = x + row_e;
 #pragma unroll
-        for (int w = 0; w < 4; ++w)
+            for (int w = 0; w < 4; ++w)
 #pragma unroll
-            for (int n = 0; n < N; ++n) {
-                const int col = col0 + w * N + n;
-                if (col >= 0 && col < W) word[w] += (uint32_t)load_code<XS>(row + col) << (S * n);
-            }
+                for (int n = 0; n < N; ++n) {
+                    const int col = col0 + w * N + n;
+                    if (col >= 0 && col < W) word[w] += (uint32_t)load_code<XS>(row + col) << (S * n);
+                }
+        } else {
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+#pragma unroll
+                for (int n = 0; n < N; ++n) {
+                    const int col = col0 + w * N + n;
+                    if (col >= 0 && col < W) word[w] += (uint32_t)load_dense_code(x, row_e + col, x_bits, XS) << (S * n);
+                }
+        }
     }
     *reinterpret_cast<uint4 *>(ap + ((size_t)plane * Hp + hp) * XBT + 4 * q) = make_uint4(word[0], word[1], word[2], word[3]);
-}
-
-// VEC input bytes of two rows per thread (VEC = 8: two 8-byte loads, one 4-byte store; VEC = 16: two
-// 16-byte loads, one 8-byte store), per-byte maxima; needs W % VEC == 0 and VEC-byte aligned input,
-// VEC/2-byte aligned output.
-template <bool SIGNED>
-__device__ __forceinline__ uint32_t pool_pairs(uint32_t a0, uint32_t a1, uint32_t b0, uint32_t b1) {
-    uint32_t v0 = SIGNED ? __vmaxs4(a0, b0) : __vmaxu4(a0, b0);     // the two rows
-    uint32_t v1 = SIGNED ? __vmaxs4(a1, b1) : __vmaxu4(a1, b1);
-    v0 = SIGNED ? __vmaxs4(v0, v0 >> 8) : __vmaxu4(v0, v0 >> 8);    // bytes 0 and 2 hold the pair maxima
-    v1 = SIGNED ? __vmaxs4(v1, v1 >> 8) : __vmaxu4(v1, v1 >> 8);
-    return __byte_perm(v0, v1, 0x6420);
 }
 
 template <bool SIGNED, int VEC>
@@ -673,7 +808,7 @@ struct TileChoice {
 // (an SM with fewer threads than that cannot fill the multiply pipe), adds the staging work of a
 // tile relative to its multiply work, and divides by the useful work.
 static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int J, int Co, int TM, int TN, int sms,
-                               int force_tr) {
+                               int force_tr, bool even_rows = false, int xo_mult = 4) {
     TileChoice best;
     best.cost = -1.0;
     for (int TNX = 1; TNX <= 16; TNX *= 2) {
@@ -687,10 +822,12 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
         const int rowmax = std::min(maxpos, 64);                  // a staged row holds at most 64 words
         int NSEG = 1, XO = X;
         if (X + J > rowmax) {
-            XO = (rowmax - J) / 4 * 4;
-            if (XO < 4) continue;
+            // xo_mult: a multiple of 4 (16-byte pieces of the packed rows); larger when the segments of a dense output
+            // row have to start on byte boundaries
+            XO = (rowmax - J) / xo_mult * xo_mult;
+            if (XO < xo_mult) continue;
             NSEG = ceil_div(X, XO);
-            XO = (ceil_div(X, NSEG) + 3) / 4 * 4;
+            XO = std::min(XO, (ceil_div(X, NSEG) + xo_mult - 1) / xo_mult * xo_mult);
             NSEG = ceil_div(X, XO);
         }
         const int XB = XO + J;
@@ -698,6 +835,7 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
         const int tr_lo = force_tr > 0 ? std::min(force_tr, tr_hi) : 1;
         const int tr_end = force_tr > 0 ? tr_lo : tr_hi;
         for (int TR = tr_lo; TR <= tr_end; ++TR) {
+            if (even_rows && (TR & 1)) continue;                      // a fused 2x2 pool needs both rows of a pair in one CTA
             int TMX = ceil_div(TR * XB, TM);
             int threads = (TMX * TNX + 31) / 32 * 32;               // whole warps
             if (threads > kMaxThreads2D) continue;
@@ -730,7 +868,8 @@ static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int 
 }
 
 static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, int pad, int p, int q, int xs, int ws,
-                      int requant, int shift, int lo, int hi, int algo, const hikonv_tuning_t *tune, Conv2dSetup *s) {
+                      int requant, int shift, int lo, int hi, int algo, const hikonv_tuning_t *tune, Conv2dSetup *s,
+                      int pool = 0, const void *d_out = nullptr, int out_bits = 8) {
     if (B < 1 || Ci < 1 || H < 1 || W < 1 || Co < 1 || K < 1 || K > kMaxK) return HIKONV_ERR_INVALID_ARG;
     if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
     if (stride != 1 || pad < 0 || pad >= K) return HIKONV_ERR_UNSUPPORTED;
@@ -773,7 +912,17 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.requant = requant ? 1 : 0; kp.shift = shift; kp.lo = lo; kp.hi = hi;
     kp.total_rows = B * Ho;
     kp.X = ceil_div(Wo, N);
-    const TileChoice tc = choose_tiles(kp.total_rows, Ho, kp.X, N, K, L.J, Co, TM, TN, sm_count(), tune ? tune->tile : 0);
+    int xo_mult = 4;
+    if (requant && out_bits < 8 && out_bits > 0) {
+        // segment width in codes (halved by the pool) times out_bits must be a multiple of 8
+        const int unit = pool ? 16 : 8;
+        int g = N * out_bits, a = unit;
+        while (a) { const int t = g % a; g = a; a = t; }               // g = gcd(N out_bits, unit)
+        const int need = unit / g;
+        while (xo_mult % need != 0) xo_mult += 4;
+    }
+    const TileChoice tc = choose_tiles(kp.total_rows, Ho, kp.X, N, K, L.J, Co, TM, TN, sm_count(), tune ? tune->tile : 0,
+                                       requant && pool, xo_mult);
     if (tc.cost < 0) return HIKONV_ERR_UNSUPPORTED;
     kp.TNX = tc.TNX; kp.TMX = tc.TMX; kp.TCO = tc.TNX * TN;
     kp.NSEG = tc.NSEG; kp.XO = tc.XO; kp.XB = tc.XB; kp.TR = tc.TR;
@@ -820,7 +969,40 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.b_words = CK * K * L.J * kBPitch;
     const size_t words = (size_t)kp.b_off + 2 * (size_t)kp.b_words;
     const size_t xch_words = s->unpacked ? 0 : (size_t)kp.TMX * N * kp.TCO;
-    kp.e_off = (int)((std::max(words, xch_words) + 3) / 4 * 4);
+    // requantised codes are staged per CTA ([channel][row][column] bytes, behind the exchange area) and written in
+    // the widest pieces that divide every row start: Wo, the segment width and the output address
+    size_t stage_words = 0;
+    kp.stage_out = 0;
+    kp.pool = 0;
+    kp.out_bits = 8;
+    if (!requant && (pool || out_bits != 8)) return HIKONV_ERR_INVALID_ARG;
+    if (requant && (pool || out_bits != 8)) {
+        // (plain byte output keeps direct stores: staged, it measured 3 % slower on the 56x56 layer)
+        if (out_bits != 8 && out_bits != 4 && out_bits != 2 && out_bits != 1) return HIKONV_ERR_INVALID_ARG;
+        if (pool && ((Ho | Wo) & 1)) return HIKONV_ERR_UNSUPPORTED;        // the fused 2x2 pool wants even output sizes
+        if (out_bits < 8 && (lo < (lo < 0 ? -(1 << (out_bits - 1)) : 0) || hi > (lo < 0 ? (1 << (out_bits - 1)) - 1 : (1 << out_bits) - 1)))
+            return HIKONV_ERR_INVALID_ARG;                                  // the clamp range must fit the stored width
+        kp.stage_out = 1;
+        kp.pool = pool ? 1 : 0;
+        kp.out_signed = lo < 0 ? 1 : 0;
+        kp.out_bits = out_bits;
+        kp.WTP = (kp.XO * N + 15) / 16 * 16;
+        kp.tile_off = (int)((xch_words + 3) / 4 * 4);
+        stage_words = (size_t)kp.tile_off + (size_t)kp.TCO * kp.TR * kp.WTP / 4;
+        const int w_out = pool ? Wo / 2 : Wo, seg_out = pool ? kp.XO * N / 2 : kp.XO * N;
+        if (pool && kp.NSEG > 1 && ((kp.XO * N) & 1)) return HIKONV_ERR_UNSUPPORTED;
+        if (out_bits == 8) {
+            int vec = pool ? 8 : 16;
+            while (vec > 1 && (w_out % vec != 0 || (kp.NSEG > 1 && seg_out % vec != 0) || ((uintptr_t)d_out % vec) != 0)) vec /= 2;
+            kp.vec = vec == 2 ? 1 : vec;
+        } else {
+            // rows and row segments must start on byte boundaries of the dense output
+            if ((w_out * out_bits) % 8 != 0 || (kp.NSEG > 1 && (seg_out * out_bits) % 8 != 0)) return HIKONV_ERR_UNSUPPORTED;
+            const int row_bytes = w_out * out_bits / 8, seg_bytes = seg_out * out_bits / 8;
+            kp.vec = (row_bytes % 4 == 0 && (kp.NSEG == 1 || seg_bytes % 4 == 0) && ((uintptr_t)d_out % 4) == 0) ? 4 : 1;
+        }
+    }
+    kp.e_off = (int)((std::max(std::max(words, xch_words), stage_words) + 3) / 4 * 4);
     const size_t e_words = s->unpacked ? 0 : (size_t)kEPitch * s->threads * 2;
     s->smem_bytes = ((size_t)kp.e_off + e_words) * 4 + 16;
     s->wp_bytes = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
@@ -877,14 +1059,16 @@ extern "C" size_t hikonv_conv2d_workspace_bytes(int B, int Ci, int H, int W, int
     return weights + align_up(acts, 256);
 }
 
-extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K, int stride,
-                             int pad, int p, int q, int x_signed, int w_signed, void *d_out, int requant, int shift, int lo,
-                             int hi, void *d_workspace, size_t workspace_bytes, int algo, const hikonv_tuning_t *tune,
-                             void *stream) {
+// One layer: packing launch, then the layer kernel.  x_bits / w_bits: storage of activations and weights (8 = one code
+// per byte, else dense); out_bits and pool describe the requantised output (see make_setup).
+static int conv2d_run(const void *d_x, int x_bits, int B, int Ci, int H, int W, const void *d_w, int w_bits, int Co, int K,
+                      int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out, int out_bits, int requant,
+                      int shift, int lo, int hi, int pool, void *d_workspace, size_t workspace_bytes, int algo,
+                      const hikonv_tuning_t *tune, void *stream) {
     if (!d_x || !d_w || !d_out) return HIKONV_ERR_INVALID_ARG;
     Conv2dSetup s;
     int rc = make_setup(B, Ci, H, W, Co, K, stride, pad, p, q, x_signed ? 1 : 0, w_signed ? 1 : 0, requant, shift, lo, hi, algo,
-                        tune, &s);
+                        tune, &s, pool, d_out, out_bits);
     if (rc != HIKONV_OK) return rc;
     if (!requant && ((uintptr_t)d_out % 4) != 0) return HIKONV_ERR_INVALID_ARG;
     const size_t need = s.wp_bytes + s.ap_words * sizeof(uint32_t);
@@ -894,22 +1078,22 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
     cudaStream_t st = (cudaStream_t)stream;
     uint32_t *d_wp = (uint32_t *)d_workspace;
     uint32_t *d_ap = (uint32_t *)((char *)d_workspace + s.wp_bytes);
-    s.kp.x = d_x;
+    s.kp.x = (const int8_t *)d_x;
     s.kp.wp = d_wp;
     s.kp.ap = d_ap;
     s.kp.out = d_out;
     // a2: reversed kernel rows packed per (ci, kh, chunk); a3: activation rows packed per block; one launch
     {
         WeightPackParams wq;
-        wq.w = d_w; wq.wp = d_wp; wq.Co = Co; wq.Ci = Ci; wq.K = K; wq.J = s.L.J; wq.Kc = s.L.Kc; wq.S = s.L.S;
-        wq.w_signed = w_signed ? 1 : 0; wq.CoP = s.kp.CoP; wq.total = Ci * K * s.L.J * s.kp.CoP;
+        wq.w = (const int8_t *)d_w; wq.wp = d_wp; wq.Co = Co; wq.Ci = Ci; wq.K = K; wq.J = s.L.J; wq.Kc = s.L.Kc; wq.S = s.L.S;
+        wq.w_signed = w_signed ? 1 : 0; wq.CoP = s.kp.CoP; wq.total = Ci * K * s.L.J * s.kp.CoP; wq.w_bits = w_bits;
         const int bpp = ceil_div(s.kp.Hp * (s.kp.XBT / 4), 256);
         const size_t act_blocks = (size_t)Ci * B * bpp, w_blocks = (size_t)ceil_div(wq.total, 256);
         if (act_blocks + w_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
         const unsigned grid = (unsigned)(act_blocks + w_blocks);
 #define HK_PACK(XSIGN, NN)                                                                                                 \
-    rc = launch_dependent(pack_operands_kernel<XSIGN, NN>, dim3(grid), dim3(256), 0, st, d_x, B, Ci, H, W, s.kp.Hp, pad, K, s.L.J, \
-                          s.L.S, s.kp.XBT, bpp, d_ap, (int)act_blocks, wq)
+    rc = launch_dependent(pack_operands_kernel<XSIGN, NN>, dim3(grid), dim3(256), 0, st, (const int8_t *)d_x, B, Ci, H, W, s.kp.Hp, \
+                          pad, K, s.L.J, s.L.S, s.kp.XBT, bpp, d_ap, (int)act_blocks, wq, x_bits)
         switch (s.L.N * 2 + (x_signed ? 1 : 0)) {
             case 2: HK_PACK(false, 1); break;
             case 3: HK_PACK(true, 1); break;
@@ -925,6 +1109,32 @@ extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, con
     }
     if (rc != HIKONV_OK) return rc;
     return launch_conv2d(s, st);
+}
+
+extern "C" int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K, int stride,
+                             int pad, int p, int q, int x_signed, int w_signed, void *d_out, int requant, int shift, int lo,
+                             int hi, void *d_workspace, size_t workspace_bytes, int algo, const hikonv_tuning_t *tune,
+                             void *stream) {
+    return conv2d_run(d_x, 8, B, Ci, H, W, d_w, 8, Co, K, stride, pad, p, q, x_signed, w_signed, d_out, 8, requant, shift, lo, hi, 0,
+                      d_workspace, workspace_bytes, algo, tune, stream);
+}
+
+static bool storage_bits_ok(int store_bits, int code_bits) {
+    return store_bits == 8 || (store_bits == code_bits && (code_bits == 1 || code_bits == 2 || code_bits == 4));
+}
+
+extern "C" int hikonv_conv2d_dense(const void *d_x, int x_store_bits, int B, int Ci, int H, int W, const void *d_w,
+                                   int w_store_bits, int Co, int K, int stride, int pad, int p, int q, int x_signed,
+                                   int w_signed, void *d_out, int out_store_bits, int requant, int shift, int lo, int hi,
+                                   int pool, void *d_workspace, size_t workspace_bytes, int algo,
+                                   const hikonv_tuning_t *tune, void *stream) {
+    if (validate_codes(p, q) != HIKONV_OK) return HIKONV_ERR_INVALID_ARG;
+    if (!storage_bits_ok(x_store_bits, p) || !storage_bits_ok(w_store_bits, q)) return HIKONV_ERR_UNSUPPORTED;
+    if (!requant && out_store_bits != 32) return HIKONV_ERR_INVALID_ARG;
+    if (requant && out_store_bits != 8 && out_store_bits != 4 && out_store_bits != 2 && out_store_bits != 1)
+        return HIKONV_ERR_INVALID_ARG;
+    return conv2d_run(d_x, x_store_bits, B, Ci, H, W, d_w, w_store_bits, Co, K, stride, pad, p, q, x_signed, w_signed, d_out,
+                      requant ? out_store_bits : 8, requant, shift, lo, hi, pool, d_workspace, workspace_bytes, algo, tune, stream);
 }
 
 // ---- scratch that needs no allocation: a fixed buffer inside the library image, one copy per GPU

@@ -50,6 +50,19 @@ def to_dense(values: np.ndarray, bits: int) -> np.ndarray:
     return np.ascontiguousarray((v << shifts).sum(axis=1).astype(np.uint8))
 
 
+def from_dense(dense: np.ndarray, count: int, bits: int, signed: bool) -> np.ndarray:
+    """Dense storage -> the first ``count`` code values (the inverse of ``to_dense``)."""
+    if bits not in (1, 2, 4, 8):
+        raise ValueError("bits must divide 8")
+    per = 8 // bits
+    b = np.asarray(dense, dtype=np.uint8).astype(np.int64)
+    shifts = (np.arange(per) * bits).astype(np.int64)
+    v = ((b[:, None] >> shifts) & ((1 << bits) - 1)).reshape(-1)[:count]
+    if signed:
+        v = np.where(v >= (1 << (bits - 1)), v - (1 << bits), v)
+    return v
+
+
 def from_storage(stored: np.ndarray, signed: bool) -> np.ndarray:
     """int8 storage bytes -> code values as int64."""
     s = np.asarray(stored)
