@@ -199,8 +199,8 @@ int hikonv_conv1d_layout(int p, int q, int f_signed, int g_signed, int K, const 
  * [(e p) % 8, (e p) % 8 + p) of byte (e p) / 8 (two's complement when f_signed); the unused bits of the
  * last byte are ignored.  ceil(len p / 8) bytes, device, caller-owned; any alignment is accepted, 4-byte
  * alignment takes the fast path.  d_g, d_y, q, K, tune, stream as for hikonv_conv1d.
- * Built for the layouts of K in {3, 5, 7} with q == p and g_signed == f_signed; any other combination
- * returns HIKONV_ERR_UNSUPPORTED (nothing is launched).
+ * Built for the layouts of K in {3, 5, 7} with q == p (signed or unsigned operands in any combination); any
+ * other combination returns HIKONV_ERR_UNSUPPORTED (nothing is launched).
  */
 int hikonv_conv1d_dense(const uint8_t *d_f_dense, size_t len, const int8_t *d_g, int K, int p, int q,
                         int f_signed, int g_signed, int32_t *d_y, const hikonv_tuning_t *tune,

@@ -310,13 +310,14 @@ int launch_conv1d_packed_tc(const Conv1dTcParams &p, int N, int J, bool sp, bool
     return HIKONV_ERR_UNSUPPORTED;
 }
 
-// Dense input: the layouts of the 1-, 2- and 4-bit cases of the sweep (K = 3, 5, 7; both operands unsigned or
-// both signed), slot width at compile time.
+// Dense input: the layouts of the 1-, 2- and 4-bit cases of the sweep (K = 3, 5, 7; any combination of signed and
+// unsigned operands: the mixed cases take the same (N, J, S)), slot width at compile time.
 #define HK_DENSE_LAYOUTS(X) X(1, 11, 1, 3) X(1, 8, 1, 4) X(2, 6, 1, 6) X(2, 5, 1, 6) X(2, 5, 1, 7) X(2, 5, 2, 7) \
                             X(4, 3, 1, 10) X(4, 3, 2, 11) X(4, 3, 3, 11)
 
 bool conv1d_packed_dense_available(int P, int N, int J, int S, bool sp, bool fs) {
-    if (sp != fs) return false;
+    (void)sp;
+    (void)fs;
 #define HK_X(pp, n, j, sc) if (P == pp && N == n && J == j && S == sc) return true;
     HK_DENSE_LAYOUTS(HK_X)
 #undef HK_X
@@ -324,10 +325,10 @@ bool conv1d_packed_dense_available(int P, int N, int J, int S, bool sp, bool fs)
 }
 
 int launch_conv1d_packed_dense(const Conv1dTcParams &p, int P, int N, int J, bool sp, bool fs, cudaStream_t st) {
-    if (sp != fs) return HIKONV_ERR_UNSUPPORTED;
 #define HK_X(pp, n, j, sc)                                                                                       \
     if (P == pp && N == n && J == j && p.S == sc) {                                                              \
         if (fs) return launch_persistent(conv1d_packed_tc_kernel<n, j, sc, true, true, pp>, p, st);             \
+        if (sp) return launch_persistent(conv1d_packed_tc_kernel<n, j, sc, true, false, pp>, p, st);            \
         return launch_persistent(conv1d_packed_tc_kernel<n, j, sc, false, false, pp>, p, st);                   \
     }
     HK_DENSE_LAYOUTS(HK_X)

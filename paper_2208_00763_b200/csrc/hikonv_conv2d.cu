@@ -808,10 +808,14 @@ struct TileChoice {
 // (an SM with fewer threads than that cannot fill the multiply pipe), adds the staging work of a
 // tile relative to its multiply work, and divides by the useful work.
 static TileChoice choose_tiles(int total_rows, int Ho, int X, int N, int K, int J, int Co, int TM, int TN, int sms,
-                               int force_tr, bool even_rows = false, int xo_mult = 4) {
+                               int force_tr, bool even_rows = false, int xo_mult = 4, int force_tnx = 0) {
     TileChoice best;
     best.cost = -1.0;
-    for (int TNX = 1; TNX <= 16; TNX *= 2) {
+    // More than four channel lanes (16 channels per CTA) never measured faster than four on the benchmark layers
+    // (sweeps over every TNX and tile height: 10x20 to 160x320 maps, 3 to 256 input channels); the automatic choice
+    // stays within 1 .. 4, a forced value may go up to 16.
+    for (int TNX = 1; TNX <= (force_tnx > 0 ? 16 : 4); TNX *= 2) {
+        if (force_tnx > 0 && TNX != force_tnx) continue;
         const int TCO = TNX * TN;
         if (TNX > 1 && TCO / 2 >= Co) break;                       // more channel lanes than channels
         const int gy = ceil_div(Co, TCO);
@@ -921,8 +925,10 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         const int need = unit / g;
         while (xo_mult % need != 0) xo_mult += 4;
     }
-    const TileChoice tc = choose_tiles(kp.total_rows, Ho, kp.X, N, K, L.J, Co, TM, TN, sm_count(), tune ? tune->tile : 0,
-                                       requant && pool, xo_mult);
+    // tune->tile > 0: rows per CTA, plus 1000 x channel lanes per CTA (1, 2, 4, 8, 16) when those are forced too
+    const int tile_arg = (tune && tune->tile > 0) ? tune->tile : 0;
+    const TileChoice tc = choose_tiles(kp.total_rows, Ho, kp.X, N, K, L.J, Co, TM, TN, sm_count(), tile_arg % 1000,
+                                       requant && pool, xo_mult, tile_arg / 1000);
     if (tc.cost < 0) return HIKONV_ERR_UNSUPPORTED;
     kp.TNX = tc.TNX; kp.TMX = tc.TMX; kp.TCO = tc.TNX * TN;
     kp.NSEG = tc.NSEG; kp.XO = tc.XO; kp.XB = tc.XB; kp.TR = tc.TR;
@@ -1031,6 +1037,10 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
     // 8-bit activations x 4-bit weights with few input channels (a network's first layer): no moves at all
     if (s.L.N == 2 && s.L.S == 17 && K == 3 && J == 2 && s.L.M >= s.kp.Ci * K && s.kp.move_every == 0)
         return launch_variant<2, 17, kTM, kTN, false, 3, 2, false, true>(s, sp, st);
+    // two pixels per word in 16-bit slots, the three taps of a kernel row in one word: 64 bits exactly, and room for
+    // up to 270 accumulated 4-bit products per slot, so layers of up to 90 input channels never move anything
+    if (s.L.N == 2 && s.L.S == 16 && K == 3 && J == 1 && s.L.M >= s.kp.Ci * K && s.kp.move_every == 0)
+        return launch_variant<2, 16, kTM, kTN, false, 3, 1, false, true>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     switch (s.L.N) {

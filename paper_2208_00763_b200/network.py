@@ -43,15 +43,27 @@ class CompactCnn:
         self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         self._ws_shape = tuple(shape)
 
-    def forward(self, d_x: torch.Tensor, algo: int = hk.ALGO_PACKED32, keep_activations: bool = False, stream=None):
+    def forward(self, d_x: torch.Tensor, algo: int = hk.ALGO_PACKED32, keep_activations: bool = False, stream=None,
+                fused_pool: bool = False):
+        """``fused_pool``: layers followed by a pool run it inside their epilogue (``hikonv_conv2d_dense`` with one code
+        per byte); otherwise the pool is a launch of its own (the default: on the benchmark network the staged
+        epilogue costs what the separate pool launch does)."""
         self._ensure_workspace(d_x.shape)
         acts = []
         a = d_x
         for L in self.layers:
-            a = hk.conv2d(a, L["d_w"], L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"],
-                          requant=(L["shift"], L["lo"], L["hi"]), algo=algo, workspace=self.workspace, stream=stream)
-            if L["pool"]:
-                a = hk.maxpool2x2_i8(a, is_signed=L["lo"] < 0, stream=stream)
+            rq = (L["shift"], L["lo"], L["hi"])
+            if L["pool"] and fused_pool:
+                B, Ci, H, W = a.shape
+                Co, _, K, _ = L["d_w"].shape
+                a = hk.conv2d_dense(a.reshape(-1), (B, Ci, H, W), 8, L["d_w"].reshape(-1), tuple(L["d_w"].shape), 8, L["pad"], L["p"],
+                                    L["q"], L["x_signed"], L["w_signed"], requant=rq, out_store_bits=8, pool=True, algo=algo,
+                                    workspace=self.workspace, stream=stream)
+            else:
+                a = hk.conv2d(a, L["d_w"], L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], requant=rq, algo=algo,
+                              workspace=self.workspace, stream=stream)
+                if L["pool"]:
+                    a = hk.maxpool2x2_i8(a, is_signed=L["lo"] < 0, stream=stream)
             if keep_activations:
                 acts.append(a)
         last = self.layers[-1]

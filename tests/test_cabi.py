@@ -190,7 +190,11 @@ def test_device_entry_points_validate_before_touching_cuda():
     # dense input: null pointers, widths that straddle bytes, layouts that are not instantiated
     assert lib.hikonv_conv1d_dense(None, 10, 8, 3, 4, 4, 0, 0, 8, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_conv1d_dense(8, 10, 8, 3, 3, 3, 0, 0, 8, None, None) == hk.ERR_UNSUPPORTED
-    assert lib.hikonv_conv1d_dense(8, 10, 8, 3, 4, 4, 0, 1, 8, None, None) == hk.ERR_UNSUPPORTED     # mixed signs
+    assert lib.hikonv_conv1d_dense(8, 10, 8, 3, 4, 2, 0, 1, 8, None, None) == hk.ERR_UNSUPPORTED     # unequal widths: a layout that is not built
+    # the dense 2-D entry point: storage widths that match no code width, outputs that need requantisation
+    assert lib.hikonv_conv2d_dense(8, 3, 1, 1, 4, 4, 8, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 32, 0, 0, 0, 0, 0, 256, 1 << 20, 0, None, None) == hk.ERR_UNSUPPORTED
+    assert lib.hikonv_conv2d_dense(8, 4, 1, 1, 4, 4, 8, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 4, 0, 0, 0, 0, 0, 256, 1 << 20, 0, None, None) == hk.ERR_INVALID_ARG
+    assert lib.hikonv_conv2d_dense(8, 4, 1, 1, 4, 4, 8, 8, 1, 3, 1, 1, 4, 4, 0, 0, 8, 32, 0, 0, 0, 0, 1, 256, 1 << 20, 0, None, None) == hk.ERR_INVALID_ARG   # pool without requant
     assert lib.hikonv_conv1d_dense(8, 10, 8, 9, 4, 4, 0, 0, 8, None, None) == hk.ERR_UNSUPPORTED     # K = 9
     assert lib.hikonv_pack(None, 10, 4, 0, 10, 3, 32, None, None) == hk.ERR_INVALID_ARG
     assert lib.hikonv_check_range(None, 10, 4, 0, 8, None, None) == hk.ERR_INVALID_ARG

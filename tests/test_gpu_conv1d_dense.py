@@ -64,10 +64,24 @@ def test_same_results_as_byte_storage_at_full_size():
     assert np.array_equal(a.cpu().numpy()[idx], want)
 
 
+@pytest.mark.parametrize("bits", [1, 2, 4])
+def test_mixed_signedness(bits):
+    # unsigned codes against signed taps and the reverse, random and extreme, several tiles and a ragged tail
+    for fs, gs in ((False, True), (True, False)):
+        for K in (3, 5, 7):
+            for n in (5, 4099, 200003):
+                f, g = inputs.conv1d_case(n, K, bits, bits, fs, gs, seed=40 + bits * 10 + K)
+                y = hk.conv1d_dense(torch.from_numpy(inputs.to_dense(f, bits)).cuda(), f.size, dev(g), bits, bits, fs, gs)
+                assert_exact(y, direct.conv1d_full(f, g), "mixed bits=%d K=%d fs=%d n=%d" % (bits, K, fs, n))
+            for f, g in inputs.extreme_1d(30001, K, bits, bits, fs, gs):
+                y = hk.conv1d_dense(torch.from_numpy(inputs.to_dense(f, bits)).cuda(), f.size, dev(g), bits, bits, fs, gs)
+                assert_exact(y, direct.conv1d_full(f, g), "mixed extreme bits=%d K=%d fs=%d" % (bits, K, fs))
+
+
 def test_unsupported_combinations_are_refused():
-    f, g = inputs.conv1d_case(1000, 3, 4, 4, False, True, seed=1)
+    f, g = inputs.conv1d_case(1000, 3, 4, 2, False, True, seed=1)
     with pytest.raises(hk.HikonvError):
-        hk.conv1d_dense(torch.from_numpy(inputs.to_dense(f, 4)).cuda(), f.size, dev(g), 4, 4, False, True)   # mixed signs
+        hk.conv1d_dense(torch.from_numpy(inputs.to_dense(f, 4)).cuda(), f.size, dev(g), 4, 2, False, True)   # unequal widths: another layout
     f, g = inputs.conv1d_case(1000, 3, 3, 3, False, False, seed=2)
     with pytest.raises(hk.HikonvError):
         hk.conv1d_dense(torch.zeros(1000, dtype=torch.uint8, device="cuda"), f.size, dev(g), 3, 3, False, False)   # 3 bits straddle bytes

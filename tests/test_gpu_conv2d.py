@@ -164,6 +164,16 @@ def test_compact_cnn_small_batch(algo):
     assert_exact(head, ref_head, "head")
 
 
+def test_compact_cnn_with_pools_fused_into_the_layers():
+    x, layers, head_w = inputs.c5_network(batch=3, H=32, W=64)
+    ref_head, ref_acts = direct.cnn_forward(x, layers, head_w)
+    net = network.CompactCnn(layers, head_w, device="cuda")
+    head, acts = net.forward(dev(x), keep_activations=True, fused_pool=True)
+    for i, (a, r) in enumerate(zip(acts, ref_acts)):
+        assert_exact(a, r, "layer %d" % (i + 1))
+    assert_exact(head, ref_head, "head")
+
+
 def test_compact_cnn_full_size_every_image():
     # the benchmark configuration (batch 64, 3x160x320): head output and every layer's activations of all 64
     # images against the oracle (the oracle runs the batch in four parts to bound its int64 buffers)
