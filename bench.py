@@ -40,12 +40,15 @@ TABLE_REPEATS = 7                    # timed repeats per cell of the per-case ta
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the last ncu capture of the kernel: six
 # consecutive launches of the p=q=4, K=3 signed case at 2^24 rotating over three input and three output
-# buffers, caches not flushed between launches (steady state): 14.2-14.7 MB read, 63.8-65.7 MB written.
-# (With the caches flushed before each launch the same kernel shows 16.8 MB read and 8-9 MB written: most
-# of a launch's output is then still in the 126 MB L2 when its counters stop.)  The SHA-256 is that of the
-# kernel source at capture time; a changed source voids the figure.
+# buffers, caches not flushed between launches (steady state): 12.5-13.4 MB read, 62.9-66.1 MB written
+# (the 8-bit K=7 case: 79.9 MB in all).  (With the caches flushed before each launch the same kernel shows
+# 16.8 MB read and 8-9 MB written: most of a launch's output is then still in the 126 MB L2 when its
+# counters stop.)  The SHA-256 values are those of the kernel sources at capture time; a changed source voids
+# the figure.
 NCU_TRAFFIC = {
-    "conv1d_bs": {"sha256": "", "sha256_run": "", "bytes_per_output": 0.0},
+    "conv1d_bs": {"sha256": "36e8f9ed30e2667834955a0cfb06cb0462a71beae17cbcfc024e007a0ee74fd9",
+                  "sha256_run": "322f9167bd95031f2841bdd2e540d4bd24431054ad2d45e0ce1474457f5564c2",
+                  "bytes_per_output": (13.08e6 + 65.07e6) / 16777218.0},
 }
 
 
@@ -270,7 +273,7 @@ def run_ours(args):
     if rank == 0:
         peaks = {}
         for kind in ("mad_wide_u32", "mad_wide_s32", "mad_lo_s32", "logic", "shift", "prmt"):
-            r = hk.pipe_rate(kind, device=dev)
+            r = hk.pipe_rate(kind, iters=512, device=dev)
             peaks[kind] = {"T_per_s": r["ops_per_second"] / 1e12, "lanes_per_clk_per_sm_at_max_clock": r["lanes_per_clock_per_sm"]}
         peaks["derived"] = {"mad_wide_T_per_s": imad_peak["packed"] / 1e12, "mad_lo_T_per_s": imad_peak["unpacked"] / 1e12,
                             "how": "SMs x lanes/clk x max SM clock (%d SMs, %d / %d lanes, %.0f MHz)"
