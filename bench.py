@@ -273,7 +273,7 @@ def run_ours(args):
     if rank == 0:
         peaks = {}
         for kind in ("mad_wide_u32", "mad_wide_s32", "mad_lo_s32", "logic", "shift", "prmt"):
-            r = hk.pipe_rate(kind, iters=512, device=dev)
+            r = hk.pipe_rate(kind, iters=2048, device=dev)
             peaks[kind] = {"T_per_s": r["ops_per_second"] / 1e12, "lanes_per_clk_per_sm_at_max_clock": r["lanes_per_clock_per_sm"]}
         peaks["derived"] = {"mad_wide_T_per_s": imad_peak["packed"] / 1e12, "mad_lo_T_per_s": imad_peak["unpacked"] / 1e12,
                             "how": "SMs x lanes/clk x max SM clock (%d SMs, %d / %d lanes, %.0f MHz)"
@@ -499,14 +499,16 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         x, layers, head_w = inputs.c5_network(seed=ranks.rank_seed(5, rank), batch=args.batch or 64)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         net = network.CompactCnn(layers, head_w, device=dev)
-        macs, muls = 0.0, None
+        macs, muls = 0.0, 0.0
         H, W = x.shape[2], x.shape[3]
         for L in layers:
             Co, Ci, K, _ = L["w"].shape
             macs += float(x.shape[0]) * Co * H * W * Ci * K * K
+            muls += hk.conv2d_multiplies(x.shape[0], Ci, H, W, Co, K, L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], algo)
             if L["pool"]:
                 H, W = H // 2, W // 2
         macs += float(x.shape[0]) * head_w.shape[0] * H * W * head_w.shape[1]
+        muls += hk.conv2d_multiplies(x.shape[0], head_w.shape[1], H, W, head_w.shape[0], 1, 0, 4, 4, False, True, algo)
 
         def step():
             net.forward(d_x, algo=algo)
@@ -544,7 +546,7 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
     }
     if muls is not None:
         line["roofline"] = alu_roofline(muls, ms, imad_peak, args.algo)
-        line["roofline"]["kernel"] = "conv2d_kernel"
+        line["roofline"]["kernel"] = "conv2d_kernel" + (" (nine layer launches, multiplies summed)" if args.workload == "c5" else "")
     if rank == 0:
         print(json.dumps(line), flush=True)
     ranks.shutdown()
@@ -683,6 +685,18 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
             rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key)}
         rec["layout"] = hk.layout(shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], shape["K"], 2, shape["Ci"] * shape["K"])
         rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
+        if rq and shape["p"] == 4 and shape["q"] == 4:
+            # the same layer with all three tensors stored densely (two 4-bit codes per byte): half the bytes per tensor
+            dx = torch.from_numpy(inputs.to_dense(x, 4)).to(dev)
+            dw = torch.from_numpy(inputs.to_dense(w, 4)).to(dev)
+            do = torch.empty(o.numel() // 2, dtype=torch.uint8, device=dev)
+            ms = time_fn(lambda: hk.conv2d_dense(dx, x.shape, 4, dw, w.shape, 4, shape["pad"], 4, 4, shape["x_signed"], shape["w_signed"],
+                                                 requant=rq, out_store_bits=4, workspace=ws, out=do))
+            n_out = float(o.numel())
+            rec["dense"] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT,
+                            "hbm_bytes_per_output": (dx.numel() + dw.numel() + do.numel()) / n_out,
+                            "byte_storage_hbm_bytes_per_output": (d_x.numel() + d_w.numel() + o.numel()) / n_out}
+            del dx, dw, do
         out[name] = rec
         del d_x, d_w, o
 
@@ -700,7 +714,15 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
     rec = {"macs": macs}
     for key, algo in (("packed", hk.ALGO_PACKED32), ("unpacked", hk.ALGO_UNPACKED_IMAD)):
         ms = time_fn(lambda: net.forward(d_x, algo=algo), iters=5)
-        rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT}
+        # multiplies the nine layer launches execute (positions incl. halo x Co x Ci x K x J, summed)
+        muls, Hl, Wl = 0.0, x.shape[2], x.shape[3]
+        for L in layers:
+            Co, Ci, K, _ = L["w"].shape
+            muls += hk.conv2d_multiplies(x.shape[0], Ci, Hl, Wl, Co, K, L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], algo)
+            if L["pool"]:
+                Hl, Wl = Hl // 2, Wl // 2
+        muls += hk.conv2d_multiplies(x.shape[0], head_w.shape[1], Hl, Wl, head_w.shape[0], 1, 0, 4, 4, False, True, algo)
+        rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key)}
     rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
     out["c5"] = rec
     return out
