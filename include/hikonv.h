@@ -92,8 +92,9 @@ typedef struct {
     int S;          /* force slot width                                             */
     int M;          /* force the number of accumulated products between two splits  */
     int tile;       /* kernel-specific tile selector (0 = automatic); conv2d: > 0 output
-                       rows per CTA, < 0 carry-save moves at stage ends instead of at
-                       fixed places inside channel groups; conv1d: > 0 the general kernel, -1 the
+                       rows per CTA + 1000 x channel lanes per CTA (1, 2, 4, 8, 16) + 100000 x
+                       positions per thread (2 or 4), each part 0 = automatic; < 0 carry-save moves
+                       at stage ends instead of at fixed places inside channel groups; conv1d: > 0 the general kernel, -1 the
                        planner's layout instead of register-aligned slots; -24 / -25 force the
                        register budget of four / five resident CTAs per SM in the register-aligned
                        kernels and the two comparators (default: whichever measured faster for the

@@ -743,6 +743,7 @@ struct Conv2dSetup {
     dim3 grid;
     int threads;
     bool unpacked;
+    int tm;               // positions per thread of the packed kernel
 };
 
 static int sm_count() {
@@ -897,12 +898,24 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         L.N = 1; L.S = 0; L.Kc = 1; L.J = K; L.segments = 1; L.top_bits = 32; L.M = Ci * K; L.signed_prod = (xs || ws) ? 1 : 0;
         L.S_paper = 0;
         TM = kTMU; TN = kTNU; N = 1;
+        s->tm = TM;
         if (K > kMaxJ) return HIKONV_ERR_UNSUPPORTED;
     } else {
         int rc = make_layout(p, q, xs, ws, K, 2, Ci * K, Wo, tune, &L);
         if (rc != HIKONV_OK) return rc;
         if (L.N > kMaxN2D || L.segments > kMaxN2DSeg) return HIKONV_ERR_UNSUPPORTED;
         TM = kTM; TN = kTN; N = L.N;
+        // Small layers are bound by the serial work of a thread, not by the multiplier: when four positions per thread
+        // would not even fill the resident thread slots of the device once (about 1.1 times, measured on the benchmark
+        // network: 10x20 maps 56 -> 32 us, 20x40 maps 83 -> 68 us; larger layers lose 2-10 %), threads take two
+        // positions and there are twice as many of them.  Built for the 3x3 kernel on N = 3, S = 13.
+        if (L.N == 3 && L.S == 13 && K == 3 && L.J == 1) {
+            const double threads4 = (double)B * Ho * (ceil_div(Wo, N) + L.J) / kTM * ceil_div(Co, kTN);
+            if (threads4 <= 1.1 * sm_count() * 2 * kMaxThreads2D) TM = 2;
+        }
+        if (tune && tune->tile >= 100000) TM = tune->tile / 100000;          // forced: 100000 x positions per thread
+        if (TM != kTM && !(TM == 2 && L.N == 3 && L.S == 13 && K == 3 && L.J == 1)) return HIKONV_ERR_UNSUPPORTED;
+        s->tm = TM;
         const SplitConsts sc = make_split_consts(L, p, q, xs, ws, K, L.M);
         kp.bias = sc.bias; kp.mask_low = sc.mask_low; kp.mask_high = sc.mask_high;
         kp.hbits = L.carry_bits; kp.nslots = L.segments;
@@ -926,7 +939,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         while (xo_mult % need != 0) xo_mult += 4;
     }
     // tune->tile > 0: rows per CTA, plus 1000 x channel lanes per CTA (1, 2, 4, 8, 16) when those are forced too
-    const int tile_arg = (tune && tune->tile > 0) ? tune->tile : 0;
+    const int tile_arg = (tune && tune->tile > 0) ? tune->tile % 100000 : 0;
     const TileChoice tc = choose_tiles(kp.total_rows, Ho, kp.X, N, K, L.J, Co, TM, TN, sm_count(), tile_arg % 1000,
                                        requant && pool, xo_mult, tile_arg / 1000);
     if (tc.cost < 0) return HIKONV_ERR_UNSUPPORTED;
@@ -1032,15 +1045,12 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
         return launch_variant<1, 0, kTMU, kTNU, true, 0, 0>(s, sp, st);
     }
     // the layouts of 3x3 and 1x1 layers with the slot width and loop bounds as compile-time constants
+    if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1 && s.tm == 2) return launch_variant<3, 13, 2, kTN, false, 3, 1, true>(s, sp, st);
     if (s.L.N == 3 && s.L.S == 13 && K == 3 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 3, 1, true>(s, sp, st);
     if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, st);
     // 8-bit activations x 4-bit weights with few input channels (a network's first layer): no moves at all
     if (s.L.N == 2 && s.L.S == 17 && K == 3 && J == 2 && s.L.M >= s.kp.Ci * K && s.kp.move_every == 0)
         return launch_variant<2, 17, kTM, kTN, false, 3, 2, false, true>(s, sp, st);
-    // two pixels per word in 16-bit slots, the three taps of a kernel row in one word: 64 bits exactly, and room for
-    // up to 270 accumulated 4-bit products per slot, so layers of up to 90 input channels never move anything
-    if (s.L.N == 2 && s.L.S == 16 && K == 3 && J == 1 && s.L.M >= s.kp.Ci * K && s.kp.move_every == 0)
-        return launch_variant<2, 16, kTM, kTN, false, 3, 1, false, true>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     switch (s.L.N) {
