@@ -640,13 +640,13 @@ __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int 
 // Packed activation rows (Eq. 5): ap[(ci * B*Hp + b*Hp + hp) * XBT + xb] packs the N input pixels of block
 // x = xb - J of padded row hp, i.e. columns (xb - J) N + K - 1 - pad + n of input row hp - pad, zero where the
 // row or a column lies in the padding.  For the comparator S == 0 and N == 1: one int32 code per word.
-// One thread packs four consecutive words of a row (one 16-byte store); a CTA stays within one
-// (ci, b) plane, whose rows are contiguous in both the input and the packed layout.  The CTAs past the
+// One thread packs four consecutive words of a row (one 16-byte store); threads are numbered through all
+// (ci, b) planes, so that small maps still fill their CTAs.  The CTAs past the
 // activation planes pack the kernel rows (one word per thread), so that a layer needs one packing launch.
 // x_bits: storage of the activations, 8 = one code per byte, 1 / 2 / 4 = dense.
 template <bool XS, int N>
 __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
-                                                            int pad, int K, int J, int S, int XBT, int blocks_per_plane,
+                                                            int pad, int K, int J, int S, int XBT,
                                                             uint32_t *__restrict__ ap, int act_blocks, const WeightPackParams wq,
                                                             int x_bits) {
     grid_dependency_release();
@@ -655,10 +655,13 @@ __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__rest
         pack_weight_word(wq, ((int)blockIdx.x - act_blocks) * 256 + (int)threadIdx.x);
         return;
     }
-    const int plane = blockIdx.x / blocks_per_plane;                 // ci * B + b
-    const int piece = (blockIdx.x - plane * blocks_per_plane) * 256 + threadIdx.x;
+    // the (plane, piece) pairs are numbered through: a CTA may span several small planes (ci * B + b)
     const int xq = XBT / 4;                                          // 16-byte pieces per packed row
-    if (piece >= Hp * xq) return;
+    const int per_plane = Hp * xq;
+    const long long item = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (item >= (long long)Ci * B * per_plane) return;
+    const int plane = (int)(item / per_plane);
+    const int piece = (int)(item - (long long)plane * per_plane);
     const int ci = plane / B, b = plane - ci * B;
     const int hp = piece / xq, q = piece - hp * xq;
     const int hi = hp - pad;
@@ -1107,13 +1110,13 @@ static int conv2d_run(const void *d_x, int x_bits, int B, int Ci, int H, int W, 
         WeightPackParams wq;
         wq.w = (const int8_t *)d_w; wq.wp = d_wp; wq.Co = Co; wq.Ci = Ci; wq.K = K; wq.J = s.L.J; wq.Kc = s.L.Kc; wq.S = s.L.S;
         wq.w_signed = w_signed ? 1 : 0; wq.CoP = s.kp.CoP; wq.total = Ci * K * s.L.J * s.kp.CoP; wq.w_bits = w_bits;
-        const int bpp = ceil_div(s.kp.Hp * (s.kp.XBT / 4), 256);
-        const size_t act_blocks = (size_t)Ci * B * bpp, w_blocks = (size_t)ceil_div(wq.total, 256);
+        const size_t act_items = (size_t)Ci * B * s.kp.Hp * (s.kp.XBT / 4);
+        const size_t act_blocks = (act_items + 255) / 256, w_blocks = (size_t)ceil_div(wq.total, 256);
         if (act_blocks + w_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
         const unsigned grid = (unsigned)(act_blocks + w_blocks);
 #define HK_PACK(XSIGN, NN)                                                                                                 \
     rc = launch_dependent(pack_operands_kernel<XSIGN, NN>, dim3(grid), dim3(256), 0, st, (const int8_t *)d_x, B, Ci, H, W, s.kp.Hp, \
-                          pad, K, s.L.J, s.L.S, s.kp.XBT, bpp, d_ap, (int)act_blocks, wq, x_bits)
+                          pad, K, s.L.J, s.L.S, s.kp.XBT, d_ap, (int)act_blocks, wq, x_bits)
         switch (s.L.N * 2 + (x_signed ? 1 : 0)) {
             case 2: HK_PACK(false, 1); break;
             case 3: HK_PACK(true, 1); break;
