@@ -77,6 +77,8 @@ struct Conv2dParams {
     int pool;                  // 2x2 max-pool fused into the copy-out
     int out_signed;            // pooled codes compare as signed bytes
     int out_bits;              // 8: one code per byte; 1 / 2 / 4: dense output, 8 / out_bits codes per byte (vec: 4 or 1 bytes)
+    // multipliers of fast_div() for the divisors fixed per launch: XB, Ho, 16-byte pieces per activation row, CK, NSEG
+    uint32_t mg_xb, mg_ho, mg_xq, mg_ck, mg_nseg;
 };
 
 template <bool UNPACKED>
@@ -96,6 +98,12 @@ __device__ __forceinline__ int small_div(int n, int d, float inv_d) {
     if (r < 0) --q;
     else if (r >= d) ++q;
     return q;
+}
+
+// n / d for 0 <= n < 2^16 and 0 < d < 2^16 with magic = ceil(2^32 / d) mod 2^32 (0 stands for d == 1): the high
+// word of n * magic is the exact quotient because n (d - 1) < 2^32.
+__device__ __forceinline__ int fast_div(int n, uint32_t magic) {
+    return magic ? (int)__umulhi((uint32_t)n, magic) : n;
 }
 
 // One multiply-accumulate of the k loop: the packed 32x32->64 product of Eq. 9 added to the 64-bit
@@ -144,15 +152,15 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     const int tid = threadIdx.x, nthreads = blockDim.x;
     const int tnx_log2 = 31 - __clz(p.TNX);                 // TNX is a power of two
     const int tn = tid & (p.TNX - 1);
-    const float inv_xb = 1.0f / (float)p.XB, inv_ho = 1.0f / (float)p.Ho;
-    const int seg = blockIdx.x % p.NSEG;
-    const int R0 = (blockIdx.x / p.NSEG) * p.TR;
+    const int row_tile = p.NSEG > 1 ? (int)(blockIdx.x / (unsigned)p.NSEG) : (int)blockIdx.x;
+    const int seg = blockIdx.x - row_tile * p.NSEG;
+    const int R0 = row_tile * p.TR;
     const int co0 = blockIdx.y * p.TCO;
     const int TRe = min(p.TR, p.total_rows - R0);
     const int b0 = R0 / p.Ho, h0 = R0 - b0 * p.Ho;
     const int Rp0 = b0 * p.Hp + h0;                         // first staged padded row
     const int Rlast = R0 + TRe - 1;
-    const int bl = Rlast / p.Ho;
+    const int bl = b0 + fast_div(h0 + TRe - 1, p.mg_ho);
     const int NR = (bl * p.Hp + (Rlast - bl * p.Ho) + p.K - 1) - Rp0 + 1;
     const int TP = TRe * p.XB;                              // positions of this tile
     const int S = SC > 0 ? SC : p.S;
@@ -170,8 +178,8 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         const int pos = wpos0 + i * lanes_m + lm;
         int off = p.lead;                                    // idle position: reads valid memory, result dropped
         if (pos < TP) {
-            const int r = small_div(pos, p.XB, inv_xb), xb = pos - r * p.XB;
-            const int db = small_div(h0 + r, p.Ho, inv_ho);          // images past the tile's first one
+            const int r = fast_div(pos, p.mg_xb), xb = pos - r * p.XB;
+            const int db = fast_div(h0 + r, p.mg_ho);                // images past the tile's first one
             off = p.lead + (db * p.Hp + (h0 + r - db * p.Ho) - h0) * p.XBS + xb;
         }
         aptr[i] = As + off;
@@ -233,20 +241,16 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     // offsets are worked out once (channel in the top byte of the destination offset, -1: none).
     constexpr int kPieces = kCopyPieces;
     int piece_src[kPieces], piece_dst[kPieces];
-    {
-        const int per_ch = NR * xq;
-        const float inv_per_ch = 1.0f / (float)per_ch, inv_xq = 1.0f / (float)xq;
 #pragma unroll
-        for (int k = 0; k < kPieces; ++k) {
-            const int q = tid + k * nthreads;
-            piece_src[k] = 0;
-            piece_dst[k] = -1;
-            if (q < p.CK * per_ch) {
-                const int cl = small_div(q, per_ch, inv_per_ch), r = q - cl * per_ch;
-                const int rl = small_div(r, xq, inv_xq), qd = r - rl * xq;
-                piece_src[k] = cl * ap_plane + rl * p.XBT + 4 * qd;
-                piece_dst[k] = (cl << 24) | (cl * p.a_plane + p.lead + rl * p.XBS + 4 * qd);
-            }
+    for (int k = 0; k < kPieces; ++k) {
+        const int q = tid + k * nthreads;                            // pieces numbered [row][channel][piece of the row]
+        piece_src[k] = 0;
+        piece_dst[k] = -1;
+        if (q < p.CK * NR * xq) {
+            const int rc = fast_div(q, p.mg_xq), qd = q - rc * xq;
+            const int rl = fast_div(rc, p.mg_ck), cl = rc - rl * p.CK;
+            piece_src[k] = cl * ap_plane + rl * p.XBT + 4 * qd;
+            piece_dst[k] = (cl << 24) | (cl * p.a_plane + p.lead + rl * p.XBS + 4 * qd);
         }
     }
     const bool pieces_in_regs = p.CK * NR * xq <= kPieces * nthreads;
@@ -262,12 +266,11 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 if (piece_dst[k] >= 0 && (piece_dst[k] >> 24) < ckn) cp_async_16(Adst + (piece_dst[k] & 0xFFFFFF), asrc + piece_src[k]);
         } else {
             const int per_ch = NR * xq;
-            const float inv_xq = 1.0f / (float)xq;
             for (int cl = 0; cl < ckn; ++cl) {
                 const uint32_t *src = asrc + (size_t)cl * ap_plane;
                 uint32_t *dst = Adst + cl * p.a_plane + p.lead;
                 for (int idx = tid; idx < per_ch; idx += nthreads) {
-                    const int rl = small_div(idx, xq, inv_xq), qd = idx - rl * xq;
+                    const int rl = fast_div(idx, p.mg_xq), qd = idx - rl * xq;
                     cp_async_16(dst + rl * p.XBS + 4 * qd, src + (size_t)rl * p.XBT + 4 * qd);
                 }
             }
@@ -389,16 +392,23 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     }
 
     // ---- extract the slots: slot m holds 2^h E_m + Q_m - (moves + 1) bias_m (uint32 arithmetic wraps by design)
+    // slots per accumulator, N + Kc - 1: a constant of the unrolled kernels (Kc = K when the kernel row is one word, else N)
+    constexpr int NS_CT = (!UNPACKED && KT > 0) ? N + (JT == 1 ? KT : N) - 1 : 0;
+    const int nslots = NS_CT > 0 ? NS_CT : p.nslots;
     uint32_t slot_sub[2 * N], slot_msk[2 * N];                        // per slot: (moves + 1) bias_m and the field mask
 #pragma unroll
     for (int m = 0; m < 2 * N; ++m) {
         slot_sub[m] = ((uint32_t)nmoves + 1u) * (uint32_t)p.slot_bias[m];
-        slot_msk[m] = (m == p.nslots - 1) ? p.top_mask : p.slot_mask;
+        slot_msk[m] = (m == nslots - 1) ? p.top_mask : p.slot_mask;
     }
     auto slot_value = [&](uint64_t Q, uint64_t Ev, int m) -> uint32_t {
-        const uint32_t qv = (uint32_t)(Q >> (S * m)) & slot_msk[m];
+        // a top slot that ends at bit 63 or beyond needs no mask: the shift leaves nothing above it
+        const bool open_top = SC > 0 && NS_CT > 0 && m == NS_CT - 1 && SC * NS_CT >= 64;
+        uint32_t qv = (uint32_t)(Q >> (S * m));
+        if (!open_top) qv &= slot_msk[m];
         if constexpr (NOE) return qv - slot_sub[m];
-        const uint32_t ev = (uint32_t)(Ev >> (S * m)) & slot_msk[m];
+        uint32_t ev = (uint32_t)(Ev >> (S * m));
+        if (!open_top) ev &= slot_msk[m];
         return (ev << p.hbits) + qv - slot_sub[m];
     };
     auto load_e = [&](int i, int t) -> uint64_t {
@@ -418,45 +428,50 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
                 for (int t = 0; t < TN; ++t)
                     xch[(warp * N + m) * p.TCO + tn * TN + t] =
-                        (N + m < p.nslots) ? slot_value((uint64_t)acc[TM - 1][t], load_e(TM - 1, t), N + m) : 0u;
+                        (N + m < nslots) ? slot_value((uint64_t)acc[TM - 1][t], load_e(TM - 1, t), N + m) : 0u;
         }
         __syncthreads();
     }
 
-    // where each position's pixels go (channel 0): element offset and number of pixels to store (0: none)
-    size_t pix_off[TM];
+    // where each position's pixels go: element offset relative to the CTA's first output (image b0, channel co0),
+    // which fits 32 bits (checked on the host), and number of pixels to store (0: none)
+    uint32_t pix_rel[TM];
     int pix_n[TM];
     int tile_pos[TM];                                                // staged output: byte offset of the position's first pixel in a channel's tile
+    const uint32_t chan_stride = (uint32_t)(p.Ho * p.Wo);
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
         const int pos = wpos0 + i * lanes_m + lm;
-        pix_off[i] = 0;
+        pix_rel[i] = 0;
         pix_n[i] = 0;
         tile_pos[i] = 0;
         if (pos < TP) {
-            const int r = small_div(pos, p.XB, inv_xb), xbl = pos - r * p.XB;
+            const int r = fast_div(pos, p.mg_xb), xbl = pos - r * p.XB;
             const int xg = seg * p.XO + xbl - p.J;                   // output block in the row; halo positions give no pixels
             if (xbl >= p.J && xg < p.X) {
-                const int db = small_div(h0 + r, p.Ho, inv_ho);
-                const int b = b0 + db, h = h0 + r - db * p.Ho;
-                pix_off[i] = (((size_t)b * p.Co) * p.Ho + h) * p.Wo + (size_t)xg * N;
+                const int db = fast_div(h0 + r, p.mg_ho);
+                const int h = h0 + r - db * p.Ho;
+                pix_rel[i] = (uint32_t)(db * p.Co) * chan_stride + (uint32_t)(h * p.Wo + xg * N);
                 pix_n[i] = min(N, p.Wo - xg * N);
                 tile_pos[i] = r * p.WTP + (xbl - p.J) * N;
             }
         }
     }
-    const size_t chan_stride = (size_t)p.Ho * p.Wo;
+    const size_t cta_off = ((size_t)b0 * p.Co + co0) * chan_stride;
 
     if (UNPACKED && p.requant && p.stage_out) __syncthreads();     // the staged tile reuses the operand buffers of the main loop
     int8_t *tile = reinterpret_cast<int8_t *>(smem + p.tile_off);
     const int tile_chan = p.TR * p.WTP;                              // bytes per channel of the staged tile
     // ---- overlap-add, optional requantisation (arithmetic shift, clamp), store
-    auto finish = [&](auto requant_tag) {
-        constexpr bool REQ = decltype(requant_tag)::value;
+    auto finish = [&](auto requant_tag, auto staged_tag) {
+        constexpr bool REQ = decltype(requant_tag)::value, STAGED = decltype(staged_tag)::value;
+        int8_t *out8 = (int8_t *)p.out + cta_off;
+        int32_t *out32 = (int32_t *)p.out + cta_off;
 #pragma unroll
         for (int t = 0; t < TN; ++t) {
-            const int co = co0 + tn * TN + t;
-            const size_t chan_off = (size_t)co * chan_stride;
+            const int cl = tn * TN + t;
+            const uint32_t chan_rel = (uint32_t)cl * chan_stride;
+            const bool chan_ok = co0 + cl < p.Co;
             uint32_t up_prev[N];                                     // upper slots of this lane's previous position
 #pragma unroll
             for (int m = 0; m < N; ++m) up_prev[m] = 0u;
@@ -469,10 +484,10 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                     for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], ev, m);
 #pragma unroll
                     for (int m = 0; m < N; ++m) {
-                        if (N + m < p.nslots) {                      // uniform over the launch
+                        if (N + m < nslots) {                        // uniform over the launch
                             const uint32_t up = slot_value((uint64_t)acc[i][t], ev, N + m);
                             uint32_t in = __shfl_sync(0xFFFFFFFFu, lm == lanes_m - 1 ? up_prev[m] : up, (lane - p.TNX) & 31);
-                            if (i == 0 && lm == 0) in = warp > 0 ? smem[((warp - 1) * N + m) * p.TCO + tn * TN + t] : 0u;
+                            if (i == 0 && lm == 0) in = warp > 0 ? smem[((warp - 1) * N + m) * p.TCO + cl] : 0u;
                             Y[m] += in;
                             up_prev[m] = up;
                         }
@@ -480,26 +495,27 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 } else {
                     Y[0] = (uint32_t)acc[i][t];
                 }
-                const size_t o = pix_off[i] + chan_off;
-                const int n_store = co < p.Co ? pix_n[i] : 0;
+                const uint32_t o = pix_rel[i] + chan_rel;
+                const int n_store = chan_ok ? pix_n[i] : 0;
 #pragma unroll
                 for (int m = 0; m < N; ++m) {
                     int32_t v = (int32_t)Y[m];
                     if constexpr (REQ) {
                         v = max(p.lo, min(p.hi, v >> p.shift));
                         if (m < n_store) {
-                            if (p.stage_out) tile[(tn * TN + t) * tile_chan + tile_pos[i] + m] = (int8_t)v;
-                            else ((int8_t *)p.out)[o + m] = (int8_t)v;
+                            if constexpr (STAGED) tile[cl * tile_chan + tile_pos[i] + m] = (int8_t)v;
+                            else out8[o + m] = (int8_t)v;
                         }
                     } else {
-                        if (m < n_store) ((int32_t *)p.out)[o + m] = v;
+                        if (m < n_store) out32[o + m] = v;
                     }
                 }
             }
         }
     };
-    if (p.requant) finish(std::true_type());
-    else finish(std::false_type());
+    if (!p.requant) finish(std::false_type(), std::false_type());
+    else if (p.stage_out) finish(std::true_type(), std::true_type());
+    else finish(std::true_type(), std::false_type());
     if (!(p.requant && p.stage_out)) return;
 
     // ---- staged codes leave the CTA: whole rows in pieces of `vec` bytes, optionally max-pooled 2x2 on the way
@@ -519,7 +535,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             const int rr = small_div(idx, ppr, inv_ppr), piece = idx - rr * ppr;
             const int cl = small_div(rr, TRq, inv_tr), rq = rr - cl * TRq;
             const int r = rq << sh;
-            const int db = small_div(h0 + r, p.Ho, inv_ho);
+            const int db = fast_div(h0 + r, p.mg_ho);
             const int b = b0 + db, h = h0 + r - db * p.Ho;
             const int8_t *src = tile + cl * tile_chan + r * p.WTP;
             const size_t e0 = ((((size_t)b * p.Co + co0 + cl) * Hq + (h >> sh)) * Wq + (col0 >> sh));   // first code of this segment's row
@@ -550,7 +566,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         for (int idx = tid; idx < ncv * TRe * ppr; idx += nthreads) {
             const int rr = small_div(idx, ppr, inv_ppr), piece = idx - rr * ppr;
             const int cl = small_div(rr, TRe, inv_tr), r = rr - cl * TRe;
-            const int db = small_div(h0 + r, p.Ho, inv_ho);
+            const int db = fast_div(h0 + r, p.mg_ho);
             const int b = b0 + db, h = h0 + r - db * p.Ho;
             const int8_t *src = tile + cl * tile_chan + r * p.WTP + piece * p.vec;
             int8_t *dst = (int8_t *)p.out + (((size_t)b * p.Co + co0 + cl) * p.Ho + h) * p.Wo + col0 + piece * p.vec;
@@ -567,7 +583,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             const int rr = small_div(idx, ppr, inv_ppr), piece = idx - rr * ppr;
             const int cl = small_div(rr, TRq, inv_tr), rq = rr - cl * TRq;
             const int r = 2 * rq;
-            const int db = small_div(h0 + r, p.Ho, inv_ho);
+            const int db = fast_div(h0 + r, p.mg_ho);
             const int b = b0 + db, h = h0 + r - db * p.Ho;
             const int8_t *src = tile + cl * tile_chan + r * p.WTP + piece * 2 * p.vec;
             int8_t *dst = (int8_t *)p.out + (((size_t)b * p.Co + co0 + cl) * Hq + (h >> 1)) * Wq + (col0 >> 1) + piece * p.vec;
@@ -886,7 +902,7 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     if (requant && (shift < 0 || shift > 31 || lo < -128 || hi > 255 || lo > hi)) return HIKONV_ERR_INVALID_ARG;
     const int Ho = H + 2 * pad - K + 1, Wo = W + 2 * pad - K + 1;
     if (Ho < 1 || Wo < 1) return HIKONV_ERR_INVALID_ARG;
-    if (Ho >= (1 << 21)) return HIKONV_ERR_UNSUPPORTED;          // the kernel's row arithmetic uses a float reciprocal
+    if (Ho >= 60000) return HIKONV_ERR_UNSUPPORTED;              // the kernel divides row numbers below 2^16 by a multiply (fast_div)
     if ((double)B * Ci * H * W >= 2147483647.0 || (double)B * Ho >= 2147483647.0) return HIKONV_ERR_UNSUPPORTED;
     // the exact sums must fit int32
     const double max_code = (double)(1 << p) * (double)(1 << q);
@@ -950,6 +966,8 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.NSEG = tc.NSEG; kp.XO = tc.XO; kp.XB = tc.XB; kp.TR = tc.TR;
     s->threads = tc.TMX * tc.TNX;
     const int span = (kp.TR + Ho - 2) / Ho + 1;              // images a tile can touch
+    // output offsets relative to a CTA's first image and channel are kept in 32 bits
+    if ((double)(span + 1) * std::max(Co, kp.TCO) * Ho * Wo >= 4294967296.0) return HIKONV_ERR_UNSUPPORTED;
     kp.NRmax = kp.TR + (K - 1) * span;
     // words per activation row in shared memory: 8, 16, 32 or 64 (the unrolled kernels have them as constants)
     kp.XBS = kp.XB <= 8 ? 8 : kp.XB <= 16 ? 16 : kp.XB <= 32 ? 32 : 64;
@@ -986,6 +1004,10 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         }
     }
     kp.CK = CK;
+    {
+        auto magic = [](int d) -> uint32_t { return d <= 1 ? 0u : (uint32_t)((0x100000000ull + (unsigned)d - 1) / (unsigned)d); };
+        kp.mg_xb = magic(kp.XB); kp.mg_ho = magic(Ho); kp.mg_xq = magic((kp.XB + 3) / 4); kp.mg_ck = magic(CK); kp.mg_nseg = magic(kp.NSEG);
+    }
     kp.a_words = CK * kp.a_plane;
     kp.b_off = 2 * kp.a_words;
     kp.b_words = CK * K * L.J * kBPitch;
