@@ -175,14 +175,11 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     const uint32_t *aptr[TM];
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
-        const int pos = wpos0 + i * lanes_m + lm;
-        int off = p.lead;                                    // idle position: reads valid memory, result dropped
-        if (pos < TP) {
-            const int r = fast_div(pos, p.mg_xb), xb = pos - r * p.XB;
-            const int db = fast_div(h0 + r, p.mg_ho);                // images past the tile's first one
-            off = p.lead + (db * p.Hp + (h0 + r - db * p.Ho) - h0) * p.XBS + xb;
-        }
-        aptr[i] = As + off;
+        // an idle position (past the tile) reads the words of position 0; its result is dropped
+        const int pos = wpos0 + i * lanes_m + lm, pc = pos < TP ? pos : 0;
+        const int r = fast_div(pc, p.mg_xb), xb = pc - r * p.XB;
+        const int db = fast_div(h0 + r, p.mg_ho);                    // images past the tile's first one: K - 1 more padded rows each
+        aptr[i] = As + p.lead + (r + db * (p.K - 1)) * p.XBS + xb;
     }
 
     static_assert(UNPACKED || TM * TN <= kEPitch, "second-accumulator pitch too small for the thread tile");
@@ -244,14 +241,10 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
 #pragma unroll
     for (int k = 0; k < kPieces; ++k) {
         const int q = tid + k * nthreads;                            // pieces numbered [row][channel][piece of the row]
-        piece_src[k] = 0;
-        piece_dst[k] = -1;
-        if (q < p.CK * NR * xq) {
-            const int rc = fast_div(q, p.mg_xq), qd = q - rc * xq;
-            const int rl = fast_div(rc, p.mg_ck), cl = rc - rl * p.CK;
-            piece_src[k] = cl * ap_plane + rl * p.XBT + 4 * qd;
-            piece_dst[k] = (cl << 24) | (cl * p.a_plane + p.lead + rl * p.XBS + 4 * qd);
-        }
+        const int rc = fast_div(q, p.mg_xq), qd = q - rc * xq;
+        const int rl = fast_div(rc, p.mg_ck), cl = rc - rl * p.CK;
+        piece_src[k] = cl * ap_plane + rl * p.XBT + 4 * qd;
+        piece_dst[k] = q < p.CK * NR * xq ? ((cl << 24) | (cl * p.a_plane + p.lead + rl * p.XBS + 4 * qd)) : -1;
     }
     const bool pieces_in_regs = p.CK * NR * xq <= kPieces * nthreads;
     const int tco4 = p.TCO / 4, tco4_log2 = 31 - __clz(tco4);        // TCO / 4 is a power of two
@@ -441,21 +434,15 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
     const uint32_t chan_stride = (uint32_t)(p.Ho * p.Wo);
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
-        const int pos = wpos0 + i * lanes_m + lm;
-        pix_rel[i] = 0;
-        pix_n[i] = 0;
-        tile_pos[i] = 0;
-        if (pos < TP) {
-            const int r = fast_div(pos, p.mg_xb), xbl = pos - r * p.XB;
-            const int xg = seg * p.XO + xbl - p.J;                   // output block in the row; halo positions give no pixels
-            if (xbl >= p.J && xg < p.X) {
-                const int db = fast_div(h0 + r, p.mg_ho);
-                const int h = h0 + r - db * p.Ho;
-                pix_rel[i] = (uint32_t)(db * p.Co) * chan_stride + (uint32_t)(h * p.Wo + xg * N);
-                pix_n[i] = min(N, p.Wo - xg * N);
-                tile_pos[i] = r * p.WTP + (xbl - p.J) * N;
-            }
-        }
+        const int pos = wpos0 + i * lanes_m + lm, pc = pos < TP ? pos : 0;
+        const int r = fast_div(pc, p.mg_xb), xbl = pc - r * p.XB;
+        const int xg = seg * p.XO + xbl - p.J;                       // output block in the row; halo positions give no pixels
+        const int db = fast_div(h0 + r, p.mg_ho);
+        const int h = h0 + r - db * p.Ho;
+        const bool valid = pos < TP && xbl >= p.J && xg < p.X;
+        pix_rel[i] = (uint32_t)(db * p.Co) * chan_stride + (uint32_t)(h * p.Wo + xg * N);
+        pix_n[i] = valid ? min(N, p.Wo - xg * N) : 0;
+        tile_pos[i] = r * p.WTP + (xbl - p.J) * N;
     }
     const size_t cta_off = ((size_t)b0 * p.Co + co0) * chan_stride;
 
