@@ -79,6 +79,10 @@ struct Conv2dParams {
     int out_bits;              // 8: one code per byte; 1 / 2 / 4: dense output, 8 / out_bits codes per byte (vec: 4 or 1 bytes)
     // multipliers of fast_div() for the divisors fixed per launch: XB, Ho, 16-byte pieces per activation row, CK, NSEG
     uint32_t mg_xb, mg_ho, mg_xq, mg_ck, mg_nseg;
+    // unsigned activations run as signed ones: every packed code is x - x_off (also outside the image, where x = 0),
+    // and corr[co] = x_off * (sum of all weights of channel co) is added back to every output (0: not used)
+    int x_off;
+    const int32_t *corr;
 };
 
 template <bool UNPACKED>
@@ -459,6 +463,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
             const int cl = tn * TN + t;
             const uint32_t chan_rel = (uint32_t)cl * chan_stride;
             const bool chan_ok = co0 + cl < p.Co;
+            const uint32_t cadd = (p.x_off != 0 && chan_ok) ? (uint32_t)__ldg(p.corr + co0 + cl) : 0u;
             uint32_t up_prev[N];                                     // upper slots of this lane's previous position
 #pragma unroll
             for (int m = 0; m < N; ++m) up_prev[m] = 0u;
@@ -468,7 +473,7 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
                 if constexpr (!UNPACKED) {
                     const uint64_t ev = load_e(i, t);
 #pragma unroll
-                    for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], ev, m);
+                    for (int m = 0; m < N; ++m) Y[m] = slot_value((uint64_t)acc[i][t], ev, m) + cadd;
 #pragma unroll
                     for (int m = 0; m < N; ++m) {
                         if (N + m < nslots) {                        // uniform over the launch
@@ -599,6 +604,9 @@ struct WeightPackParams {
     uint32_t *wp;
     int Co, Ci, K, J, Kc, S, w_signed, CoP, total;
     int w_bits;                // storage: 8 = one code per byte, 1 / 2 / 4 = dense (8 / w_bits codes per byte)
+    int w_blocks;              // CTAs that pack kernel rows; the CTAs after them sum the weights of a channel (x_off != 0)
+    int x_off;                 // offset taken from every activation code (0: none)
+    int32_t *corr;             // corr[co] = x_off * sum of the weights of channel co, CoP entries
 };
 
 // Code number e of a tensor stored densely with `bits` (1, 2, 4 or 8) bits per code: code e occupies bits
@@ -640,6 +648,27 @@ __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int 
     q.wp[idx] = word;
 }
 
+// corr[co] = x_off * sum_{ci, kh, kw} W[co][ci][kh][kw]: one warp per output channel (its Ci K K codes are contiguous).
+__device__ __forceinline__ void sum_channel_weights(const WeightPackParams &q, int co, int lane) {
+    if (co >= q.CoP) return;
+    int32_t sum = 0;
+    if (co < q.Co) {
+        const int per_co = q.Ci * q.K * q.K;
+        const size_t e0 = (size_t)co * per_co;
+        for (int e = lane; e < per_co; e += 32) {
+            if (q.w_bits == 8) {
+                const int8_t raw = __ldg(q.w + e0 + e);
+                sum += q.w_signed ? (int32_t)raw : (int32_t)(uint8_t)raw;
+            } else {
+                sum += load_dense_code(q.w, e0 + e, q.w_bits, q.w_signed != 0);
+            }
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+    }
+    if (lane == 0) q.corr[co] = sum * q.x_off;
+}
+
 // Packed activation rows (Eq. 5): ap[(ci * B*Hp + b*Hp + hp) * XBT + xb] packs the N input pixels of block
 // x = xb - J of padded row hp, i.e. columns (xb - J) N + K - 1 - pad + n of input row hp - pad, zero where the
 // row or a column lies in the padding.  For the comparator S == 0 and N == 1: one int32 code per word.
@@ -647,6 +676,7 @@ __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int 
 // (ci, b) planes, so that small maps still fill their CTAs.  The CTAs past the
 // activation planes pack the kernel rows (one word per thread), so that a layer needs one packing launch.
 // x_bits: storage of the activations, 8 = one code per byte, 1 / 2 / 4 = dense.
+// With wq.x_off != 0 every slot holds code - x_off, the slots outside the image included (code 0 there).
 template <bool XS, int N>
 __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
                                                             int pad, int K, int J, int S, int XBT,
@@ -655,7 +685,9 @@ __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__rest
     grid_dependency_release();
     grid_dependency_wait();                                          // the input may come from the kernel before; the workspace may still be read by it
     if ((int)blockIdx.x >= act_blocks) {
-        pack_weight_word(wq, ((int)blockIdx.x - act_blocks) * 256 + (int)threadIdx.x);
+        const int wb = (int)blockIdx.x - act_blocks;
+        if (wb < wq.w_blocks) pack_weight_word(wq, wb * 256 + (int)threadIdx.x);
+        else sum_channel_weights(wq, (wb - wq.w_blocks) * 8 + ((int)threadIdx.x >> 5), (int)threadIdx.x & 31);
         return;
     }
     // the (plane, piece) pairs are numbered through: a CTA may span several small planes (ci * B + b)
@@ -668,7 +700,12 @@ __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__rest
     const int ci = plane / B, b = plane - ci * B;
     const int hp = piece / xq, q = piece - hp * xq;
     const int hi = hp - pad;
-    uint32_t word[4] = {0u, 0u, 0u, 0u};
+    uint32_t fill = 0u;                                              // a word whose N slots all hold -x_off
+    if (wq.x_off != 0) {
+#pragma unroll
+        for (int n = 0; n < N; ++n) fill += (uint32_t)(-wq.x_off) << (S * n);
+    }
+    uint32_t word[4] = {fill, fill, fill, fill};
     if (hi >= 0 && hi < H) {
         const size_t row_e = (((size_t)b * Ci + ci) * H + hi) * W;  // first code of the input row
         const int col0 = (4 * q - J) * N + K - 1 - pad;              // input column of slot 0 of the first word
@@ -744,7 +781,8 @@ struct Conv2dSetup {
     hikonv_layout_t L;
     Conv2dParams kp;
     size_t smem_bytes;
-    size_t wp_bytes;      // packed weights in the workspace (256-byte multiple), packed activations follow
+    size_t wp_bytes;      // packed weights and the per-channel correction in the workspace (256-byte multiple), packed activations follow
+    size_t corr_off;      // byte offset of the correction (CoP int32) in the workspace
     size_t ap_words;      // packed activation words
     dim3 grid;
     int threads;
@@ -909,6 +947,20 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     } else {
         int rc = make_layout(p, q, xs, ws, K, 2, Ci * K, Wo, tune, &L);
         if (rc != HIKONV_OK) return rc;
+        // Unsigned activations against signed weights: the products of codes x - 2^(p-1) span about half the range,
+        // so a slot takes nearly twice as many of them between two carry-save moves.  Deep layers (measured: 256
+        // input channels 239 -> 222 us; 64 channels on small maps lose 2 us to the extra packing work) whose signed
+        // layout allows at least half again as many products run on the shifted codes and get
+        // 2^(p-1) * (sum of the channel's weights) added back in the epilogue.
+        if (!xs && ws && L.M < Ci * K && Ci >= 128) {
+            hikonv_layout_t Ls;
+            if (make_layout(p, q, 1, ws, K, 2, Ci * K, Wo, tune, &Ls) == HIKONV_OK && Ls.N >= L.N && Ls.J <= L.J &&
+                2 * Ls.M >= 3 * L.M) {
+                L = Ls;
+                xs = 1;
+                kp.x_off = 1 << (p - 1);
+            }
+        }
         if (L.N > kMaxN2D || L.segments > kMaxN2DSeg) return HIKONV_ERR_UNSUPPORTED;
         TM = kTM; TN = kTN; N = L.N;
         // Small layers are bound by the serial work of a thread, not by the multiplier: when four positions per thread
@@ -1036,7 +1088,8 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
     kp.e_off = (int)((std::max(std::max(words, xch_words), stage_words) + 3) / 4 * 4);
     const size_t e_words = s->unpacked ? 0 : (size_t)kEPitch * s->threads * 2;
     s->smem_bytes = ((size_t)kp.e_off + e_words) * 4 + 16;
-    s->wp_bytes = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
+    s->corr_off = align_up((size_t)Ci * K * L.J * kp.CoP * sizeof(uint32_t), 256);
+    s->wp_bytes = s->corr_off + align_up((size_t)kp.CoP * sizeof(int32_t), 256);
     s->ap_words = (size_t)Ci * B * kp.Hp * kp.XBT;
     if (s->ap_words >= 0x7FFFFFFFull || (size_t)Ci * K * L.J * kp.CoP >= 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
     if (s->smem_bytes > 200 * 1024) return HIKONV_ERR_UNSUPPORTED;
@@ -1083,7 +1136,9 @@ extern "C" size_t hikonv_conv2d_workspace_bytes(int B, int Ci, int H, int W, int
     const long long Ho = (long long)H + 2 * pad - K + 1, Wo = (long long)W + 2 * pad - K + 1;
     if (Ho < 1 || Wo < 1) return 0;
     // packed kernel rows: at most K words per (ci, kh) row (one tap per word in the comparator), Co rounded up to 4
-    const size_t weights = align_up((size_t)Ci * K * K * ((Co + 3) / 4 * 4) * sizeof(uint32_t), 256);
+    // (plus one int32 per channel: the correction of layers that run unsigned activations as signed ones)
+    const size_t weights = align_up((size_t)Ci * K * K * ((Co + 3) / 4 * 4) * sizeof(uint32_t), 256) +
+                           align_up((size_t)((Co + 3) / 4 * 4) * sizeof(int32_t), 256);
     // packed activation rows: at most one word per output pixel plus K halo words per row (the comparator's
     // layout), rounded up to 16-byte pieces, with one more piece per row segment (segments hold >= 32 blocks)
     const size_t row_words = (size_t)(Wo + K + 3) / 4 * 4 + 16 + (size_t)(Wo + K) / 8;
@@ -1110,6 +1165,8 @@ static int conv2d_run(const void *d_x, int x_bits, int B, int Ci, int H, int W, 
     cudaStream_t st = (cudaStream_t)stream;
     uint32_t *d_wp = (uint32_t *)d_workspace;
     uint32_t *d_ap = (uint32_t *)((char *)d_workspace + s.wp_bytes);
+    int32_t *d_corr = (int32_t *)((char *)d_workspace + s.corr_off);
+    s.kp.corr = d_corr;
     s.kp.x = (const int8_t *)d_x;
     s.kp.wp = d_wp;
     s.kp.ap = d_ap;
@@ -1119,10 +1176,13 @@ static int conv2d_run(const void *d_x, int x_bits, int B, int Ci, int H, int W, 
         WeightPackParams wq;
         wq.w = (const int8_t *)d_w; wq.wp = d_wp; wq.Co = Co; wq.Ci = Ci; wq.K = K; wq.J = s.L.J; wq.Kc = s.L.Kc; wq.S = s.L.S;
         wq.w_signed = w_signed ? 1 : 0; wq.CoP = s.kp.CoP; wq.total = Ci * K * s.L.J * s.kp.CoP; wq.w_bits = w_bits;
+        wq.x_off = s.kp.x_off; wq.corr = d_corr;
         const size_t act_items = (size_t)Ci * B * s.kp.Hp * (s.kp.XBT / 4);
         const size_t act_blocks = (act_items + 255) / 256, w_blocks = (size_t)ceil_div(wq.total, 256);
-        if (act_blocks + w_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
-        const unsigned grid = (unsigned)(act_blocks + w_blocks);
+        const size_t corr_blocks = s.kp.x_off ? (size_t)ceil_div(s.kp.CoP, 8) : 0;      // one warp per channel
+        wq.w_blocks = (int)w_blocks;
+        if (act_blocks + w_blocks + corr_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
+        const unsigned grid = (unsigned)(act_blocks + w_blocks + corr_blocks);
 #define HK_PACK(XSIGN, NN)                                                                                                 \
     rc = launch_dependent(pack_operands_kernel<XSIGN, NN>, dim3(grid), dim3(256), 0, st, (const int8_t *)d_x, B, Ci, H, W, s.kp.Hp, \
                           pad, K, s.L.J, s.L.S, s.kp.XBT, d_ap, (int)act_blocks, wq, x_bits)

@@ -88,6 +88,22 @@ def test_carry_save_schedules(ci):
             assert_exact(_layer(x, w, 1, 4, 4, False, True, hk.ALGO_PACKED32, tune=tune), direct.conv2d_nchw(x, w, 1), "extreme ci=%d" % ci)
 
 
+@pytest.mark.parametrize("p", [1, 2, 3, 4, 6, 8])
+def test_deep_unsigned_layers_on_shifted_codes(p):
+    # unsigned activations x signed weights with 128 or more input channels may be packed as x - 2^(p-1) (the padding
+    # included) and get 2^(p-1) * (the channel's weight sum) back in the epilogue: image borders, valid convolution,
+    # several kernel sizes, channel counts that are not multiples of four, requantised output, extreme codes
+    for (K, pad, q, Co) in ((3, 1, 4, 7), (3, 0, 2, 4), (1, 0, 4, 18), (5, 2, 2, 5), (3, 2, 3, 6)):
+        x, w = inputs.conv2d_case(2, 131, 6, 11, Co, K, p, q, False, True, seed=7000 + 10 * p + K + pad)
+        ref = direct.conv2d_nchw(x, w, pad)
+        assert_exact(_layer(x, w, pad, p, q, False, True, hk.ALGO_PACKED32), ref, "p=%d q=%d K=%d pad=%d" % (p, q, K, pad))
+        rq = (p + q - 2, 0, 15)
+        assert_exact(_layer(x, w, pad, p, q, False, True, hk.ALGO_PACKED32, requant=rq), direct.requant(ref, *rq),
+                     "requant p=%d q=%d K=%d pad=%d" % (p, q, K, pad))
+    for x, w in inputs.extreme_2d(1, 160, 5, 9, 6, 3, p, 4, False, True):
+        assert_exact(_layer(x, w, 1, p, 4, False, True, hk.ALGO_PACKED32), direct.conv2d_nchw(x, w, 1), "extreme p=%d" % p)
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_extreme_codes(algo):
     for (p, q, xs, ws) in ((4, 4, True, True), (4, 4, False, True), (8, 4, False, True), (8, 8, True, True), (1, 1, True, True)):

@@ -82,6 +82,20 @@ def test_first_layer_bytes_in_dense_out_pooled():
     assert np.array_equal(got, ref)
 
 
+def test_deep_layer_dense_in_and_out_on_shifted_codes():
+    # 128 and more input channels, unsigned dense activations against signed dense weights: the layer runs on codes
+    # shifted by 2^(p-1); dense, pooled and plain outputs
+    for (B, Ci, H, W, Co, bits) in ((2, 128, 8, 16, 12, 4), (1, 200, 6, 32, 5, 2), (2, 136, 4, 8, 9, 1)):
+        x, w = inputs.conv2d_case(B, Ci, H, W, Co, 3, bits, 4 if bits == 4 else bits, False, True, seed=900 + Ci)
+        q = 4 if bits == 4 else bits
+        got, ref = _run(x, w, 1, bits, q, False, True, bits, q, None, 32, False, hk.ALGO_PACKED32)
+        assert np.array_equal(got, ref), (B, Ci, H, W, Co, bits)
+        for pool in (False, True):
+            for out_store in (4, 8):
+                got, ref = _run(x, w, 1, bits, q, False, True, bits, q, (bits + q - 1, 0, 15), out_store, pool, hk.ALGO_PACKED32)
+                assert np.array_equal(got, ref), (B, Ci, H, W, Co, bits, pool, out_store)
+
+
 def test_extreme_codes_dense():
     for xs, ws in ((True, True), (False, True)):
         for x, w in inputs.extreme_2d(2, 20, 8, 16, 9, 3, 4, 4, xs, ws):
