@@ -272,12 +272,17 @@ def run_ours(args):
     peaks = None
     if rank == 0:
         peaks = {}
-        for kind in ("mad_wide_u32", "mad_wide_s32", "mad_lo_s32", "logic", "shift", "prmt"):
+        for kind in ("mad_wide_u32", "mad_wide_s32", "mad_lo_s32", "logic", "shift", "prmt", "mad_wide_with_logic"):
             r = hk.pipe_rate(kind, iters=2048, device=dev)
             peaks[kind] = {"T_per_s": r["ops_per_second"] / 1e12, "lanes_per_clk_per_sm_at_max_clock": r["lanes_per_clock_per_sm"]}
         peaks["derived"] = {"mad_wide_T_per_s": imad_peak["packed"] / 1e12, "mad_lo_T_per_s": imad_peak["unpacked"] / 1e12,
                             "how": "SMs x lanes/clk x max SM clock (%d SMs, %d / %d lanes, %.0f MHz)"
                                    % (sms, IMAD_WIDE_PER_CLK_PER_SM, IMAD32_PER_CLK_PER_SM, sm_max_mhz)}
+        # scheduler cycles per warp-wide multiply-add = 128 / (lanes per clock and SM); the mixed kernel issues one logic
+        # instruction per two multiply-adds, so twice the difference is what one such instruction costs the multiply stream
+        pure, mixed = (peaks[k]["lanes_per_clk_per_sm_at_max_clock"] for k in ("mad_wide_u32", "mad_wide_with_logic"))
+        peaks["issue_model"] = {"cycles_per_wide_multiply_add": 128.0 / pure,
+                                "cycles_added_per_other_instruction": 2.0 * (128.0 / mixed - 128.0 / pure)}
         imad_peak["packed_measured"] = max(peaks["mad_wide_u32"]["T_per_s"], peaks["mad_wide_s32"]["T_per_s"]) * 1e12
         imad_peak["unpacked_measured"] = peaks["mad_lo_s32"]["T_per_s"] * 1e12
 

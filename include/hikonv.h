@@ -335,7 +335,7 @@ double hikonv_conv2d_multiplies(int B, int Ci, int H, int W, int Co, int K, int 
  * (best of three launches after a warm-up; the call SYNCHRONISES) and returns instructions x 32 lanes per second
  * in *h_ops_per_second and, if h_lanes_per_clock_per_sm is not NULL, that rate divided by (SM count x the device's
  * maximum SM clock).  d_scratch_word: one 4-byte device word owned by the caller.  iters: loop trips of 64
- * instructions per thread (1 .. 2^20).
+ * instructions per thread (1 .. 2^20; the mixed kind runs 32 logic instructions on top, which are not counted).
  */
 typedef enum {
     HIKONV_PIPE_MAD_WIDE_U32 = 0, /* mad.wide.u32: the packed multiply of unsigned layouts       */
@@ -343,7 +343,10 @@ typedef enum {
     HIKONV_PIPE_MAD_LO_S32 = 2,   /* mad.lo.s32: the comparator's 32-bit multiply-add            */
     HIKONV_PIPE_LOGIC = 3,        /* lop3.b32: masks of the split and of the carry-save moves    */
     HIKONV_PIPE_SHIFT = 4,        /* shf.r: the funnel shifts of the split                       */
-    HIKONV_PIPE_PRMT = 5          /* prmt.b32: code extraction and byte-aligned slot extraction  */
+    HIKONV_PIPE_PRMT = 5,         /* prmt.b32: code extraction and byte-aligned slot extraction  */
+    HIKONV_PIPE_MAD_WIDE_WITH_LOGIC = 6 /* mad.wide.u32 with one lop3.b32 (on other registers) per two of them:
+                                     the rate of the multiply-adds alone in that mix; against kind 0 it tells what an
+                                     instruction of another pipe costs the stream of packed multiplies              */
 } hikonv_pipe_kind;
 int hikonv_pipe_rate(int kind, int iters, uint32_t *d_scratch_word, double *h_ops_per_second,
                      double *h_lanes_per_clock_per_sm, void *stream);

@@ -18,7 +18,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NO_FIT, ERR_WORKSPACE, ERR_CUDA, ERR_T
 STATIC_SCRATCH_BYTES = 4 << 20
 ALGO_PACKED32, ALGO_PACKED64EMU, ALGO_UNPACKED_IMAD, ALGO_DP4A = 0, 1, 2, 3
 GB_SINGLE, GB_1D, GB_DNN = 0, 1, 2
-PIPE_KINDS = {"mad_wide_u32": 0, "mad_wide_s32": 1, "mad_lo_s32": 2, "logic": 3, "shift": 4, "prmt": 5}
+PIPE_KINDS = {"mad_wide_u32": 0, "mad_wide_s32": 1, "mad_lo_s32": 2, "logic": 3, "shift": 4, "prmt": 5,
+              "mad_wide_with_logic": 6}
 
 
 class HikonvError(RuntimeError):

@@ -5,6 +5,10 @@
 // eight independent dependency chains of the instruction in registers; the multiplicand of each step is the
 // low half of the NEXT chain's accumulator, so no product is loop-invariant and nothing can be hoisted or folded.
 // The wide multiply-adds use the library's own helper (mad_wide), so the measurement counts what the kernels run.
+// HIKONV_PIPE_MAD_WIDE_WITH_LOGIC interleaves one three-input logic instruction (on registers of its own) per two
+// wide multiply-adds and reports the rate of the multiply-adds alone: what an instruction of another pipe costs
+// the multiply-add stream (the layer kernels spend one to two such instructions per multiply-add on loads, carry-save
+// moves and the split).
 // Grid: four CTAs of 256 threads per SM (eight warps per scheduler, 64 independent instructions in flight on
 // each), timed with CUDA events around the launch.
 #include "hikonv_cuda.cuh"
@@ -19,8 +23,11 @@ __global__ void __launch_bounds__(256) pipe_rate_kernel(int iters, uint32_t seed
     const uint32_t tid = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t b = seed | 1u;                              // an odd multiplier: the chain never collapses to zero
     uint64_t acc[kChains];
+    uint32_t side[kChains / 2];                                // the logic instructions of the mixed kind work on these
 #pragma unroll
     for (int c = 0; c < kChains; ++c) acc[c] = ((uint64_t)(tid + 1) << 20) + 977u * c + seed;
+#pragma unroll
+    for (int c = 0; c < kChains / 2; ++c) side[c] = tid * 2654435761u + c;
     for (int it = 0; it < iters; ++it) {
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
@@ -29,7 +36,13 @@ __global__ void __launch_bounds__(256) pipe_rate_kernel(int iters, uint32_t seed
                 const uint32_t lo = (uint32_t)acc[c];
                 const uint32_t hi = (uint32_t)(acc[c] >> 32);
                 const uint32_t other = (uint32_t)acc[(c + 1) % kChains];
-                if (KIND == HIKONV_PIPE_MAD_WIDE_U32) {
+                if (KIND == HIKONV_PIPE_MAD_WIDE_WITH_LOGIC) {
+                    mad_wide<false>(acc[c], other, b);
+                    if (c & 1) {
+                        const int j = c >> 1;
+                        asm volatile("lop3.b32 %0, %0, %1, %2, 0x96;" : "+r"(side[j]) : "r"(b), "r"(side[(j + 1) % (kChains / 2)]));
+                    }
+                } else if (KIND == HIKONV_PIPE_MAD_WIDE_U32) {
                     mad_wide<false>(acc[c], other, b);
                 } else if (KIND == HIKONV_PIPE_MAD_WIDE_S32) {
                     mad_wide<true>(acc[c], other, b);
@@ -56,6 +69,8 @@ __global__ void __launch_bounds__(256) pipe_rate_kernel(int iters, uint32_t seed
     uint32_t x = 0;
 #pragma unroll
     for (int c = 0; c < kChains; ++c) x ^= (uint32_t)acc[c] ^ (uint32_t)(acc[c] >> 32);
+#pragma unroll
+    for (int c = 0; c < kChains / 2; ++c) x ^= side[c];
     if (x == 0x9E3779B9u) sink[0] = x;                          // keeps the chains alive; practically never true
 }
 
@@ -72,6 +87,7 @@ static int launch_kind(int kind, int iters, unsigned grid, cudaStream_t st, uint
         case HIKONV_PIPE_LOGIC: return run_kind<HIKONV_PIPE_LOGIC>(iters, grid, st, d_sink);
         case HIKONV_PIPE_SHIFT: return run_kind<HIKONV_PIPE_SHIFT>(iters, grid, st, d_sink);
         case HIKONV_PIPE_PRMT: return run_kind<HIKONV_PIPE_PRMT>(iters, grid, st, d_sink);
+        case HIKONV_PIPE_MAD_WIDE_WITH_LOGIC: return run_kind<HIKONV_PIPE_MAD_WIDE_WITH_LOGIC>(iters, grid, st, d_sink);
         default: return HIKONV_ERR_INVALID_ARG;
     }
 }
@@ -83,7 +99,7 @@ using namespace hikonv;
 extern "C" int hikonv_pipe_rate(int kind, int iters, uint32_t *d_scratch_word, double *h_ops_per_second,
                                 double *h_lanes_per_clock_per_sm, void *stream) {
     if (!d_scratch_word || !h_ops_per_second || iters < 1 || iters > (1 << 20)) return HIKONV_ERR_INVALID_ARG;
-    if (kind < HIKONV_PIPE_MAD_WIDE_U32 || kind > HIKONV_PIPE_PRMT) return HIKONV_ERR_INVALID_ARG;
+    if (kind < HIKONV_PIPE_MAD_WIDE_U32 || kind > HIKONV_PIPE_MAD_WIDE_WITH_LOGIC) return HIKONV_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     int dev = 0, sms = 0, khz = 0;
     HIKONV_CUDA_TRY(cudaGetDevice(&dev));
