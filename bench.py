@@ -688,7 +688,8 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
             muls = hk.conv2d_multiplies(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
                                         shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], algo)
             rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key)}
-        rec["layout"] = hk.layout(shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], shape["K"], 2, shape["Ci"] * shape["K"])
+        rec["layout"] = hk.conv2d_layout(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
+                                         shape["p"], shape["q"], shape["x_signed"], shape["w_signed"])
         rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
         if rq and shape["p"] == 4 and shape["q"] == 4:
             # the same layer with all three tensors stored densely (two 4-bit codes per byte): half the bytes per tensor

@@ -234,7 +234,10 @@ int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, 
  * d_workspace: hikonv_conv2d_workspace_bytes(...) bytes of device memory, 256-byte aligned; the call
  * overwrites it and needs nothing from it afterwards.  The unpacked comparator uses the same workspace for
  * int32 copies of the weights and codes.
- * stride must be 1 and 0 <= pad < K.
+ * stride must be 1 and 0 <= pad < K.  Limits (HIKONV_ERR_UNSUPPORTED beyond them): Ho < 60000; B Ci H W and B Ho
+ * below 2^31; (images a tile of rows can touch + 1) x Co x Ho x Wo below 2^32 (output offsets inside a CTA are 32-bit).
+ * Layers with unsigned activations, signed weights and 128 or more input channels may run on activation codes shifted
+ * by 2^(p-1) (see hikonv_conv2d_layout); results are the same exact sums.
  */
 int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,
                   int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out,
@@ -242,9 +245,20 @@ int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *
                   int algo, const hikonv_tuning_t *tune, void *stream);
 
 /*
- * hikonv_conv2d_dense - hikonv_conv2d on tensors stored without their unused bits (Section V-B, "Single convolver
- * architecture": weights are kept compressed in memory, and "the same compression can also be applied to the
- * feature data during runtime"), with the layer's requantised output written in the same compressed form and,
+ * hikonv_conv2d_layout - the packed layout hikonv_conv2d(HIKONV_ALGO_PACKED32) runs this layer with (host only).
+ * *out: N, S, Kc, J, slots, M (accumulated (ci, kh) pairs between two carry-save moves), as hikonv_layout reports them.
+ * *x_shift (may be NULL): 0, or 2^(p-1) when the layer runs its unsigned activations as signed codes x - 2^(p-1):
+ * the span of a product halves, a slot takes about twice as many products between moves, and the epilogue adds
+ * 2^(p-1) x (sum of the output channel's weights) back.  *out is then the layout for signed activations, which is
+ * not what hikonv_layout reports for the layer's own signs.  Arguments and errors as for hikonv_conv2d.
+ */
+int hikonv_conv2d_layout(int B, int Ci, int H, int W, int Co, int K, int pad, int p, int q, int x_signed,
+                         int w_signed, const hikonv_tuning_t *tune, hikonv_layout_t *out, int *x_shift);
+
+/*
+ * hikonv_conv2d_dense - hikonv_conv2d on tensors stored without their unused bits (Section V-B, single convolver
+ * architecture: the weights sit in memory in compressed form, and the section notes that features can be kept
+ * that way at run time too), with the layer's requantised output written in the same compressed form and,
  * optionally, max-pooled on the way out.
  *   Dense storage of a tensor of b-bit codes, b in {1, 2, 4}: the codes in their NCHW (OIHW) order, 8 / b per
  *   byte, code e in bits [(e b) % 8, (e b) % 8 + b) of byte (e b) / 8, two's complement when signed;

@@ -68,6 +68,7 @@ _SIGNATURES = {
     "hikonv_maxpool2x2_i8": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _vp]),
     "hikonv_conv1d_multiplies": (_d, [_sz, _i, _i, _i, _i, _i, _i, ctypes.POINTER(TuningT)]),
     "hikonv_conv2d_multiplies": (_d, [_i] * 12 + [ctypes.POINTER(TuningT)]),
+    "hikonv_conv2d_layout": (_i, [_i] * 11 + [ctypes.POINTER(TuningT), ctypes.POINTER(LayoutT), ctypes.POINTER(_i)]),
     "hikonv_pipe_rate": (_i, [_i, _i, _vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), _vp]),
     "hikonv_status_string": (ctypes.c_char_p, [_i]),
 }
@@ -169,6 +170,17 @@ def conv1d_layout(p, q, f_signed, g_signed, K, tune=None) -> dict:
     _check(lib().hikonv_conv1d_layout(p, q, int(f_signed), int(g_signed), K, _tune(tune), ctypes.byref(out)),
            "hikonv_conv1d_layout")
     return {n: getattr(out, n) for n, _ in LayoutT._fields_}
+
+
+def conv2d_layout(B, Ci, H, W, Co, K, pad, p, q, x_signed, w_signed, tune=None) -> dict:
+    """The layout ``conv2d`` (packed algorithm) runs this layer with, plus ``x_shift``: 0, or 2^(p-1) when the layer
+    runs its unsigned activations as signed codes shifted by that much."""
+    out, shift = LayoutT(), ctypes.c_int(0)
+    _check(lib().hikonv_conv2d_layout(B, Ci, H, W, Co, K, pad, p, q, int(x_signed), int(w_signed), _tune(tune), ctypes.byref(out),
+                                      ctypes.byref(shift)), "hikonv_conv2d_layout")
+    d = {n: getattr(out, n) for n, _ in LayoutT._fields_}
+    d["x_shift"] = shift.value
+    return d
 
 
 # ------------------------------------------------------------------ device entry points

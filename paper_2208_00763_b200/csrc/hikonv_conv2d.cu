@@ -1339,6 +1339,18 @@ extern "C" int hikonv_maxpool2x2_i8(const int8_t *d_in, int B, int C, int H, int
                         is_signed ? 1 : 0, d_out);
 }
 
+extern "C" int hikonv_conv2d_layout(int B, int Ci, int H, int W, int Co, int K, int pad, int p, int q, int x_signed,
+                                    int w_signed, const hikonv_tuning_t *tune, hikonv_layout_t *out, int *x_shift) {
+    if (!out) return HIKONV_ERR_INVALID_ARG;
+    Conv2dSetup s;
+    const int rc = make_setup(B, Ci, H, W, Co, K, 1, pad, p, q, x_signed ? 1 : 0, w_signed ? 1 : 0, 0, 0, 0, 0,
+                              HIKONV_ALGO_PACKED32, tune, &s);
+    if (rc != HIKONV_OK) return rc;
+    *out = s.L;
+    if (x_shift) *x_shift = s.kp.x_off;
+    return HIKONV_OK;
+}
+
 extern "C" double hikonv_conv2d_multiplies(int B, int Ci, int H, int W, int Co, int K, int pad, int p, int q, int x_signed,
                                            int w_signed, int algo, const hikonv_tuning_t *tune) {
     Conv2dSetup s;

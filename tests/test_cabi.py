@@ -319,3 +319,26 @@ def test_register_aligned_layout_conditions():
                         else:
                             plan = hk.conv1d_layout(p, q, fs, gs, K, {"tile": -1})
                             assert got == (plan["N"], plan["S"], plan["Kc"], plan["J"]), (p, q, fs, gs, K)
+
+
+def test_conv2d_layout_reports_the_shifted_activation_codes():
+    # deep layers with unsigned activations and signed weights run on codes x - 2^(p-1): the signed layout's larger M,
+    # at least half again the unsigned one's; shallower layers, signed activations and unsigned weights keep their own
+    deep = hk.conv2d_layout(64, 256, 14, 14, 256, 3, 1, 4, 4, False, True)
+    own = hk.layout(4, 4, False, True, 3, 2, 256 * 3)
+    signed = hk.layout(4, 4, True, True, 3, 2, 256 * 3)
+    assert deep["x_shift"] == 8
+    assert (deep["N"], deep["S"], deep["M"]) == (signed["N"], signed["S"], signed["M"])
+    assert 2 * deep["M"] >= 3 * own["M"] and deep["N"] >= own["N"]
+    assert hk.conv2d_layout(64, 64, 20, 40, 64, 3, 1, 4, 4, False, True)["x_shift"] == 0          # fewer than 128 channels
+    assert hk.conv2d_layout(32, 256, 14, 14, 64, 3, 1, 4, 4, True, True)["x_shift"] == 0          # signed already
+    assert hk.conv2d_layout(32, 256, 14, 14, 64, 3, 1, 4, 4, False, False)["x_shift"] == 0        # products never negative
+    for p in (1, 2, 3, 5, 8):
+        L = hk.conv2d_layout(2, 200, 9, 11, 8, 3, 1, p, 4, False, True)
+        assert L["x_shift"] in (0, 1 << (p - 1))
+    # the multiply count follows the layout that runs
+    L = hk.conv2d_layout(2, 130, 6, 17, 12, 3, 1, 4, 4, False, True)
+    muls = hk.conv2d_multiplies(2, 130, 6, 17, 12, 3, 1, 4, 4, False, True, hk.ALGO_PACKED32)
+    assert muls > 0 and muls % (130 * 3 * L["J"] * 12) == 0
+    with pytest.raises(hk.HikonvError):
+        hk.conv2d_layout(1, 4, 60000, 8, 4, 3, 1, 4, 4, True, True)                                # rows beyond the index arithmetic
