@@ -110,6 +110,27 @@ __device__ __forceinline__ int fast_div(int n, uint32_t magic) {
     return magic ? (int)__umulhi((uint32_t)n, magic) : n;
 }
 
+// n / d for any 32-bit n and a divisor d >= 1 fixed per launch (division by invariant integers using
+// multiplication, Granlund and Montgomery 1994): with L = ceil(log2 d) and m = floor(2^32 (2^L - d) / d) + 1,
+// t = mulhi(m, n) and n / d = (t + ((n - t) >> min(L, 1))) >> max(L - 1, 0).  Five instructions instead of the
+// twenty-odd of a hardware-less 32-bit division.
+struct Div32 {
+    uint32_t m, s1, s2;
+};
+__host__ inline Div32 make_div32(uint32_t d) {
+    uint32_t L = 0;
+    while (L < 32 && (1ull << L) < d) ++L;
+    Div32 r;
+    r.m = (uint32_t)(((1ull << 32) * ((1ull << L) - d)) / d + 1);
+    r.s1 = L < 1 ? L : 1;
+    r.s2 = L > 1 ? L - 1 : 0;
+    return r;
+}
+__device__ __forceinline__ uint32_t div32(uint32_t n, const Div32 &d) {
+    const uint32_t t = __umulhi(d.m, n);
+    return (t + ((n - t) >> d.s1)) >> d.s2;
+}
+
 // One multiply-accumulate of the k loop: the packed 32x32->64 product of Eq. 9 added to the 64-bit
 // accumulator, or (comparator) one 32-bit product added to an int32 sum.
 template <bool UNPACKED, bool SP>
@@ -605,6 +626,7 @@ struct WeightPackParams {
     int Co, Ci, K, J, Kc, S, w_signed, CoP, total;
     int w_bits;                // storage: 8 = one code per byte, 1 / 2 / 4 = dense (8 / w_bits codes per byte)
     int w_blocks;              // CTAs that pack kernel rows; the CTAs after them sum the weights of a channel (x_off != 0)
+    Div32 d_cop, d_j, d_k;     // divisions of pack_weight_word
     int x_off;                 // offset taken from every activation code (0: none)
     int32_t *corr;             // corr[co] = x_off * sum of the weights of channel co, CoP entries
 };
@@ -622,12 +644,14 @@ __device__ __forceinline__ int32_t load_dense_code(const int8_t *base, size_t e,
 
 __device__ __forceinline__ void pack_weight_word(const WeightPackParams &q, int idx) {
     if (idx >= q.total) return;
-    const int co = idx % q.CoP;
-    int rest = idx / q.CoP;
-    const int j = rest % q.J;
-    rest /= q.J;
-    const int kh = rest % q.K;
-    const int ci = rest / q.K;
+    uint32_t rest = div32((uint32_t)idx, q.d_cop);
+    const int co = idx - (int)rest * q.CoP;
+    uint32_t up = div32(rest, q.d_j);
+    const int j = (int)(rest - up * q.J);
+    rest = up;
+    up = div32(rest, q.d_k);
+    const int kh = (int)(rest - up * q.K);
+    const int ci = (int)up;
     uint32_t word = 0;
     if (co < q.Co) {
         const size_t row_e = (((size_t)co * q.Ci + ci) * q.K + kh) * q.K;       // first code of the kernel row
@@ -673,32 +697,38 @@ __device__ __forceinline__ void sum_channel_weights(const WeightPackParams &q, i
 // x = xb - J of padded row hp, i.e. columns (xb - J) N + K - 1 - pad + n of input row hp - pad, zero where the
 // row or a column lies in the padding.  For the comparator S == 0 and N == 1: one int32 code per word.
 // One thread packs four consecutive words of a row (one 16-byte store); threads are numbered through all
-// (ci, b) planes, so that small maps still fill their CTAs.  The CTAs past the
-// activation planes pack the kernel rows (one word per thread), so that a layer needs one packing launch.
+// (ci, b) planes, so that small maps still fill their CTAs.  The first CTAs of the launch sum the channels' weights
+// (when the layer runs on shifted codes) and pack the kernel rows (one word per thread), so that a layer needs one
+// packing launch and its longest serial work starts first.
 // x_bits: storage of the activations, 8 = one code per byte, 1 / 2 / 4 = dense.
 // With wq.x_off != 0 every slot holds code - x_off, the slots outside the image included (code 0 there).
+struct ActPackDivs {
+    Div32 per_plane, b, xq;    // pieces per (ci, b) plane, images, 16-byte pieces per packed row
+};
+
 template <bool XS, int N>
 __global__ void __launch_bounds__(256) pack_operands_kernel(const int8_t *__restrict__ x, int B, int Ci, int H, int W, int Hp,
                                                             int pad, int K, int J, int S, int XBT,
-                                                            uint32_t *__restrict__ ap, int act_blocks, const WeightPackParams wq,
-                                                            int x_bits) {
+                                                            uint32_t *__restrict__ ap, int weight_blocks, const WeightPackParams wq,
+                                                            int x_bits, const ActPackDivs dv, unsigned act_items) {
     grid_dependency_release();
     grid_dependency_wait();                                          // the input may come from the kernel before; the workspace may still be read by it
-    if ((int)blockIdx.x >= act_blocks) {
-        const int wb = (int)blockIdx.x - act_blocks;
-        if (wb < wq.w_blocks) pack_weight_word(wq, wb * 256 + (int)threadIdx.x);
-        else sum_channel_weights(wq, (wb - wq.w_blocks) * 8 + ((int)threadIdx.x >> 5), (int)threadIdx.x & 31);
+    // the first CTAs sum the channels' weights (the longest serial work of the launch) and pack the kernel rows
+    if ((int)blockIdx.x < weight_blocks) {
+        const int cb = weight_blocks - wq.w_blocks;                  // CTAs that sum weights (0 unless x_off != 0)
+        if ((int)blockIdx.x < cb) sum_channel_weights(wq, (int)blockIdx.x * 8 + ((int)threadIdx.x >> 5), (int)threadIdx.x & 31);
+        else pack_weight_word(wq, ((int)blockIdx.x - cb) * 256 + (int)threadIdx.x);
         return;
     }
     // the (plane, piece) pairs are numbered through: a CTA may span several small planes (ci * B + b)
     const int xq = XBT / 4;                                          // 16-byte pieces per packed row
     const int per_plane = Hp * xq;
-    const long long item = (long long)blockIdx.x * 256 + threadIdx.x;
-    if (item >= (long long)Ci * B * per_plane) return;
-    const int plane = (int)(item / per_plane);
-    const int piece = (int)(item - (long long)plane * per_plane);
-    const int ci = plane / B, b = plane - ci * B;
-    const int hp = piece / xq, q = piece - hp * xq;
+    const unsigned item = (blockIdx.x - (unsigned)weight_blocks) * 256u + threadIdx.x;
+    if (item >= act_items) return;
+    const int plane = (int)div32(item, dv.per_plane);
+    const int piece = (int)(item - (unsigned)plane * (unsigned)per_plane);
+    const int ci = (int)div32((uint32_t)plane, dv.b), b = plane - ci * B;
+    const int hp = (int)div32((uint32_t)piece, dv.xq), q = piece - hp * xq;
     const int hi = hp - pad;
     uint32_t fill = 0u;                                              // a word whose N slots all hold -x_off
     if (wq.x_off != 0) {
@@ -1177,15 +1207,20 @@ static int conv2d_run(const void *d_x, int x_bits, int B, int Ci, int H, int W, 
         wq.w = (const int8_t *)d_w; wq.wp = d_wp; wq.Co = Co; wq.Ci = Ci; wq.K = K; wq.J = s.L.J; wq.Kc = s.L.Kc; wq.S = s.L.S;
         wq.w_signed = w_signed ? 1 : 0; wq.CoP = s.kp.CoP; wq.total = Ci * K * s.L.J * s.kp.CoP; wq.w_bits = w_bits;
         wq.x_off = s.kp.x_off; wq.corr = d_corr;
-        const size_t act_items = (size_t)Ci * B * s.kp.Hp * (s.kp.XBT / 4);
+        wq.d_cop = make_div32((uint32_t)s.kp.CoP); wq.d_j = make_div32((uint32_t)s.L.J); wq.d_k = make_div32((uint32_t)K);
+        const size_t act_items = (size_t)Ci * B * s.kp.Hp * (s.kp.XBT / 4);              // below 2^29: ap_words is below 2^31
         const size_t act_blocks = (act_items + 255) / 256, w_blocks = (size_t)ceil_div(wq.total, 256);
         const size_t corr_blocks = s.kp.x_off ? (size_t)ceil_div(s.kp.CoP, 8) : 0;      // one warp per channel
         wq.w_blocks = (int)w_blocks;
         if (act_blocks + w_blocks + corr_blocks > 0x7FFFFFFFull) return HIKONV_ERR_UNSUPPORTED;
         const unsigned grid = (unsigned)(act_blocks + w_blocks + corr_blocks);
+        ActPackDivs dv;
+        dv.per_plane = make_div32((uint32_t)(s.kp.Hp * (s.kp.XBT / 4)));
+        dv.b = make_div32((uint32_t)B);
+        dv.xq = make_div32((uint32_t)(s.kp.XBT / 4));
 #define HK_PACK(XSIGN, NN)                                                                                                 \
     rc = launch_dependent(pack_operands_kernel<XSIGN, NN>, dim3(grid), dim3(256), 0, st, (const int8_t *)d_x, B, Ci, H, W, s.kp.Hp, \
-                          pad, K, s.L.J, s.L.S, s.kp.XBT, d_ap, (int)act_blocks, wq, x_bits)
+                          pad, K, s.L.J, s.L.S, s.kp.XBT, d_ap, (int)(w_blocks + corr_blocks), wq, x_bits, dv, (unsigned)act_items)
         switch (s.L.N * 2 + (x_signed ? 1 : 0)) {
             case 2: HK_PACK(false, 1); break;
             case 3: HK_PACK(true, 1); break;
