@@ -517,7 +517,7 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
 
         def step():
             net.forward(d_x, algo=algo)
-        launches_per_step = 2 * 9 + 4   # nine layers of two launches, four pools
+        launches_per_step = 2 * 9       # nine layers of two launches (packing + layer; the four pools run inside their layers)
         name = "c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head" % x.shape[0]
         h2d = d_x.numel()
         d2h = x.shape[0] * 36 * H * W * 4

@@ -180,11 +180,12 @@ def test_compact_cnn_small_batch(algo):
     assert_exact(head, ref_head, "head")
 
 
-def test_compact_cnn_with_pools_fused_into_the_layers():
+@pytest.mark.parametrize("fused_pool", [True, False])
+def test_compact_cnn_with_pools_fused_into_the_layers_or_launched_apart(fused_pool):
     x, layers, head_w = inputs.c5_network(batch=3, H=32, W=64)
     ref_head, ref_acts = direct.cnn_forward(x, layers, head_w)
     net = network.CompactCnn(layers, head_w, device="cuda")
-    head, acts = net.forward(dev(x), keep_activations=True, fused_pool=True)
+    head, acts = net.forward(dev(x), keep_activations=True, fused_pool=fused_pool)
     for i, (a, r) in enumerate(zip(acts, ref_acts)):
         assert_exact(a, r, "layer %d" % (i + 1))
     assert_exact(head, ref_head, "head")
