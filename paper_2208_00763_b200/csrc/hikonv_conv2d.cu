@@ -12,7 +12,9 @@
 //
 // Activations are packed once per layer by pack_operands_kernel into Ap[ci][b*Hp + hp][xb] (zero padding
 // rows and halo words materialised), weights by the same launch into Bw[(ci,kh,j)][co]; the layer
-// kernel streams both with 16-byte asynchronous copies into double-buffered shared memory.
+// kernel streams both with 16-byte asynchronous copies into double-buffered shared memory.  Deep layers with
+// unsigned activations and signed weights are packed as x - 2^(p-1), padding included, and get the constant
+// 2^(p-1) sum(W[co]) back in the epilogue (make_setup says when and why).
 //
 // A CTA computes TR consecutive output rows (one row segment each) times TCO output channels; it
 // is a register-tiled integer "GEMM" over packed words: each thread owns TM positions times TN
