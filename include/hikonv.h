@@ -236,7 +236,7 @@ int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, 
  * int32 copies of the weights and codes.
  * stride must be 1 and 0 <= pad < K.  Limits (HIKONV_ERR_UNSUPPORTED beyond them): Ho < 60000; B Ci H W and B Ho
  * below 2^31; (images a tile of rows can touch + 1) x Co x Ho x Wo below 2^32 (output offsets inside a CTA are 32-bit).
- * Layers with unsigned activations, signed weights and 128 or more input channels may run on activation codes shifted
+ * Layers with unsigned activations, signed weights and 32 or more input channels may run on activation codes shifted
  * by 2^(p-1) (see hikonv_conv2d_layout); results are the same exact sums.
  */
 int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,

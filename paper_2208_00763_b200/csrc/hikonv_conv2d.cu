@@ -980,11 +980,15 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         int rc = make_layout(p, q, xs, ws, K, 2, Ci * K, Wo, tune, &L);
         if (rc != HIKONV_OK) return rc;
         // Unsigned activations against signed weights: the products of codes x - 2^(p-1) span about half the range,
-        // so a slot takes nearly twice as many of them between two carry-save moves.  Deep layers (measured: 256
-        // input channels 239 -> 222 us; 64 channels on small maps lose 2 us to the extra packing work) whose signed
-        // layout allows at least half again as many products run on the shifted codes and get
-        // 2^(p-1) * (sum of the channel's weights) added back in the epilogue.
-        if (!xs && ws && L.M < Ci * K && Ci >= 128) {
+        // so a slot takes nearly twice as many of them between two carry-save moves.  Layers whose signed layout
+        // allows at least half again as many products run on the shifted codes and get
+        // 2^(p-1) * (sum of the channel's weights) added back in the epilogue: from 128 input channels on always
+        // (measured: 256 channels on 14x14 maps 239 -> 218 us), from 32 on when the layer is large enough to keep four
+        // positions per thread (32 channels on 40x80 maps 112 -> 106 us; the 64-channel layers on 10x20 maps, bound by
+        // the latency of one thread's work, lose 2 us to the longer packing launch and keep their own codes).
+        const double threads4_own = (double)B * Ho * (ceil_div(Wo, L.N) + L.J) / kTM * ceil_div(Co, kTN);
+        const bool small_layer = threads4_own <= 1.1 * sm_count() * 2 * kMaxThreads2D;
+        if (!xs && ws && L.M < Ci * K && (Ci >= 128 || (Ci >= 32 && !small_layer))) {
             hikonv_layout_t Ls;
             if (make_layout(p, q, 1, ws, K, 2, Ci * K, Wo, tune, &Ls) == HIKONV_OK && Ls.N >= L.N && Ls.J <= L.J &&
                 2 * Ls.M >= 3 * L.M) {

@@ -330,7 +330,9 @@ def test_conv2d_layout_reports_the_shifted_activation_codes():
     assert deep["x_shift"] == 8
     assert (deep["N"], deep["S"], deep["M"]) == (signed["N"], signed["S"], signed["M"])
     assert 2 * deep["M"] >= 3 * own["M"] and deep["N"] >= own["N"]
-    assert hk.conv2d_layout(64, 64, 20, 40, 64, 3, 1, 4, 4, False, True)["x_shift"] == 0          # fewer than 128 channels
+    assert hk.conv2d_layout(64, 64, 20, 40, 64, 3, 1, 4, 4, False, True)["x_shift"] == 0          # fewer than 128 channels, small layer
+    assert hk.conv2d_layout(64, 32, 40, 80, 64, 3, 1, 4, 4, False, True)["x_shift"] == 8          # 32 channels on a large layer
+    assert hk.conv2d_layout(64, 16, 80, 160, 32, 3, 1, 4, 4, False, True)["x_shift"] == 0         # fewer than 32 channels
     assert hk.conv2d_layout(32, 256, 14, 14, 64, 3, 1, 4, 4, True, True)["x_shift"] == 0          # signed already
     assert hk.conv2d_layout(32, 256, 14, 14, 64, 3, 1, 4, 4, False, False)["x_shift"] == 0        # products never negative
     for p in (1, 2, 3, 5, 8):
