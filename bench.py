@@ -504,12 +504,13 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         x, layers, head_w = inputs.c5_network(seed=ranks.rank_seed(5, rank), batch=args.batch or 64)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         net = network.CompactCnn(layers, head_w, device=dev)
+        tiles = net.tune_tiles(d_x, algo=algo)              # set-up: the network times tile shapes once per input shape
         macs, muls = 0.0, 0.0
         H, W = x.shape[2], x.shape[3]
-        for L in layers:
+        for L, tile in zip(layers, tiles):
             Co, Ci, K, _ = L["w"].shape
             macs += float(x.shape[0]) * Co * H * W * Ci * K * K
-            muls += hk.conv2d_multiplies(x.shape[0], Ci, H, W, Co, K, L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], algo)
+            muls += hk.conv2d_multiplies(x.shape[0], Ci, H, W, Co, K, L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], algo, tile)
             if L["pool"]:
                 H, W = H // 2, W // 2
         macs += float(x.shape[0]) * head_w.shape[0] * H * W * head_w.shape[1]
@@ -518,7 +519,8 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         def step():
             net.forward(d_x, algo=algo)
         launches_per_step = 2 * 9       # nine layers of two launches (packing + layer; the four pools run inside their layers)
-        name = "c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head" % x.shape[0]
+        name = ("c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head; tile shapes timed once at set-up "
+                "(tuned: %s)" % (x.shape[0], [t["tile"] if t else None for t in tiles]))
         h2d = d_x.numel()
         d2h = x.shape[0] * 36 * H * W * 4
 
@@ -719,16 +721,19 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
     macs += float(x.shape[0]) * head_w.shape[0] * H * W * head_w.shape[1]
     rec = {"macs": macs}
     for key, algo in (("packed", hk.ALGO_PACKED32), ("unpacked", hk.ALGO_UNPACKED_IMAD)):
+        untuned_ms = time_fn(lambda: net.forward(d_x, algo=algo), iters=5)
+        tiles = net.tune_tiles(d_x, algo=algo)              # set-up: the network times tile shapes once per input shape
         ms = time_fn(lambda: net.forward(d_x, algo=algo), iters=5)
         # multiplies the nine layer launches execute (positions incl. halo x Co x Ci x K x J, summed)
         muls, Hl, Wl = 0.0, x.shape[2], x.shape[3]
-        for L in layers:
+        for L, tile in zip(layers, tiles):
             Co, Ci, K, _ = L["w"].shape
-            muls += hk.conv2d_multiplies(x.shape[0], Ci, Hl, Wl, Co, K, L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], algo)
+            muls += hk.conv2d_multiplies(x.shape[0], Ci, Hl, Wl, Co, K, L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], algo, tile)
             if L["pool"]:
                 Hl, Wl = Hl // 2, Wl // 2
         muls += hk.conv2d_multiplies(x.shape[0], head_w.shape[1], Hl, Wl, head_w.shape[0], 1, 0, 4, 4, False, True, algo)
-        rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key)}
+        rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key),
+                    "ms_with_the_library_s_own_tiles": untuned_ms, "tuned_tiles": [t["tile"] if t else None for t in tiles]}
     rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
     out["c5"] = rec
     return out

@@ -245,6 +245,24 @@ int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *
                   int algo, const hikonv_tuning_t *tune, void *stream);
 
 /*
+ * hikonv_conv2d_tune - times the tile shapes of one layer on the device and returns the fastest (a set-up aid with no
+ * counterpart in the paper: the automatic choice comes from a cost model, which on small layers misses tiles that
+ * measure 10-20 % faster).  Arguments up to `algo` are those of hikonv_conv2d_dense (one code per byte: storage 8 / 8,
+ * out_store_bits 8, or 32 without requant).  The call runs the layer with the library's own tile and with every forced
+ * tile (positions per thread 4 and 2 x channel lanes 1, 2, 4, 8 x output rows per CTA 1 .. 48; shapes the layer does not
+ * support are skipped), each as groups of four launches between two CUDA events on `stream`, best of `repeats` (1 .. 100)
+ * groups, and SYNCHRONISES.  Every launch writes the layer's complete, correct output to d_out.
+ * *h_tile: the value for hikonv_tuning_t.tile in later calls on this shape, or 0 when no forced tile is at least 3 %
+ * faster than the automatic one.  *h_us / *h_default_us (may be NULL): microseconds per launch of the winner and of
+ * the automatic choice.  Errors as for hikonv_conv2d_dense; results never depend on the tile.
+ */
+int hikonv_conv2d_tune(const void *d_x, int x_store_bits, int B, int Ci, int H, int W, const void *d_w,
+                       int w_store_bits, int Co, int K, int stride, int pad, int p, int q, int x_signed,
+                       int w_signed, void *d_out, int out_store_bits, int requant, int shift, int lo, int hi,
+                       int pool, void *d_workspace, size_t workspace_bytes, int algo, int repeats, int *h_tile,
+                       double *h_us, double *h_default_us, void *stream);
+
+/*
  * hikonv_conv2d_layout - the packed layout hikonv_conv2d(HIKONV_ALGO_PACKED32) runs this layer with (host only).
  * *out: N, S, Kc, J, slots, M (accumulated (ci, kh) pairs between two carry-save moves), as hikonv_layout reports them.
  * *x_shift (may be NULL): 0, or 2^(p-1) when the layer runs its unsigned activations as signed codes x - 2^(p-1):

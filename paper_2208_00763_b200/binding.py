@@ -59,6 +59,8 @@ _SIGNATURES = {
                            ctypes.POINTER(TuningT), _vp]),
     "hikonv_conv2d_dense": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz,
                                  _i, ctypes.POINTER(TuningT), _vp]),
+    "hikonv_conv2d_tune": (_i, [_vp, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _vp, _sz,
+                                _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_d), ctypes.POINTER(_d), _vp]),
     "hikonv_conv2d_workspace_bytes": (_sz, [_i] * 7),
     "hikonv_conv2d_static_scratch": (_i, [_vp, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _i, _i, _vp, _i, _i, _i, _i, _i,
                                           ctypes.POINTER(TuningT), _vp]),
@@ -274,10 +276,21 @@ def conv2d(d_x: torch.Tensor, d_w: torch.Tensor, pad: int, p: int, q: int, x_sig
     return out
 
 
+def conv2d_tune(d_x: torch.Tensor, x_shape, x_store_bits: int, d_w: torch.Tensor, w_shape, w_store_bits: int, pad: int, p: int,
+                q: int, x_signed: bool, w_signed: bool, requant: Optional[tuple] = None, out_store_bits: int = 8,
+                pool: bool = False, algo: int = ALGO_PACKED32, workspace: Optional[torch.Tensor] = None,
+                out: Optional[torch.Tensor] = None, stride: int = 1, stream=None, repeats: int = 3) -> dict:
+    """Times the tile shapes of this layer on the device (``hikonv_conv2d_tune``; arguments as for ``conv2d_dense``).
+    Returns ``{"tune": {"tile": t} or None, "us": best, "default_us": the automatic choice's, "out": the layer's output}``;
+    pass ``tune`` to later calls on this shape.  Synchronises."""
+    return conv2d_dense(d_x, x_shape, x_store_bits, d_w, w_shape, w_store_bits, pad, p, q, x_signed, w_signed, requant, out_store_bits,
+                        pool, algo, None, workspace, out, stride, stream, _tuner_repeats=int(repeats))
+
+
 def conv2d_dense(d_x: torch.Tensor, x_shape, x_store_bits: int, d_w: torch.Tensor, w_shape, w_store_bits: int, pad: int, p: int,
                  q: int, x_signed: bool, w_signed: bool, requant: Optional[tuple] = None, out_store_bits: int = 8,
                  pool: bool = False, algo: int = ALGO_PACKED32, tune=None, workspace: Optional[torch.Tensor] = None,
-                 out: Optional[torch.Tensor] = None, stride: int = 1, stream=None) -> torch.Tensor:
+                 out: Optional[torch.Tensor] = None, stride: int = 1, stream=None, _tuner_repeats: Optional[int] = None):
     """``conv2d`` on densely stored tensors.  ``d_x`` / ``d_w`` are flat uint8 (dense) or int8 (one code per byte)
     tensors holding the codes of ``x_shape`` = (B, Ci, H, W) / ``w_shape`` = (Co, Ci, K, K).  Returns int32
     [B, Co, Ho, Wo] without ``requant``; with it a flat uint8 tensor of the (optionally pooled) output codes,
@@ -305,6 +318,15 @@ def conv2d_dense(d_x: torch.Tensor, x_shape, x_store_bits: int, d_w: torch.Tenso
                    else torch.empty(nbytes, dtype=torch.uint8, device=d_x.device))
         out_ptr, store = _dev_out(out, "out", nbytes, _CODE_DTYPES, d_x), out_store_bits
     shift, lo, hi = requant if requant else (0, 0, 0)
+    if _tuner_repeats is not None:
+        tile, us, default_us = ctypes.c_int(0), ctypes.c_double(0.0), ctypes.c_double(0.0)
+        with torch.cuda.device(d_x.device):
+            _check(lib().hikonv_conv2d_tune(d_x.data_ptr(), x_store_bits, B, Ci, H, W, d_w.data_ptr(), w_store_bits, Co, K, stride, pad,
+                                            p, q, int(x_signed), int(w_signed), out_ptr, store, 1 if requant else 0, shift, lo, hi,
+                                            1 if pool else 0, workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                            algo, _tuner_repeats, ctypes.byref(tile), ctypes.byref(us), ctypes.byref(default_us),
+                                            _stream(stream)), "hikonv_conv2d_tune")
+        return {"tune": {"tile": tile.value} if tile.value else None, "us": us.value, "default_us": default_us.value, "out": out}
     _check(lib().hikonv_conv2d_dense(d_x.data_ptr(), x_store_bits, B, Ci, H, W, d_w.data_ptr(), w_store_bits, Co, K, stride, pad, p, q,
                                      int(x_signed), int(w_signed), out_ptr, store, 1 if requant else 0, shift, lo, hi,
                                      1 if pool else 0, workspace.data_ptr(), workspace.numel() * workspace.element_size(), algo,

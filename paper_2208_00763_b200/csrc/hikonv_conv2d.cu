@@ -1270,6 +1270,90 @@ extern "C" int hikonv_conv2d_dense(const void *d_x, int x_store_bits, int B, int
                       requant ? out_store_bits : 8, requant, shift, lo, hi, pool, d_workspace, workspace_bytes, algo, tune, stream);
 }
 
+// Times the layer with the library's own tile and with every forced tile shape (positions per thread x channel lanes x
+// rows per CTA), `batch` launches between two events, best of `repeats`; the result of every launch is the layer's output.
+extern "C" int hikonv_conv2d_tune(const void *d_x, int x_store_bits, int B, int Ci, int H, int W, const void *d_w,
+                                  int w_store_bits, int Co, int K, int stride, int pad, int p, int q, int x_signed,
+                                  int w_signed, void *d_out, int out_store_bits, int requant, int shift, int lo, int hi,
+                                  int pool, void *d_workspace, size_t workspace_bytes, int algo, int repeats, int *h_tile,
+                                  double *h_us, double *h_default_us, void *stream) {
+    if (!h_tile || repeats < 1 || repeats > 100) return HIKONV_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t e0, e1;
+    HIKONV_CUDA_TRY(cudaEventCreate(&e0));
+    if (cudaEventCreate(&e1) != cudaSuccess) {
+        cudaEventDestroy(e0);
+        return HIKONV_ERR_CUDA;
+    }
+    constexpr int kBatch = 4;
+    // best time in microseconds per launch with this tuning record; negative: the library refused it; rc_cuda set on a CUDA error
+    int rc_cuda = HIKONV_OK;
+    auto run = [&](const hikonv_tuning_t *tune) {
+        return hikonv_conv2d_dense(d_x, x_store_bits, B, Ci, H, W, d_w, w_store_bits, Co, K, stride, pad, p, q, x_signed, w_signed,
+                                   d_out, out_store_bits, requant, shift, lo, hi, pool, d_workspace, workspace_bytes, algo, tune, stream);
+    };
+    auto time_of = [&](const hikonv_tuning_t *tune, double give_up_above) -> double {
+        float ms = 0.0f;
+        if (cudaEventRecord(e0, st) != cudaSuccess) { rc_cuda = HIKONV_ERR_CUDA; return -1.0; }
+        const int rc = run(tune);
+        if (rc != HIKONV_OK) {
+            if (rc == HIKONV_ERR_CUDA) rc_cuda = rc;
+            return -1.0;
+        }
+        if (cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc_cuda = HIKONV_ERR_CUDA; return -1.0; }
+        if (ms * 1e3 > give_up_above) return ms * 1e3;               // a first launch this slow cannot win
+        double best = 1e30;
+        for (int rep = 0; rep < repeats; ++rep) {
+            if (cudaEventRecord(e0, st) != cudaSuccess) { rc_cuda = HIKONV_ERR_CUDA; return -1.0; }
+            for (int k = 0; k < kBatch; ++k)
+                if (run(tune) != HIKONV_OK) { rc_cuda = HIKONV_ERR_CUDA; return -1.0; }
+            if (cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+                cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc_cuda = HIKONV_ERR_CUDA; return -1.0; }
+            best = std::min(best, (double)ms * 1e3 / kBatch);
+        }
+        return best;
+    };
+    int rc = run(nullptr);                                            // argument errors surface here, before any timing
+    double base = -1.0;
+    if (rc == HIKONV_OK) {
+        base = time_of(nullptr, 1e30);
+        if (base < 0.0) rc = rc_cuda != HIKONV_OK ? rc_cuda : HIKONV_ERR_CUDA;
+    }
+    double best = base;
+    int best_tile = 0;
+    if (rc == HIKONV_OK) {
+        const long long rows = (long long)B * ((long long)H + 2 * pad - K + 1);
+        for (int tm = 4; tm >= 2 && rc_cuda == HIKONV_OK; tm -= 2)
+            for (int tnx = 1; tnx <= 8 && rc_cuda == HIKONV_OK; tnx *= 2)
+                for (int tr = 1; tr <= 48 && tr <= rows && rc_cuda == HIKONV_OK; ++tr) {
+                    hikonv_tuning_t tune;
+                    std::memset(&tune, 0, sizeof(tune));
+                    tune.tile = tr + 1000 * tnx + 100000 * tm;
+                    const double t = time_of(&tune, 2.0 * best);
+                    if (t >= 0.0 && t < best) { best = t; best_tile = tune.tile; }
+                }
+        if (rc_cuda != HIKONV_OK) rc = rc_cuda;
+    }
+    if (rc == HIKONV_OK && best_tile != 0 && best > 0.97 * base) { best = base; best_tile = 0; }   // not worth forcing
+    if (rc == HIKONV_OK && best_tile != 0) {
+        hikonv_tuning_t tune;                                          // leave d_out written by a complete, untimed launch
+        std::memset(&tune, 0, sizeof(tune));
+        tune.tile = best_tile;
+        rc = run(&tune);
+    } else if (rc == HIKONV_OK) {
+        rc = run(nullptr);
+    }
+    if (rc == HIKONV_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = HIKONV_ERR_CUDA;
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (rc != HIKONV_OK) return rc;
+    *h_tile = best_tile;
+    if (h_us) *h_us = best;
+    if (h_default_us) *h_default_us = base;
+    return HIKONV_OK;
+}
+
 // ---- scratch that needs no allocation: a fixed buffer inside the library image, one copy per GPU
 static __device__ __align__(256) unsigned char g_static_scratch[HIKONV_STATIC_SCRATCH_BYTES];
 

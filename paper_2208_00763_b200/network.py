@@ -25,6 +25,7 @@ class CompactCnn:
         self.head_w = torch.from_numpy(inputs.to_storage(head_w)).to(self.device)
         self.workspace = None
         self._ws_shape = None
+        self._tiles = {}          # (algo, fused_pool, input shape) -> per-layer tuning records found by tune_tiles()
 
     def _ensure_workspace(self, shape):
         """One workspace large enough for every layer of a batch of this input shape."""
@@ -43,27 +44,54 @@ class CompactCnn:
         self.workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         self._ws_shape = tuple(shape)
 
+    def _layer(self, a, L, algo, fused_pool, tune, stream):
+        """One conv3x3 layer with its requantisation and, if it has one, its pool."""
+        rq = (L["shift"], L["lo"], L["hi"])
+        if L["pool"] and fused_pool:
+            B, Ci, H, W = a.shape
+            return hk.conv2d_dense(a.reshape(-1), (B, Ci, H, W), 8, L["d_w"].reshape(-1), tuple(L["d_w"].shape), 8, L["pad"], L["p"],
+                                   L["q"], L["x_signed"], L["w_signed"], requant=rq, out_store_bits=8, pool=True, algo=algo,
+                                   tune=tune, workspace=self.workspace, stream=stream)
+        a = hk.conv2d(a, L["d_w"], L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], requant=rq, algo=algo, tune=tune,
+                      workspace=self.workspace, stream=stream)
+        if L["pool"]:
+            a = hk.maxpool2x2_i8(a, is_signed=L["lo"] < 0, stream=stream)
+        return a
+
+    def tune_tiles(self, d_x: torch.Tensor, algo: int = hk.ALGO_PACKED32, fused_pool: bool = True, repeats: int = 3) -> List[Optional[dict]]:
+        """Lets the library time, layer by layer on this input, every tile shape it accepts against its own choice
+        (``hikonv_conv2d_tune``) and keeps a forced tile where it measures at least 3 % faster; later ``forward`` calls
+        on inputs of this shape and these options use the kept tiles.  Results do not depend on the tile.  Returns the
+        per-layer tuning records (None: the library's choice stays)."""
+        self._ensure_workspace(d_x.shape)
+        kept: List[Optional[dict]] = []
+        a = d_x
+        for L in self.layers:
+            B, Ci, H, W = a.shape
+            rq = (L["shift"], L["lo"], L["hi"])
+            pool_here = bool(L["pool"] and fused_pool)
+            found = hk.conv2d_tune(a.reshape(-1), (B, Ci, H, W), 8, L["d_w"].reshape(-1), tuple(L["d_w"].shape), 8, L["pad"], L["p"],
+                                   L["q"], L["x_signed"], L["w_signed"], requant=rq, out_store_bits=8, pool=pool_here, algo=algo,
+                                   workspace=self.workspace, repeats=repeats)
+            kept.append(found["tune"])
+            a = found["out"]
+            if L["pool"] and not fused_pool:
+                a = hk.maxpool2x2_i8(a, is_signed=L["lo"] < 0)
+        torch.cuda.synchronize()
+        self._tiles[(algo, bool(fused_pool), tuple(d_x.shape))] = kept
+        return kept
+
     def forward(self, d_x: torch.Tensor, algo: int = hk.ALGO_PACKED32, keep_activations: bool = False, stream=None,
                 fused_pool: bool = True):
         """``fused_pool``: layers followed by a pool run it inside their epilogue (``hikonv_conv2d_dense`` with one code
         per byte; the default: four launches fewer, 0.651 against 0.654 ms on the benchmark network); otherwise the pool
         is a launch of its own."""
         self._ensure_workspace(d_x.shape)
+        tiles = self._tiles.get((algo, bool(fused_pool), tuple(d_x.shape)))
         acts = []
         a = d_x
-        for L in self.layers:
-            rq = (L["shift"], L["lo"], L["hi"])
-            if L["pool"] and fused_pool:
-                B, Ci, H, W = a.shape
-                Co, _, K, _ = L["d_w"].shape
-                a = hk.conv2d_dense(a.reshape(-1), (B, Ci, H, W), 8, L["d_w"].reshape(-1), tuple(L["d_w"].shape), 8, L["pad"], L["p"],
-                                    L["q"], L["x_signed"], L["w_signed"], requant=rq, out_store_bits=8, pool=True, algo=algo,
-                                    workspace=self.workspace, stream=stream)
-            else:
-                a = hk.conv2d(a, L["d_w"], L["pad"], L["p"], L["q"], L["x_signed"], L["w_signed"], requant=rq, algo=algo,
-                              workspace=self.workspace, stream=stream)
-                if L["pool"]:
-                    a = hk.maxpool2x2_i8(a, is_signed=L["lo"] < 0, stream=stream)
+        for i, L in enumerate(self.layers):
+            a = self._layer(a, L, algo, fused_pool, tiles[i] if tiles else None, stream)
             if keep_activations:
                 acts.append(a)
         last = self.layers[-1]

@@ -344,3 +344,12 @@ def test_conv2d_layout_reports_the_shifted_activation_codes():
     assert muls > 0 and muls % (130 * 3 * L["J"] * 12) == 0
     with pytest.raises(hk.HikonvError):
         hk.conv2d_layout(1, 4, 60000, 8, 4, 3, 1, 4, 4, True, True)                                # rows beyond the index arithmetic
+
+
+def test_tuner_refuses_bad_arguments_before_touching_the_device():
+    tile = ctypes.c_int(-1)
+    args = [None, 8, 1, 1, 4, 4, None, 8, 1, 3, 1, 1, 4, 4, 1, 1, None, 8, 1, 6, -8, 7, 0, None, 0, hk.ALGO_PACKED32]
+    assert hk.lib().hikonv_conv2d_tune(*args, 3, None, None, None, None) == hk.ERR_INVALID_ARG          # nowhere to put the tile
+    assert hk.lib().hikonv_conv2d_tune(*args, 0, ctypes.byref(tile), None, None, None) == hk.ERR_INVALID_ARG
+    assert hk.lib().hikonv_conv2d_tune(*args, 101, ctypes.byref(tile), None, None, None) == hk.ERR_INVALID_ARG
+    assert tile.value == -1

@@ -194,18 +194,44 @@ def test_compact_cnn_with_pools_fused_into_the_layers_or_launched_apart(fused_po
 def test_compact_cnn_full_size_every_image():
     # the benchmark configuration (batch 64, 3x160x320): head output and every layer's activations of all 64
     # images against the oracle (the oracle runs the batch in four parts to bound its int64 buffers)
+    # ... once with the library's own tiles, once with the tiles the network's tuning pass picks on the device
     x, layers, head_w = inputs.c5_network()
     net = network.CompactCnn(layers, head_w, device="cuda")
-    head, acts = net.forward(dev(x), keep_activations=True)
+    d_x = dev(x)
+    results = [net.forward(d_x, keep_activations=True)]
+    kept = net.tune_tiles(d_x)
+    assert len(kept) == len(layers) and all(t is None or t["tile"] > 0 for t in kept)
+    results.append(net.forward(d_x, keep_activations=True))
     torch.cuda.synchronize()
-    g = head.cpu().numpy().astype(np.int64)
-    assert g.shape == (64, 36, 10, 20)
-    g_acts = [a.cpu().numpy() for a in acts]
+    got = [(head.cpu().numpy().astype(np.int64), [a.cpu().numpy() for a in acts]) for head, acts in results]
+    assert got[0][0].shape == (64, 36, 10, 20)
     for b0 in range(0, 64, 16):
         ref_head, ref_acts = direct.cnn_forward(x[b0:b0 + 16], layers, head_w)
-        assert np.array_equal(g[b0:b0 + 16], ref_head), "head, images %d..%d" % (b0, b0 + 15)
-        for i, (a, r) in enumerate(zip(g_acts, ref_acts)):
-            assert np.array_equal(a[b0:b0 + 16].astype(np.int64), r), "layer %d, images %d..%d" % (i + 1, b0, b0 + 15)
+        for which, (g, g_acts) in enumerate(got):
+            assert np.array_equal(g[b0:b0 + 16], ref_head), "head, images %d..%d, pass %d" % (b0, b0 + 15, which)
+            for i, (a, r) in enumerate(zip(g_acts, ref_acts)):
+                assert np.array_equal(a[b0:b0 + 16].astype(np.int64), r), "layer %d, images %d..%d, pass %d" % (i + 1, b0, b0 + 15, which)
+
+
+def test_tuner_times_tiles_and_returns_one_that_gives_the_same_result():
+    for (B, Ci, H, W, Co, p, xs, pool) in ((4, 16, 12, 20, 24, 4, True, False), (8, 64, 10, 20, 64, 4, False, True), (2, 3, 16, 40, 16, 8, False, False)):
+        x, w = inputs.conv2d_case(B, Ci, H, W, Co, 3, p, 4, xs, True, seed=77 + Ci)
+        rq = (6, -8, 7) if xs else (6, 0, 15)
+        want = direct.requant(direct.conv2d_nchw(x, w, 1), *rq)
+        if pool:
+            want = direct.maxpool2x2(want)
+        d_x, d_w = dev(x), dev(w)
+        found = hk.conv2d_tune(d_x.reshape(-1), x.shape, 8, d_w.reshape(-1), w.shape, 8, 1, p, 4, xs, True, requant=rq, pool=pool, repeats=2)
+        assert found["us"] > 0 and found["default_us"] > 0 and found["us"] <= found["default_us"]
+        assert found["tune"] is None or (found["tune"]["tile"] > 0 and found["us"] <= 0.97 * found["default_us"])
+        assert_exact(found["out"], want, "output left by the tuner")
+        again = hk.conv2d_dense(d_x.reshape(-1), x.shape, 8, d_w.reshape(-1), w.shape, 8, 1, p, 4, xs, True, requant=rq, pool=pool,
+                                tune=found["tune"])
+        assert_exact(again, want, "layer with the tuned tile %s" % (found["tune"],))
+    # argument errors come back as they would from the layer call
+    with pytest.raises(hk.HikonvError) as err:
+        hk.conv2d_tune(d_x.reshape(-1), x.shape, 8, d_w.reshape(-1), w.shape, 8, 5, p, 4, xs, True, requant=rq)      # pad >= K
+    assert err.value.status == hk.ERR_UNSUPPORTED
 
 
 def test_layer_chain_captured_in_a_cuda_graph():
