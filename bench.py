@@ -94,6 +94,16 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
+    def keep_busy_until_sampled(self, run_step, synchronize, min_samples: int = 2, timeout_s: float = 3.0):
+        """The timed region can be shorter than nvidia-smi's first sampling period: keep the same steps running,
+        untimed, until the sampler has seen the GPU under this load."""
+        if self.proc is None:
+            return
+        t0 = time.time()
+        while len(self.lines) < min_samples and time.time() - t0 < timeout_s:
+            run_step()
+            synchronize()
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -340,6 +350,8 @@ def run_ours(args):
     main_algo = {"packed": hk.ALGO_PACKED32, "unpacked": hk.ALGO_UNPACKED_IMAD, "dp4a": hk.ALGO_DP4A,
                  "emu64": hk.ALGO_PACKED64EMU}[args.algo]
     total_ms = max_over_ranks(timed_graph(lambda: sweep(main_algo), args.steps, args.warmup))
+    if rank == 0:
+        sampler.keep_busy_until_sampled(lambda: sweep(main_algo), torch.cuda.synchronize)
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step = total_ms / args.steps
     value = ranks.whole_job_rate(macs_per_step, args.steps, total_ms, world)
@@ -504,7 +516,11 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         x, layers, head_w = inputs.c5_network(seed=ranks.rank_seed(5, rank), batch=args.batch or 64)
         d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
         net = network.CompactCnn(layers, head_w, device=dev)
-        tiles = net.tune_tiles(d_x, algo=algo)              # set-up: the network times tile shapes once per input shape
+        if args.c5_tiles == "tune":
+            tiles = net.tune_tiles(d_x, algo=algo)          # set-up: the network times tile shapes once per input shape
+        else:                                               # "auto": the library's own tiles; else tile values found earlier, one per layer
+            tiles = [None] * len(layers) if args.c5_tiles == "auto" else [{"tile": int(t)} if int(t) else None for t in args.c5_tiles.split(",")]
+            net.set_tiles(d_x.shape, tiles, algo=algo)
         macs, muls = 0.0, 0.0
         H, W = x.shape[2], x.shape[3]
         for L, tile in zip(layers, tiles):
@@ -519,8 +535,9 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         def step():
             net.forward(d_x, algo=algo)
         launches_per_step = 2 * 9       # nine layers of two launches (packing + layer; the four pools run inside their layers)
-        name = ("c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head; tile shapes timed once at set-up "
-                "(tuned: %s)" % (x.shape[0], [t["tile"] if t else None for t in tiles]))
+        name = ("c5: compact 4-bit CNN, batch %d, 3x160x320, 8 conv3x3 + 4 pools + 1x1 head; tiles %s: %s"
+                % (x.shape[0], {"tune": "timed once at set-up", "auto": "the library's own"}.get(args.c5_tiles, "given"),
+                   [t["tile"] if t else None for t in tiles]))
         h2d = d_x.numel()
         d2h = x.shape[0] * 36 * H * W * 4
 
@@ -541,6 +558,8 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         total += e0.elapsed_time(e1)
     barrier()
     total = max_over_ranks(total)
+    if rank == 0:
+        sampler.keep_busy_until_sampled(step, torch.cuda.synchronize)
     clocks = sampler.stop() if rank == 0 else None
     ms = total / args.steps
     line = {
@@ -750,6 +769,9 @@ def main():
     ap.add_argument("--length", type=int, default=1 << 24, help="signal length of the sweep (benchmark value: 2^24)")
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"],
                     help="c2 = 1-D sweep (default, the benchmark step); c3/c4 = one 2-D layer; c5 = the compact CNN")
+    ap.add_argument("--c5-tiles", default="tune",
+                    help="c5 only: tune = time tile shapes once at set-up (default); auto = the library's own tiles; or the tile "
+                         "values of an earlier tuning pass, one per conv3x3 layer, comma-separated, 0 = automatic (for profiling)")
     ap.add_argument("--cases", default="", help="c2 only: comma-separated subset such as p4_K3_s,p8_K7_u (for profiling)")
     ap.add_argument("--case-copies", type=int, default=3, help="with --cases: buffer copies per case")
     ap.add_argument("--batch", type=int, default=0, help="c3/c4/c5: override the batch size (for profiling)")

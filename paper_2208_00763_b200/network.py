@@ -81,6 +81,12 @@ class CompactCnn:
         self._tiles[(algo, bool(fused_pool), tuple(d_x.shape))] = kept
         return kept
 
+    def set_tiles(self, shape, tiles: List[Optional[dict]], algo: int = hk.ALGO_PACKED32, fused_pool: bool = True) -> None:
+        """Tuning records found earlier (``tune_tiles``) for inputs of this shape, one per layer (None: automatic)."""
+        if len(tiles) != len(self.layers):
+            raise ValueError("one tuning record per layer")
+        self._tiles[(algo, bool(fused_pool), tuple(shape))] = list(tiles)
+
     def forward(self, d_x: torch.Tensor, algo: int = hk.ALGO_PACKED32, keep_activations: bool = False, stream=None,
                 fused_pool: bool = True):
         """``fused_pool``: layers followed by a pool run it inside their epilogue (``hikonv_conv2d_dense`` with one code
