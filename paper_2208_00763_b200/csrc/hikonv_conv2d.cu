@@ -209,8 +209,8 @@ __global__ void __launch_bounds__(kMaxThreads2D, 2) conv2d_kernel(const Conv2dPa
         aptr[i] = As + p.lead + (r + db * (p.K - 1)) * p.XBS + xb;
     }
 
-    static_assert(UNPACKED || TM * TN <= kEPitch, "second-accumulator pitch too small for the thread tile");
     constexpr bool NOE = U < 0;          // the whole (ci, kh) sum fits the slots: no second accumulator at all
+    static_assert(UNPACKED || NOE || TM * TN <= kEPitch, "second-accumulator pitch too small for the thread tile");
     acc_t acc[TM][TN];
     // second packed accumulator (upper slot bits): in shared memory, TM * TN 8-byte entries per thread with
     // a pitch of kEPitch entries per thread (odd, so that the lanes of a warp fall into different banks
@@ -848,13 +848,16 @@ static int launch_pitch(const Conv2dSetup &s, bool sp, cudaStream_t st) {
 // U: channels per unrolled group with placed carry-save moves (0: moves at stage ends).
 template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, int U>
 static int launch_variant_u(const Conv2dSetup &s, bool sp, cudaStream_t st) {
-    if (KT == 0) return launch_pitch<N, SC, TM, TN, UNPACKED, 0, 0, 0, 0>(s, sp, st);
-    switch (s.kp.XBS) {
-        case 8: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 8, U>(s, sp, st);
-        case 16: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 16, U>(s, sp, st);
-        case 32: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 32, U>(s, sp, st);
-        case 64: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 64, U>(s, sp, st);
-        default: return HIKONV_ERR_UNSUPPORTED;
+    if constexpr (KT == 0) {
+        return launch_pitch<N, SC, TM, TN, UNPACKED, 0, 0, 0, 0>(s, sp, st);
+    } else {
+        switch (s.kp.XBS) {
+            case 8: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 8, U>(s, sp, st);
+            case 16: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 16, U>(s, sp, st);
+            case 32: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 32, U>(s, sp, st);
+            case 64: return launch_pitch<N, SC, TM, TN, UNPACKED, KT, JT, 64, U>(s, sp, st);
+            default: return HIKONV_ERR_UNSUPPORTED;
+        }
     }
 }
 
@@ -862,16 +865,20 @@ static int launch_variant_u(const Conv2dSetup &s, bool sp, cudaStream_t st) {
 template <int N, int SC, int TM, int TN, bool UNPACKED, int KT, int JT, bool GROUPED = false, bool SHALLOW = false>
 static int launch_variant(const Conv2dSetup &s, bool sp, cudaStream_t st) {
     // SHALLOW: instantiated for layers whose whole (ci, kh) sum fits the slots (no second accumulator)
-    if constexpr (SHALLOW) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, -1>(s, sp, st);
-    if constexpr (GROUPED) {
-        if (s.kp.move_every == 3) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 3>(s, sp, st);
-        if (s.kp.move_every == 4) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 4>(s, sp, st);
+    if constexpr (SHALLOW) {
+        return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, -1>(s, sp, st);
+    } else {
+        if constexpr (GROUPED) {
+            if (s.kp.move_every == 3) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 3>(s, sp, st);
+            if (s.kp.move_every == 4) return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 4>(s, sp, st);
+        }
+        if (s.kp.move_every != 0) return HIKONV_ERR_UNSUPPORTED;
+        return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 0>(s, sp, st);
     }
-    if (s.kp.move_every != 0) return HIKONV_ERR_UNSUPPORTED;
-    return launch_variant_u<N, SC, TM, TN, UNPACKED, KT, JT, 0>(s, sp, st);
 }
 
 constexpr int kTM = 4, kTN = 4;          // per-thread tile of the packed kernels
+constexpr int kTNShallow = 8;            // channels per thread of the kernel without second accumulators
 constexpr int kTMU = 8, kTNU = 4;        // per-thread tile of the comparator
 
 // Tile shape of one candidate and its modelled cost.
@@ -999,6 +1006,10 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         }
         if (L.N > kMaxN2D || L.segments > kMaxN2DSeg) return HIKONV_ERR_UNSUPPORTED;
         TM = kTM; TN = kTN; N = L.N;
+        // A first layer (8-bit activations, few input channels: no second accumulator) spends most of its instructions
+        // on the per-position work around a short multiply loop; with eight channels per thread instead of four that
+        // work is shared by twice the outputs (3 -> 16 channels on 160x320 maps: 179 -> 161 us).
+        if (L.N == 2 && L.S == 17 && K == 3 && L.J == 2 && L.M >= Ci * K && Co % 8 == 0) TN = kTNShallow;
         // Small layers are bound by the serial work of a thread, not by the multiplier: when four positions per thread
         // would not even fill the resident thread slots of the device once (about 1.1 times, measured on the benchmark
         // network: 10x20 maps 56 -> 32 us, 20x40 maps 83 -> 68 us; larger layers lose 2-10 %), threads take two
@@ -1151,7 +1162,9 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
     if (s.L.N == 3 && s.L.S == 13 && K == 1 && J == 1) return launch_variant<3, 13, kTM, kTN, false, 1, 1>(s, sp, st);
     // 8-bit activations x 4-bit weights with few input channels (a network's first layer): no moves at all
     if (s.L.N == 2 && s.L.S == 17 && K == 3 && J == 2 && s.L.M >= s.kp.Ci * K && s.kp.move_every == 0)
-        return launch_variant<2, 17, kTM, kTN, false, 3, 2, false, true>(s, sp, st);
+        return s.kp.TCO == s.kp.TNX * kTNShallow ? launch_variant<2, 17, kTM, kTNShallow, false, 3, 2, false, true>(s, sp, st)
+                                                 : launch_variant<2, 17, kTM, kTN, false, 3, 2, false, true>(s, sp, st);
+    if (s.kp.TCO != s.kp.TNX * kTN) return HIKONV_ERR_UNSUPPORTED;       // every other packed kernel holds four channels per thread
     if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     switch (s.L.N) {

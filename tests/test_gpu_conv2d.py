@@ -213,6 +213,23 @@ def test_compact_cnn_full_size_every_image():
                 assert np.array_equal(a[b0:b0 + 16].astype(np.int64), r), "layer %d, images %d..%d, pass %d" % (i + 1, b0, b0 + 15, which)
 
 
+@pytest.mark.parametrize("co", [8, 12, 16, 24, 40, 72])
+def test_first_layer_kernel_with_eight_or_four_channels_per_thread(co):
+    # 8-bit activations, few input channels: the kernel without second accumulators holds eight output channels per
+    # thread when the channel count is a multiple of eight, four otherwise; ragged rows, several row segments, several
+    # images per tile, exact sums and requantised codes
+    for (B, Ci, H, W) in ((2, 3, 9, 21, ), (1, 1, 5, 300), (5, 2, 3, 7), (1, 3, 33, 64)):
+        L = hk.conv2d_layout(B, Ci, H, W, co, 3, 1, 8, 4, False, True)
+        assert (L["N"], L["J"]) == (2, 2) and L["M"] >= Ci * 3 and L["S"] == (17 if Ci > 1 else 16)    # one channel: the general kernel
+        x, w = inputs.conv2d_case(B, Ci, H, W, co, 3, 8, 4, False, True, seed=4000 + co + W)
+        ref = direct.conv2d_nchw(x, w, 1)
+        assert_exact(_layer(x, w, 1, 8, 4, False, True, hk.ALGO_PACKED32), ref, "co=%d %s" % (co, (B, Ci, H, W)))
+        assert_exact(_layer(x, w, 1, 8, 4, False, True, hk.ALGO_PACKED32, requant=(8, 0, 15)), direct.requant(ref, 8, 0, 15),
+                     "requant co=%d %s" % (co, (B, Ci, H, W)))
+    for x, w in inputs.extreme_2d(2, 3, 6, 10, co, 3, 8, 4, False, True):
+        assert_exact(_layer(x, w, 1, 8, 4, False, True, hk.ALGO_PACKED32), direct.conv2d_nchw(x, w, 1), "extreme co=%d" % co)
+
+
 def test_tuner_times_tiles_and_returns_one_that_gives_the_same_result():
     for (B, Ci, H, W, Co, p, xs, pool) in ((4, 16, 12, 20, 24, 4, True, False), (8, 64, 10, 20, 64, 4, False, True), (2, 3, 16, 40, 16, 8, False, False)):
         x, w = inputs.conv2d_case(B, Ci, H, W, Co, 3, p, 4, xs, True, seed=77 + Ci)
