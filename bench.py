@@ -727,6 +727,25 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
         out[name] = rec
         del d_x, d_w, o
 
+    # the C3 layer shape at every bitwidth p = q = 1 .. 8 (signed codes, exact int32 sums): packed against one product per multiply
+    by_bits = {}
+    B, Ci, H, W, Co = 32, 64, 56, 56, 64
+    for p in range(1, 9):
+        x, w = inputs.conv2d_case(B, Ci, H, W, Co, 3, p, p, True, True, seed=40 + p)
+        d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
+        d_w = torch.from_numpy(inputs.to_storage(w)).to(dev)
+        ws = torch.empty(hk.conv2d_workspace_bytes(B, Ci, H, W, Co, 3, 1), dtype=torch.uint8, device=dev)
+        o = torch.empty((B, Co, H, W), dtype=torch.int32, device=dev)
+        row = {}
+        for key, algo in (("packed", hk.ALGO_PACKED32), ("unpacked", hk.ALGO_UNPACKED_IMAD)):
+            row[key + "_ms"] = time_fn(lambda: hk.conv2d(d_x, d_w, 1, p, p, True, True, algo=algo, workspace=ws, out=o), iters=5)
+        L = hk.conv2d_layout(B, Ci, H, W, Co, 3, 1, p, p, True, True)
+        row["unpacked_over_packed"] = row["unpacked_ms"] / row["packed_ms"]
+        row["layout"] = {k: L[k] for k in ("N", "S", "J", "M")}
+        by_bits["p%d" % p] = row
+        del d_x, d_w, o, ws
+    out["c3_shape_by_bitwidth"] = by_bits
+
     x, layers, head_w = inputs.c5_network()
     d_x = torch.from_numpy(inputs.to_storage(x)).to(dev)
     net = network.CompactCnn(layers, head_w, device=dev)

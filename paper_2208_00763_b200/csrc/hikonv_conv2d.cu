@@ -1165,8 +1165,15 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
         return s.kp.TCO == s.kp.TNX * kTNShallow ? launch_variant<2, 17, kTM, kTNShallow, false, 3, 2, false, true>(s, sp, st)
                                                  : launch_variant<2, 17, kTM, kTN, false, 3, 2, false, true>(s, sp, st);
     if (s.kp.TCO != s.kp.TNX * kTN) return HIKONV_ERR_UNSUPPORTED;       // every other packed kernel holds four channels per thread
+    // 1- and 2-bit codes: four pixels per word, the whole 3x3 kernel row in one word
+    if (s.L.N == 4 && K == 3 && J == 1)
+        return (s.L.M >= s.kp.Ci * K && s.kp.move_every == 0) ? launch_variant<4, 0, kTM, kTN, false, 3, 1, false, true>(s, sp, st)
+                                                              : launch_variant<4, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
+    // pointwise layers at the other widths
+    if (s.L.N == 4 && K == 1 && J == 1) return launch_variant<4, 0, kTM, kTN, false, 1, 1>(s, sp, st);
+    if (s.L.N == 2 && K == 1 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 1, 1>(s, sp, st);
     switch (s.L.N) {
         case 1: return launch_variant<1, 0, kTM, kTN, false, 0, 0>(s, sp, st);
         case 2: return launch_variant<2, 0, kTM, kTN, false, 0, 0>(s, sp, st);

@@ -47,11 +47,14 @@ def test_layer_shapes(shape, algo):
 
 @pytest.mark.parametrize("bits", range(1, 9))
 def test_every_bitwidth(bits):
+    # 3x3 and pointwise layers; shallow (no carry-save moves) and deep enough to need them
     for signed in (False, True):
-        x, w = inputs.conv2d_case(2, 10, 7, 13, 12, 3, bits, bits, signed, signed, seed=bits)
-        ref = direct.conv2d_nchw(x, w, 1)
-        for algo in ALGOS:
-            assert_exact(_layer(x, w, 1, bits, bits, signed, signed, algo), ref, "bits=%d signed=%d algo=%d" % (bits, signed, algo))
+        for (Ci, K, pad) in ((10, 3, 1), (10, 1, 0), (150, 3, 1), (150, 1, 0)):
+            x, w = inputs.conv2d_case(2, Ci, 7, 13, 12, K, bits, bits, signed, signed, seed=bits + Ci + K)
+            ref = direct.conv2d_nchw(x, w, pad)
+            for algo in ALGOS:
+                assert_exact(_layer(x, w, pad, bits, bits, signed, signed, algo), ref,
+                             "bits=%d signed=%d Ci=%d K=%d algo=%d" % (bits, signed, Ci, K, algo))
 
 
 @pytest.mark.parametrize("n", [1, 2, 3, 4])
