@@ -987,18 +987,22 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         int rc = make_layout(p, q, xs, ws, K, 2, Ci * K, Wo, tune, &L);
         if (rc != HIKONV_OK) return rc;
         // Unsigned activations against signed weights: the products of codes x - 2^(p-1) span about half the range,
-        // so a slot takes nearly twice as many of them between two carry-save moves.  Layers whose signed layout
-        // allows at least half again as many products run on the shifted codes and get
+        // so a slot takes nearly twice as many of them between two carry-save moves, or a word one more pixel (5-bit
+        // codes: three instead of two).  Layers whose signed layout is cheaper by the estimate below run on the shifted codes and get
         // 2^(p-1) * (sum of the channel's weights) added back in the epilogue: from 128 input channels on always
         // (measured: 256 channels on 14x14 maps 239 -> 218 us), from 32 on when the layer is large enough to keep four
         // positions per thread (32 channels on 40x80 maps 112 -> 106 us; the 64-channel layers on 10x20 maps, bound by
         // the latency of one thread's work, lose 2 us to the longer packing launch and keep their own codes).
         const double threads4_own = (double)B * Ho * (ceil_div(Wo, L.N) + L.J) / kTM * ceil_div(Co, kTN);
         const bool small_layer = threads4_own <= 1.1 * sm_count() * 2 * kMaxThreads2D;
-        if (!xs && ws && L.M < Ci * K && (Ci >= 128 || (Ci >= 32 && !small_layer))) {
+        if (!xs && ws) {
             hikonv_layout_t Ls;
-            if (make_layout(p, q, 1, ws, K, 2, Ci * K, Wo, tune, &Ls) == HIKONV_OK && Ls.N >= L.N && Ls.J <= L.J &&
-                2 * Ls.M >= 3 * L.M) {
+            // issue cycles per pixel and (ci, kh) pair: J multiplies of about four cycles and, every M pairs, a move of
+            // about thirteen, shared by the N pixels of a word; the shifted codes are taken for a gain of 7 % or more,
+            // always when they put more pixels into a word, else under the depth conditions above
+            auto cycles = [&](const hikonv_layout_t &l) { return (l.J * 4.1 + 13.0 / std::min(l.M, Ci * K)) / l.N; };
+            if (make_layout(p, q, 1, ws, K, 2, Ci * K, Wo, tune, &Ls) == HIKONV_OK && cycles(Ls) <= 0.93 * cycles(L) &&
+                (Ls.N > L.N || (L.M < Ci * K && (Ci >= 128 || (Ci >= 32 && !small_layer))))) {
                 L = Ls;
                 xs = 1;
                 kp.x_off = 1 << (p - 1);
@@ -1169,7 +1173,9 @@ static int launch_conv2d(const Conv2dSetup &s, cudaStream_t st) {
     if (s.L.N == 4 && K == 3 && J == 1)
         return (s.L.M >= s.kp.Ci * K && s.kp.move_every == 0) ? launch_variant<4, 0, kTM, kTN, false, 3, 1, false, true>(s, sp, st)
                                                               : launch_variant<4, 0, kTM, kTN, false, 3, 1>(s, sp, st);
-    if (s.L.N == 2 && K == 3 && J == 2) return launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
+    if (s.L.N == 2 && K == 3 && J == 2)
+        return (s.L.M >= s.kp.Ci * K && s.kp.move_every == 0) ? launch_variant<2, 0, kTM, kTN, false, 3, 2, false, true>(s, sp, st)
+                                                              : launch_variant<2, 0, kTM, kTN, false, 3, 2>(s, sp, st);
     if (s.L.N == 2 && K == 3 && J == 1) return launch_variant<2, 0, kTM, kTN, false, 3, 1>(s, sp, st);
     // pointwise layers at the other widths
     if (s.L.N == 4 && K == 1 && J == 1) return launch_variant<4, 0, kTM, kTN, false, 1, 1>(s, sp, st);

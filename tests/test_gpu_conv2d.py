@@ -91,7 +91,7 @@ def test_carry_save_schedules(ci):
             assert_exact(_layer(x, w, 1, 4, 4, False, True, hk.ALGO_PACKED32, tune=tune), direct.conv2d_nchw(x, w, 1), "extreme ci=%d" % ci)
 
 
-@pytest.mark.parametrize("p", [1, 2, 3, 4, 6, 8])
+@pytest.mark.parametrize("p", [1, 2, 3, 4, 5, 6, 8])
 def test_deep_unsigned_layers_on_shifted_codes(p):
     # unsigned activations x signed weights with 128 or more input channels may be packed as x - 2^(p-1) (the padding
     # included) and get 2^(p-1) * (the channel's weight sum) back in the epilogue: image borders, valid convolution,
