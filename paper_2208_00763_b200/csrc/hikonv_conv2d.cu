@@ -1078,14 +1078,21 @@ static int make_setup(int B, int Ci, int H, int W, int Co, int K, int stride, in
         const int CF = L.M / K;
         int U = 0;
         if (L.N == 3 && L.S == 13 && K == 3 && L.J == 1 && !(tune && tune->tile < 0)) U = CF >= 6 ? 0 : CF >= 4 ? 4 : CF == 3 ? 3 : 0;
-        if (U > 0 && (ceil_div(Ci, U) > (1 << L.carry_bits) || ck_cap < U)) U = 0;
+        if (U > 0 && ck_cap < U) U = 0;
         if (U > 0) {
-            kp.move_every = U;
             CK = ck_cap / U * U;
             // a stage's activation pieces should fit the per-thread copy descriptors (kPieces each): small CTAs
             // stage one group at a time
             const int pieces_per_channel = kp.NRmax * ((kp.XB + 3) / 4);
             while (CK > U && CK * pieces_per_channel > kCopyPieces * s->threads) CK -= U;
+            // every group of every stage moves once, the zero-weight channels that fill the last stage included
+            if (ceil_div(Ci, CK) * (CK / U) > (1 << L.carry_bits)) {
+                U = 0;
+                CK = std::min(ck_cap, Ci);
+            }
+        }
+        if (U > 0) {
+            kp.move_every = U;
         } else {
             int fc = 1;
             const int eff = pick_chunking(CF, Ci, &CK, &fc, ck_cap);
