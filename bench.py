@@ -52,6 +52,14 @@ NCU_TRAFFIC = {
 }
 
 
+# Warp instructions one launch of the packed layer kernel executes (smsp__inst_executed.sum of the captures behind
+# profiles/conv2d_kernel_c3.txt and _c4.txt), for the issue model of the 2-D rooflines; void when the source changes.
+NCU_INSTRUCTIONS = {
+    "c3": {"sha256": "dd5f48402620b0de3ccab755f40e1210a87800596c3d25131297b506941b6beb", "warp_instructions": 41575448.0},
+    "c4": {"sha256": "dd5f48402620b0de3ccab755f40e1210a87800596c3d25131297b506941b6beb", "warp_instructions": 87595968.0},
+}
+
+
 def _source_hash(name: str) -> str:
     with open(os.path.join(ROOT, "paper_2208_00763_b200", "csrc", name), "rb") as fh:
         return hashlib.sha256(fh.read()).hexdigest()
@@ -293,6 +301,7 @@ def run_ours(args):
         pure, mixed = (peaks[k]["lanes_per_clk_per_sm_at_max_clock"] for k in ("mad_wide_u32", "mad_wide_with_logic"))
         peaks["issue_model"] = {"cycles_per_wide_multiply_add": 128.0 / pure,
                                 "cycles_added_per_other_instruction": 2.0 * (128.0 / mixed - 128.0 / pure)}
+        imad_peak["issue"] = dict(peaks["issue_model"], schedulers=4 * sms, clock_hz=sm_max_mhz * 1e6)
         imad_peak["packed_measured"] = max(peaks["mad_wide_u32"]["T_per_s"], peaks["mad_wide_s32"]["T_per_s"]) * 1e12
         imad_peak["unpacked_measured"] = peaks["mad_lo_s32"]["T_per_s"] * 1e12
 
@@ -571,7 +580,7 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
         "gpu_launches": args.steps * launches_per_step, "clocks": clocks,
     }
     if muls is not None:
-        line["roofline"] = alu_roofline(muls, ms, imad_peak, args.algo)
+        line["roofline"] = alu_roofline(muls, ms, imad_peak, args.algo, args.workload)
         line["roofline"]["kernel"] = "conv2d_kernel" + (" (nine layer launches, multiplies summed)" if args.workload == "c5" else "")
     if rank == 0:
         print(json.dumps(line), flush=True)
@@ -579,7 +588,7 @@ def run_layer_main(args, torch, np, ranks, hk, inputs, network, dev, world, rank
     return 0
 
 
-def alu_roofline(muls: float, ms: float, imad_peak: dict, key: str) -> dict:
+def alu_roofline(muls: float, ms: float, imad_peak: dict, key: str, workload: str = None) -> dict:
     """Multiplies executed per second against the rate of that multiply: `peak` is the rate the library's own
     register-only kernel reached on this GPU (hikonv_pipe_rate) when it was measured, `frac_of_derived` divides by
     SMs x lanes per clock x maximum SM clock instead.  The step also holds the packing kernel of the layer."""
@@ -587,10 +596,22 @@ def alu_roofline(muls: float, ms: float, imad_peak: dict, key: str) -> dict:
     derived = imad_peak[key]
     measured = imad_peak.get(key + "_measured")
     peak = measured if measured else derived
-    return {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "T multiply-add/s",
-            "frac": achieved / peak, "traffic": None,
-            "peak_kind": "of measured (register-only multiply-add kernel, this run)" if measured else "of derived",
-            "frac_of_derived": achieved / derived, "derived_peak": derived / 1e12}
+    out = {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "T multiply-add/s",
+           "frac": achieved / peak, "traffic": None,
+           "peak_kind": "of measured (register-only multiply-add kernel, this run)" if measured else "of derived",
+           "frac_of_derived": achieved / derived, "derived_peak": derived / 1e12}
+    # Issue model: a scheduler spends the measured cycles on every warp-wide multiply-add and on every other warp
+    # instruction of the layer kernel (counted under ncu); the sum over the device's schedulers is the time the layer
+    # kernel cannot go below with this instruction mix, to be read against the step (which also holds the packing launch).
+    rec, issue = NCU_INSTRUCTIONS.get(workload or ""), imad_peak.get("issue")
+    if key == "packed" and rec and issue and rec["sha256"] == _source_hash("hikonv_conv2d.cu"):
+        mads = muls / 32.0
+        others = rec["warp_instructions"] - mads
+        cycles = issue["cycles_per_wide_multiply_add"] * mads + issue["cycles_added_per_other_instruction"] * others
+        out["issue_model"] = {"wide_multiply_add_warp_instructions": mads, "other_warp_instructions": others,
+                              "modelled_layer_kernel_ms": cycles / (issue["schedulers"] * issue["clock_hz"]) * 1e3,
+                              "multiply_share_of_modelled_cycles": issue["cycles_per_wide_multiply_add"] * mads / cycles}
+    return out
 
 
 def small_case(torch, hk, inputs, dev):
@@ -708,7 +729,7 @@ def layer_workloads(torch, np, hk, inputs, network, dev, imad_peak):
                                            requant=rq, algo=algo, workspace=ws, out=o))
             muls = hk.conv2d_multiplies(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
                                         shape["p"], shape["q"], shape["x_signed"], shape["w_signed"], algo)
-            rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key)}
+            rec[key] = {"ms": ms, "value": macs / (ms * 1e-3), "unit": UNIT, "roofline": alu_roofline(muls, ms, imad_peak, key, name)}
         rec["layout"] = hk.conv2d_layout(shape["B"], shape["Ci"], shape["H"], shape["W"], shape["Co"], shape["K"], shape["pad"],
                                          shape["p"], shape["q"], shape["x_signed"], shape["w_signed"])
         rec["packed_over_unpacked"] = rec["unpacked"]["ms"] / rec["packed"]["ms"]
