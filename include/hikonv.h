@@ -236,8 +236,8 @@ int hikonv_conv1d_host(const int8_t *h_f, size_t len, const int8_t *h_g, int K, 
  * int32 copies of the weights and codes.
  * stride must be 1 and 0 <= pad < K.  Limits (HIKONV_ERR_UNSUPPORTED beyond them): Ho < 60000; B Ci H W and B Ho
  * below 2^31; (images a tile of rows can touch + 1) x Co x Ho x Wo below 2^32 (output offsets inside a CTA are 32-bit).
- * Layers with unsigned activations, signed weights and 32 or more input channels may run on activation codes shifted
- * by 2^(p-1) (see hikonv_conv2d_layout); results are the same exact sums.
+ * Layers with unsigned activations and signed weights may run on activation codes shifted by 2^(p-1) where that
+ * saves carry-save moves or puts one more pixel into a word (see hikonv_conv2d_layout); results are the same exact sums.
  */
 int hikonv_conv2d(const int8_t *d_x, int B, int Ci, int H, int W, const int8_t *d_w, int Co, int K,
                   int stride, int pad, int p, int q, int x_signed, int w_signed, void *d_out,
@@ -266,7 +266,8 @@ int hikonv_conv2d_tune(const void *d_x, int x_store_bits, int B, int Ci, int H, 
  * hikonv_conv2d_layout - the packed layout hikonv_conv2d(HIKONV_ALGO_PACKED32) runs this layer with (host only).
  * *out: N, S, Kc, J, slots, M (accumulated (ci, kh) pairs between two carry-save moves), as hikonv_layout reports them.
  * *x_shift (may be NULL): 0, or 2^(p-1) when the layer runs its unsigned activations as signed codes x - 2^(p-1):
- * the span of a product halves, a slot takes about twice as many products between moves, and the epilogue adds
+ * the span of a product halves, a slot takes about twice as many products between moves (or the word one more
+ * pixel), and the epilogue adds
  * 2^(p-1) x (sum of the output channel's weights) back.  *out is then the layout for signed activations, which is
  * not what hikonv_layout reports for the layer's own signs.  Arguments and errors as for hikonv_conv2d.
  */
